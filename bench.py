@@ -1,0 +1,370 @@
+#!/usr/bin/env python
+"""Benchmark of the DP-SGD privatised-gradient step at BERT-Large shapes.
+
+One step = one microbatch of 256 examples x 128 tokens through the whole path on one GPU:
+per-example norms over 24 encoder blocks + the token embedding -> clip factors -> clipped accumulate
+-> fused noise + scaling + AdamW over ~334M fp32 parameters.  Inputs are seeded and synthetic and
+stay resident in HBM (32 GB per microbatch, far larger than L2, so no flush is needed).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W]          device-timed line (+ e2e, roofline, cpu_baseline)
+  python bench.py --impl reference ...                         the CPU checker timed on the host cores
+
+Under torchrun (N > 1) each rank processes its own microbatches (weak scaling); the accumulators are
+reduce-scattered once per step, the noise/AdamW pass runs on the local shard and theta is all-gathered.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "dp_sgd_examples_per_s_bert_large"
+UNIT = "examples/s"
+WORKLOAD = "bert_large"
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": p["hbm_gbs"], "tf_burst": p["bf16_tflops"], "tf_sustained": p["bf16_tflops_sustained"],
+                "source": "measured"}
+    return {"hbm_gbs": 6650.0, "tf_burst": 1590.0, "tf_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, device_index: int):
+        self.rows = []
+        self.proc = None
+        try:
+            uuid = str(torch.cuda.get_device_properties(device_index).uuid)
+            if not uuid.startswith("GPU-"):
+                uuid = "GPU-" + uuid
+            self.cmd = ["nvidia-smi", f"--id={uuid}", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                        "-lms", "100"]
+        except Exception:
+            self.cmd = None
+
+    def start(self):
+        if self.cmd is None:
+            return
+        try:
+            self.proc = subprocess.Popen(self.cmd, stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            f = [x.strip() for x in r.split(",")]
+            if len(f) < 8:
+                continue
+            try:
+                sm.append(float(f[0]))
+                mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, f[4:8]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def oracle_layers(data, rows):
+    from oracle import dp_oracle as O
+    out = []
+    for ld in data:
+        out.append(O.OracleLayer(kind=ld.spec.kind, G=ld.G[rows].double().cpu().numpy(),
+                                 A=None if ld.A is None else ld.A[rows].double().cpu().numpy(),
+                                 ids=None if ld.ids is None else ld.ids[rows].cpu().numpy().astype(np.int64),
+                                 has_bias=ld.spec.has_bias, vocab=ld.spec.d_in if ld.spec.kind == "embedding" else 0))
+    return out
+
+
+def time_oracle(wl, data, n_params, budget_s=15.0, max_examples=4):
+    """The CPU checker as it stands on a bounded sample: k examples through every layer (norms, clip,
+    accumulate) plus noise + AdamW on 1/64 of the parameters; scaled linearly to one 256-example step."""
+    from oracle import dp_oracle as O
+    t0 = time.perf_counter()
+    k = 0
+    accs = None
+    while k < max_examples:
+        ol = oracle_layers(data, slice(k, k + 1))
+        ta = time.perf_counter()
+        n = O.per_example_sqnorms(ol)
+        c = O.clip_factors(n, wl.C)
+        accs = O.zero_accumulators(ol) if accs is None else accs
+        O.clipped_accumulate(ol, c, accs)
+        per_ex = time.perf_counter() - ta
+        k += 1
+        if time.perf_counter() - t0 + per_ex > budget_s:
+            break
+    t_examples = time.perf_counter() - t0
+    # time only the arithmetic, not the device->host conversion of inputs
+    frac = 64
+    n_s = n_params // frac
+    S = np.zeros(n_s)
+    th = np.zeros(n_s)
+    tb = time.perf_counter()
+    g = O.add_noise_and_scale(S, wl.sigma, wl.C, wl.B, 0, 1, 0)
+    O.adamw_step(th, th, th, g, wl.lr, wl.beta1, wl.beta2, wl.xi, wl.weight_decay, 1)
+    t_update = (time.perf_counter() - tb) * frac
+    step_s = t_examples / k * wl.B + t_update
+    cores = len(os.sched_getaffinity(0)) if hasattr(os, "sched_getaffinity") else os.cpu_count()
+    threads = torch.get_num_threads()
+    return {"value": wl.B / step_s, "unit": UNIT, "cores": min(cores, threads) if threads else cores, "kind": "oracle",
+            "sample": f"{k} of {wl.B} examples through all {len(data)} layers (incl. host conversion of their "
+                      f"inputs) + noise/AdamW on 1/{frac} of {n_params} parameters, scaled linearly to one step "
+                      f"(extrapolated); measured {t_examples:.1f}s + {t_update / frac:.1f}s"}
+
+
+def run_reference(args):
+    """The reference arm: the CPU checker (numpy, fp64) on the host cores, same config and metric."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from paper_2108_01624_b200 import synth
+    wl = synth.workload(WORKLOAD)
+    n_params = wl.n_params()
+    data = synth.generate(wl, seed=0, device="cpu", B=4)
+    values = []
+    cb = None
+    for it in range(args.warmup + args.steps):
+        budget = 3.0 if it < args.warmup else max(4.0, 60.0 / max(1, args.steps))
+        cb = time_oracle(wl, data, n_params, budget_s=budget, max_examples=4)
+        if it >= args.warmup:
+            values.append(cb["value"])
+    v = float(np.mean(values)) if values else cb["value"]
+    cb["value"] = v
+    line = {"impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * wl.B / v, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": WORKLOAD, "B": wl.B, "T": wl.T, "layers": len(wl.specs), "params": n_params},
+            "cpu_baseline": cb,
+            "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--e2e-steps", type=int, default=2)
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+        return
+    args.warmup = max(args.warmup, 3)
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+
+    import paper_2108_01624_b200 as pkg
+    from paper_2108_01624_b200 import build as builder
+    from paper_2108_01624_b200 import synth
+    from paper_2108_01624_b200.parallel import ShardedUpdate
+    if rank == 0:
+        builder.build()
+    if dist is not None:
+        dist.barrier()
+
+    wl = synth.workload(WORKLOAD)
+    data = synth.generate(wl, seed=1000 + rank, device=dev)
+    step = pkg.DPStep(wl.specs, dev, wl.C, wl.sigma, wl.lr, wl.beta1, wl.beta2, wl.xi, wl.weight_decay, seed=0)
+    step.theta.copy_(synth.initial_weights(step.n_flat, 0, dev))
+    n_params = wl.n_params()
+    lin_idx = [k for k, sp in enumerate(wl.specs) if sp.kind == "linear"]
+    rest_idx = [k for k, sp in enumerate(wl.specs) if sp.kind != "linear"]
+    ll_all = step.layer_list(data)
+    ll_lin = pkg.LayerList([ll_all.layers[k] for k in lin_idx])
+    ll_rest = pkg.LayerList([ll_all.layers[k] for k in rest_idx])
+    ws = torch.empty(max(pkg.dp_workspace_bytes(ll_all), 256), dtype=torch.uint8, device=dev)
+    sq = torch.empty(wl.B, dtype=torch.float32, device=dev)
+    clip = torch.empty(wl.B, dtype=torch.float32, device=dev)
+    sharded = ShardedUpdate(step, dist, world, rank) if world > 1 else None
+    stream = torch.cuda.current_stream()
+
+    def one_step(ev=None):
+        if ev:
+            ev[0].record(stream)
+        pkg.dp_per_example_sqnorms(ll_all, sq, False, ws)
+        pkg.dp_clip_factors(sq, wl.C, clip)
+        if ev:
+            ev[1].record(stream)
+        pkg.dp_clipped_accumulate(ll_lin, clip, ws)
+        if ev:
+            ev[2].record(stream)
+        pkg.dp_clipped_accumulate(ll_rest, clip, ws)
+        if ev:
+            ev[3].record(stream)
+        step.examples_seen = wl.B * world
+        if sharded is None:
+            step.finish_macro_batch()
+        else:
+            sharded.finish_macro_batch()
+        if ev:
+            ev[4].record(stream)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        one_step()
+    barrier()
+    if pkg.dp_poll_status() != 0:
+        raise RuntimeError("device status not clean after warm-up")
+
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(args.steps)]
+    sampler = ClockSampler(local)
+    sampler.start()
+    l0 = pkg.dp_launch_count()
+    barrier()
+    t_start = torch.cuda.Event(enable_timing=True)
+    t_end = torch.cuda.Event(enable_timing=True)
+    t_start.record(stream)
+    for k in range(args.steps):
+        one_step(evs[k])
+    t_end.record(stream)
+    barrier()
+    launches = pkg.dp_launch_count() - l0
+    clocks = sampler.stop()
+    total_ms = t_start.elapsed_time(t_end)
+    if dist is not None:
+        t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    ms_per_step = total_ms / args.steps
+    value = wl.B * world / (ms_per_step * 1e-3)
+    phases = np.array([[e[i].elapsed_time(e[i + 1]) for i in range(4)] for e in evs]).mean(axis=0)
+
+    peaks = measured_peaks()
+    T, B = wl.T, wl.B
+    flops_acc = sum(2.0 * B * T * wl.specs[k].d_in * wl.specs[k].d_out for k in lin_idx)
+    ach_tf = flops_acc / (phases[1] * 1e-3) / 1e12
+    roofline = {"kernel": "clipped-accumulate GEMM (all linear layers, one call)", "bound": "tensor",
+                "achieved": ach_tf, "peak": peaks["tf_sustained"], "unit": "TFLOP/s",
+                "frac": ach_tf / peaks["tf_sustained"], "frac_of_burst": ach_tf / peaks["tf_burst"],
+                "peak_source": peaks["source"] + " (sustained bf16; kernel timed inside a long step)",
+                "traffic": None}
+    bytes_norm = sum(2.0 * B * T * (wl.specs[k].d_in + wl.specs[k].d_out) for k in lin_idx) \
+        + sum(2.0 * 2 * B * T * wl.specs[k].d_out for k in rest_idx if wl.specs[k].kind == "layernorm") \
+        + sum(2.0 * B * T * wl.specs[k].d_out + 4.0 * B * T for k in rest_idx if wl.specs[k].kind == "embedding")
+    bytes_upd = 32.0 * step.n_flat
+    extra = {
+        "norm_pass": {"bound": "hbm", "achieved": bytes_norm / (phases[0] * 1e-3) / 1e9, "peak": peaks["hbm_gbs"],
+                      "unit": "GB/s", "frac": bytes_norm / (phases[0] * 1e-3) / 1e9 / peaks["hbm_gbs"]},
+        "noise_adamw": {"bound": "hbm", "achieved": bytes_upd / (phases[3] * 1e-3) / 1e9, "peak": peaks["hbm_gbs"],
+                        "unit": "GB/s", "frac": bytes_upd / (phases[3] * 1e-3) / 1e9 / peaks["hbm_gbs"]},
+    }
+
+    e2e = None
+    if not args.no_e2e and world == 1:
+        e2e = run_e2e(pkg, wl, data, one_step, clip, stream, args.e2e_steps)
+    cpu_baseline = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        cpu_baseline = time_oracle(wl, data, n_params)
+
+    if rank == 0:
+        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+                "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+                "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+                "config": {"workload": WORKLOAD, "B": B, "T": T, "layers": len(wl.specs), "params": n_params,
+                           "microbatches_per_step": 1, "parallelism": f"dp{world}",
+                           "l2": "inputs (32 GB per microbatch) far exceed L2; no flush"},
+                "phases_ms": {"norms+clip": phases[0], "accumulate_linear": phases[1],
+                              "accumulate_ln_embedding": phases[2], "noise_adamw": phases[3]},
+                "roofline": roofline, "rooflines_other": extra, "cpu_baseline": cpu_baseline, "e2e": e2e,
+                "gpu_launches": int(launches), "clocks": clocks}
+        print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def run_e2e(pkg, wl, data, one_step, clip, stream, n_steps):
+    """Same step through the public API with HOST buffers: every step copies all layer inputs from pinned host
+    memory to the device and reads the clip factors back."""
+    host = []
+    try:
+        for ld in data:
+            host.append([None if t is None else torch.empty(t.shape, dtype=t.dtype, pin_memory=True).copy_(t)
+                         for t in (ld.A, ld.G, ld.ids)])
+        mirror = "full pinned mirror of every layer's inputs"
+    except RuntimeError:
+        host = None
+    if host is None:
+        return None
+    clip_h = torch.empty(clip.shape, dtype=clip.dtype, pin_memory=True)
+    h2d = sum(t.numel() * t.element_size() for h in host for t in h if t is not None)
+    d2h = clip_h.numel() * clip_h.element_size()
+
+    def e2e_step():
+        for ld, h in zip(data, host):
+            for dst, src in zip((ld.A, ld.G, ld.ids), h):
+                if dst is not None:
+                    dst.copy_(src, non_blocking=True)
+        one_step()
+        clip_h.copy_(clip, non_blocking=True)
+
+    e2e_step()
+    torch.cuda.synchronize()
+    a, b_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record(stream)
+    for _ in range(n_steps):
+        e2e_step()
+        stream.synchronize()
+    b_.record(stream)
+    torch.cuda.synchronize()
+    ms = a.elapsed_time(b_) / n_steps
+    return {"value": wl.B / (ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
+            "ms_per_step": ms, "steps": n_steps, "host_buffers": mirror}
+
+
+if __name__ == "__main__":
+    main()

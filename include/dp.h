@@ -1,0 +1,142 @@
+/*
+ * dp.h -- C ABI of the B200 (sm_100a) DP-SGD privatised-gradient step.
+ *
+ * The library implements the update of Algorithm 1 of "Large-Scale Differentially
+ * Private BERT" (arXiv 2108.01624): per-example clipping of the whole-model gradient,
+ * summation over the (micro)batches of a mega-batch (Section 5.3), one Gaussian draw
+ * N(0, sigma^2 C^2 I) per macro-batch, division by the batch size, and the Adam update
+ * with decoupled weight decay.  Per-example gradients are never written to memory:
+ * a layer is described by its per-token inputs A and output-gradients G (Section 4.3:
+ * the gradient of a fully connected layer is grad_s * x^T, summed over tokens).
+ *
+ * Conventions for every entry point
+ *   - All data pointers are DEVICE pointers owned by the caller, unless marked HOST.
+ *     The `layers` descriptor array itself is a HOST array and is read during the call.
+ *   - Calls only enqueue work on `cuda_stream` (a cudaStream_t passed as void*; NULL is
+ *     the default stream).  They do not synchronise the host, except dp_poll_status.
+ *   - The library allocates no device memory.  Kernels that need scratch take it from the
+ *     caller's `workspace` (size from dp_workspace_bytes, 256-byte aligned).  The contents
+ *     of the workspace carry no meaning between calls.
+ *   - Return value: DP_OK (0) or a negative dp_status.  Arguments are validated on the
+ *     host before anything is launched; nothing throws, aborts or traps.
+ *   - Matrices are row-major with the feature index fastest.  bf16 tensors must be
+ *     16-byte aligned; accumulators and optimizer state are fp32.
+ *   - G must be the gradient of the PER-EXAMPLE loss (no 1/B folded in), because the clip
+ *     of Algorithm 1 acts on grad L(theta; x_j) of a single example.
+ */
+#ifndef DP_B200_H_
+#define DP_B200_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define DP_API __attribute__((visibility("default")))
+#else
+#define DP_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  DP_OK = 0,
+  DP_ERR_ARG = -1,         /* null pointer, non-positive size, non-finite scalar, bad enum */
+  DP_ERR_ALIGN = -2,       /* pointer not aligned as required */
+  DP_ERR_UNSUPPORTED = -3, /* valid request this build cannot run (e.g. forced path on a shape it excludes) */
+  DP_ERR_CUDA = -4,        /* a CUDA runtime/driver call failed */
+  DP_ERR_TIMEOUT = -5,     /* a bounded device-side wait ran out (reported by dp_poll_status) */
+  DP_ERR_WORKSPACE = -6,   /* workspace missing, misaligned or too small */
+  DP_ERR_BAD_ID = -7       /* a token id outside [0, V) was met and skipped (dp_poll_status) */
+} dp_status;
+
+typedef enum { DP_LINEAR = 0, DP_LAYERNORM = 1, DP_EMBEDDING = 2 } dp_kind;
+typedef enum { DP_F32 = 0, DP_BF16 = 1 } dp_dtype;
+/* How a layer's per-example squared norm is obtained.
+ *   GRAM          <A_i A_i^T (+ 1 1^T with a bias), G_i G_i^T>  over T x T token Grams;
+ *                 for an embedding the first factor is the token-id equality mask.
+ *   MATERIALIZED  tiles of A_i^T G_i formed on chip, squared and summed; for an embedding,
+ *                 rows with equal ids are summed first.
+ *   AUTO          GRAM iff T * (d_in + d_out) < d_in * d_out, the flop count of either way. */
+typedef enum { DP_PATH_AUTO = 0, DP_PATH_GRAM = 1, DP_PATH_MATERIALIZED = 2 } dp_path;
+
+/* One trainable layer of one microbatch.  B and T must be equal across the layers of a call. */
+typedef struct dp_layer {
+  int32_t kind;      /* dp_kind */
+  int32_t dtype;     /* dp_dtype of A and G */
+  int32_t path;      /* dp_path (norms only; ignored for LAYERNORM) */
+  int32_t has_bias;  /* LINEAR: a bias [d_out] is trained and acc_b is given */
+  int32_t B, T;      /* examples in the microbatch, tokens per example */
+  int32_t d_in;      /* LINEAR: input width.  LAYERNORM: d (= d_out).  EMBEDDING: vocabulary size V */
+  int32_t d_out;     /* width of G */
+  const void* A;     /* LINEAR: [B,T,d_in] layer input.  LAYERNORM: [B,T,d] normalised input.  EMBEDDING: NULL */
+  const int32_t* ids;/* EMBEDDING: [B,T] token ids, 0 <= id < V.  Otherwise NULL */
+  const void* G;     /* [B,T,d_out] output-gradient of the per-example loss */
+  float* acc_w;      /* LINEAR: [d_in,d_out] = sum_i c_i A_i^T G_i.  LAYERNORM: gain [d].  EMBEDDING: [V,d_out].
+                        Accumulated in place (+=).  May be NULL for dp_per_example_sqnorms. */
+  float* acc_b;      /* LINEAR with bias: [d_out].  LAYERNORM: bias [d].  Otherwise NULL */
+} dp_layer;
+
+/* Bytes of scratch that dp_per_example_sqnorms / dp_clipped_accumulate need for these layers. */
+DP_API size_t dp_workspace_bytes(const dp_layer* layers /*HOST*/, int n_layers);
+
+/* Squared L2 norm of every example's whole gradient over the given layers (Algorithm 1 clips
+ * grad L(theta; x_j) as one vector; Section 4.3 gives the per-layer form).
+ *   sqnorm[B] fp32.  accumulate_into = 0: overwritten; 1: added to (so a model can be passed
+ *   in several calls).  The per-layer path follows dp_layer.path. */
+DP_API int dp_per_example_sqnorms(const dp_layer* layers /*HOST*/, int n_layers, float* sqnorm, int accumulate_into,
+                           void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* c_i = min(1, C / sqrt(sqnorm_i)), c_i = 1 when sqnorm_i = 0: the factor of clip(., C) in
+ * Algorithm 1.  C > 0. */
+DP_API int dp_clip_factors(const float* sqnorm, int B, float C, float* clip, void* cuda_stream);
+
+/* acc += sum_i clip_i * g_i for every layer: the sum of clipped gradients of Algorithm 1,
+ * accumulated over microbatches as in Section 5.3.  clip[B] fp32 from dp_clip_factors. */
+DP_API int dp_clipped_accumulate(const dp_layer* layers /*HOST*/, int n_layers, const float* clip,
+                          void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* acc <- (acc + sigma * C * z) / batch_size in place, z ~ N(0, I): the g_t line of Algorithm 1.
+ * z_e depends only on (seed, step, e) with e = elem_offset + index: Philox4x32-10 block e >> 2 with
+ * counter (lo(e>>2), hi(e>>2), lo(step), hi(step)) and key (lo(seed), hi(seed)); Box-Muller on the word
+ * pairs (x0,x1), (x2,x3).  n >= 0 elements; sigma >= 0, C > 0, batch_size > 0. */
+DP_API int dp_add_noise_and_scale(float* acc, int64_t n, int64_t elem_offset, float sigma, float C,
+                           int64_t batch_size, uint64_t seed, uint64_t step, void* cuda_stream);
+
+/* Adam with bias correction and decoupled weight decay (Algorithm 1):
+ *   m <- b1 m + (1-b1) g;  v <- b2 v + (1-b2) g^2;
+ *   theta <- theta - lr * ( (m/(1-b1^t)) / (sqrt(v/(1-b2^t)) + xi) + weight_decay * theta ),  t >= 1.
+ * The bias corrections are formed on the host in double precision. */
+DP_API int dp_adamw_step(float* theta, float* m, float* v, const float* g, int64_t n, float lr, float beta1,
+                  float beta2, float xi, float weight_decay, int64_t t, void* cuda_stream);
+
+/* The two calls above in one pass over memory (same arithmetic, same Philox indexing): reads acc, theta,
+ * m, v and writes theta, m, v; with zero_acc != 0 it also clears acc for the next macro-batch. */
+DP_API int dp_noise_scale_adamw_step(float* theta, float* m, float* v, float* acc, int zero_acc, int64_t n,
+                              int64_t elem_offset, float sigma, float C, int64_t batch_size, uint64_t seed,
+                              uint64_t step, float lr, float beta1, float beta2, float xi, float weight_decay,
+                              int64_t t, void* cuda_stream);
+
+/* Test utility: out[k] = the raw Philox word of element elem_offset + k (lane (e & 3) of block e >> 2). */
+DP_API int dp_philox_u32(uint32_t* out, int64_t n_words, int64_t elem_offset, uint64_t seed, uint64_t step,
+                  void* cuda_stream);
+
+/* Test utility: mask[i,t,s] = (ids[i,t] == ids[i,s]) as bytes, the first factor of the embedding Gram. */
+DP_API int dp_token_equality_mask(const int32_t* ids, int B, int T, uint8_t* mask, void* cuda_stream);
+
+/* Waits for the stream, then returns and clears the sticky device-side status (DP_OK, DP_ERR_TIMEOUT
+ * or DP_ERR_BAD_ID).  Device code never traps: a wait that runs out or an id out of range is recorded
+ * here and the offending work is skipped. */
+DP_API int dp_poll_status(void* cuda_stream);
+
+/* Number of kernels this library has launched in the calling process so far (host-side counter). */
+DP_API long long dp_launch_count(void);
+
+DP_API const char* dp_status_string(int status);
+DP_API int dp_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DP_B200_H_ */

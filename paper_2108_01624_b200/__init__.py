@@ -1,0 +1,12 @@
+"""B200-native DP-SGD privatised-gradient step (per-example clip, accumulate, noise, AdamW).
+
+The compute lives in libdp_b200.so (hand-written sm_100a CUDA behind the C ABI of include/dp.h);
+`binding` marshals torch tensors into it and `step` strings the calls into a macro-step.
+Importing the package does not load the library; the first call does, and fails loudly if it is absent.
+"""
+from . import binding, synth  # noqa: F401
+from .binding import (DP_PATH_AUTO, DP_PATH_GRAM, DP_PATH_MATERIALIZED, DpError, Layer, LayerList,  # noqa: F401
+                      alloc_workspace, dp_adamw_step, dp_add_noise_and_scale, dp_clip_factors,
+                      dp_clipped_accumulate, dp_noise_scale_adamw_step, dp_per_example_sqnorms, dp_philox_u32,
+                      dp_launch_count, dp_poll_status, dp_token_equality_mask, dp_version, dp_workspace_bytes)
+from .step import DPStep  # noqa: F401

@@ -1,0 +1,233 @@
+"""ctypes binding of libdp_b200.so: the same entry points as include/dp.h, taking torch tensors.
+
+Argument marshalling only -- every step runs in the library's CUDA kernels.  There is no CPU or
+PyTorch fallback: if the shared library is missing or a call fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from dataclasses import dataclass
+from typing import List, Optional, Sequence
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libdp_b200.so")
+
+DP_OK = 0
+DP_LINEAR, DP_LAYERNORM, DP_EMBEDDING = 0, 1, 2
+DP_F32, DP_BF16 = 0, 1
+DP_PATH_AUTO, DP_PATH_GRAM, DP_PATH_MATERIALIZED = 0, 1, 2
+_KINDS = {"linear": DP_LINEAR, "layernorm": DP_LAYERNORM, "embedding": DP_EMBEDDING}
+
+EXPORTS = ["dp_workspace_bytes", "dp_per_example_sqnorms", "dp_clip_factors", "dp_clipped_accumulate",
+           "dp_add_noise_and_scale", "dp_adamw_step", "dp_noise_scale_adamw_step", "dp_philox_u32",
+           "dp_token_equality_mask", "dp_poll_status", "dp_launch_count", "dp_status_string", "dp_version"]
+
+
+class dp_layer(C.Structure):
+    _fields_ = [("kind", C.c_int32), ("dtype", C.c_int32), ("path", C.c_int32), ("has_bias", C.c_int32),
+                ("B", C.c_int32), ("T", C.c_int32), ("d_in", C.c_int32), ("d_out", C.c_int32),
+                ("A", C.c_void_p), ("ids", C.c_void_p), ("G", C.c_void_p),
+                ("acc_w", C.c_void_p), ("acc_b", C.c_void_p)]
+
+
+class DpError(RuntimeError):
+    def __init__(self, fn: str, code: int):
+        self.code = code
+        super().__init__(f"{fn} failed: {code} ({status_string(code)})")
+
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    """Load the shared library (built by paper_2108_01624_b200.build); fails loudly when absent."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(f"{LIB_PATH} not found: run `python -m paper_2108_01624_b200.build` (needs nvcc). "
+                              "There is no fallback implementation.")
+        L = C.CDLL(LIB_PATH)
+        vp, i32, i64, u64, f32, sz = C.c_void_p, C.c_int, C.c_int64, C.c_uint64, C.c_float, C.c_size_t
+        L.dp_workspace_bytes.restype = sz
+        L.dp_workspace_bytes.argtypes = [vp, i32]
+        L.dp_per_example_sqnorms.argtypes = [vp, i32, vp, i32, vp, sz, vp]
+        L.dp_clip_factors.argtypes = [vp, i32, f32, vp, vp]
+        L.dp_clipped_accumulate.argtypes = [vp, i32, vp, vp, sz, vp]
+        L.dp_add_noise_and_scale.argtypes = [vp, i64, i64, f32, f32, i64, u64, u64, vp]
+        L.dp_adamw_step.argtypes = [vp, vp, vp, vp, i64, f32, f32, f32, f32, f32, i64, vp]
+        L.dp_noise_scale_adamw_step.argtypes = [vp, vp, vp, vp, i32, i64, i64, f32, f32, i64, u64, u64,
+                                                f32, f32, f32, f32, f32, i64, vp]
+        L.dp_philox_u32.argtypes = [vp, i64, i64, u64, u64, vp]
+        L.dp_token_equality_mask.argtypes = [vp, i32, i32, vp, vp]
+        L.dp_poll_status.argtypes = [vp]
+        L.dp_status_string.restype = C.c_char_p
+        L.dp_status_string.argtypes = [i32]
+        L.dp_version.restype = i32
+        L.dp_launch_count.restype = C.c_longlong
+        for name in EXPORTS:
+            getattr(L, name)          # AttributeError if the library does not export it
+        _lib = L
+    return _lib
+
+
+def status_string(code: int) -> str:
+    return lib().dp_status_string(int(code)).decode()
+
+
+def _check(fn: str, code: int):
+    if code != DP_OK:
+        raise DpError(fn, code)
+
+
+def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
+    if t is None:
+        return None
+    if not t.is_cuda:
+        raise ValueError("device tensor expected")
+    if not t.is_contiguous():
+        raise ValueError("contiguous tensor expected")
+    return t.data_ptr()
+
+
+def _stream(stream=None) -> int:
+    s = torch.cuda.current_stream() if stream is None else stream
+    return s.cuda_stream
+
+
+@dataclass
+class Layer:
+    """Python-side layer description; tensors live on the GPU."""
+    kind: str
+    G: torch.Tensor
+    A: Optional[torch.Tensor] = None
+    ids: Optional[torch.Tensor] = None
+    acc_w: Optional[torch.Tensor] = None
+    acc_b: Optional[torch.Tensor] = None
+    has_bias: bool = False
+    vocab: int = 0
+    path: int = DP_PATH_AUTO
+
+
+class LayerList:
+    """A HOST array of dp_layer descriptors plus references that keep the tensors alive."""
+
+    def __init__(self, layers: Sequence[Layer]):
+        self.layers = list(layers)
+        self.array = (dp_layer * len(self.layers))()
+        for k, L in enumerate(self.layers):
+            d = self.array[k]
+            B, T, d_out = L.G.shape
+            if L.G.dtype not in (torch.float32, torch.bfloat16):
+                raise ValueError("A and G must be fp32 or bf16")
+            d.kind = _KINDS[L.kind]
+            d.dtype = DP_F32 if L.G.dtype == torch.float32 else DP_BF16
+            d.path = int(L.path)
+            d.has_bias = int(bool(L.has_bias))
+            d.B, d.T, d.d_out = B, T, d_out
+            if L.kind == "embedding":
+                if L.ids is None or L.ids.dtype != torch.int32:
+                    raise ValueError("embedding needs int32 ids")
+                d.d_in = int(L.vocab)
+            else:
+                if L.A is None or L.A.dtype != L.G.dtype:
+                    raise ValueError("A must have G's dtype")
+                d.d_in = L.A.shape[2]
+            d.A, d.ids, d.G = _ptr(L.A), _ptr(L.ids), _ptr(L.G)
+            d.acc_w, d.acc_b = _ptr(L.acc_w), _ptr(L.acc_b)
+            for acc in (L.acc_w, L.acc_b):
+                if acc is not None and acc.dtype != torch.float32:
+                    raise ValueError("accumulators are fp32")
+
+    @property
+    def ptr(self):
+        return C.cast(self.array, C.c_void_p)
+
+    def __len__(self):
+        return len(self.layers)
+
+    @property
+    def B(self) -> int:
+        return int(self.array[0].B)
+
+
+def dp_version() -> int:
+    return lib().dp_version()
+
+
+def dp_workspace_bytes(layers: LayerList) -> int:
+    return int(lib().dp_workspace_bytes(layers.ptr, len(layers)))
+
+
+def alloc_workspace(layers: LayerList) -> Optional[torch.Tensor]:
+    """Caller-owned scratch for the two layer-list calls (torch's allocator aligns to 512 bytes)."""
+    n = dp_workspace_bytes(layers)
+    dev = layers.layers[0].G.device
+    return torch.empty(max(n, 256), dtype=torch.uint8, device=dev)
+
+
+def dp_per_example_sqnorms(layers: LayerList, sqnorm: torch.Tensor, accumulate_into: bool = False,
+                           workspace: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    ws_p, ws_n = (_ptr(workspace), workspace.numel() * workspace.element_size()) if workspace is not None else (None, 0)
+    _check("dp_per_example_sqnorms",
+           lib().dp_per_example_sqnorms(layers.ptr, len(layers), _ptr(sqnorm), int(accumulate_into), ws_p, ws_n,
+                                        _stream(stream)))
+    return sqnorm
+
+
+def dp_clip_factors(sqnorm: torch.Tensor, C_: float, clip: torch.Tensor, stream=None) -> torch.Tensor:
+    _check("dp_clip_factors", lib().dp_clip_factors(_ptr(sqnorm), sqnorm.numel(), float(C_), _ptr(clip), _stream(stream)))
+    return clip
+
+
+def dp_clipped_accumulate(layers: LayerList, clip: torch.Tensor, workspace: Optional[torch.Tensor] = None,
+                          stream=None) -> None:
+    ws_p, ws_n = (_ptr(workspace), workspace.numel() * workspace.element_size()) if workspace is not None else (None, 0)
+    _check("dp_clipped_accumulate",
+           lib().dp_clipped_accumulate(layers.ptr, len(layers), _ptr(clip), ws_p, ws_n, _stream(stream)))
+
+
+def dp_add_noise_and_scale(acc: torch.Tensor, sigma: float, C_: float, batch_size: int, seed: int, step: int,
+                           elem_offset: int = 0, stream=None) -> torch.Tensor:
+    _check("dp_add_noise_and_scale",
+           lib().dp_add_noise_and_scale(_ptr(acc), acc.numel(), int(elem_offset), float(sigma), float(C_),
+                                        int(batch_size), int(seed), int(step), _stream(stream)))
+    return acc
+
+
+def dp_adamw_step(theta, m, v, g, lr, beta1, beta2, xi, weight_decay, t, stream=None) -> None:
+    _check("dp_adamw_step",
+           lib().dp_adamw_step(_ptr(theta), _ptr(m), _ptr(v), _ptr(g), theta.numel(), float(lr), float(beta1),
+                               float(beta2), float(xi), float(weight_decay), int(t), _stream(stream)))
+
+
+def dp_noise_scale_adamw_step(theta, m, v, acc, zero_acc, sigma, C_, batch_size, seed, step, lr, beta1, beta2,
+                              xi, weight_decay, t, elem_offset: int = 0, stream=None) -> None:
+    _check("dp_noise_scale_adamw_step",
+           lib().dp_noise_scale_adamw_step(_ptr(theta), _ptr(m), _ptr(v), _ptr(acc), int(bool(zero_acc)),
+                                           theta.numel(), int(elem_offset), float(sigma), float(C_),
+                                           int(batch_size), int(seed), int(step), float(lr), float(beta1),
+                                           float(beta2), float(xi), float(weight_decay), int(t), _stream(stream)))
+
+
+def dp_philox_u32(out: torch.Tensor, elem_offset: int, seed: int, step: int, stream=None) -> torch.Tensor:
+    """out: int32 tensor (bit pattern of the uint32 words)."""
+    _check("dp_philox_u32", lib().dp_philox_u32(_ptr(out), out.numel(), int(elem_offset), int(seed), int(step),
+                                                _stream(stream)))
+    return out
+
+
+def dp_token_equality_mask(ids: torch.Tensor, mask: torch.Tensor, stream=None) -> torch.Tensor:
+    B, T = ids.shape
+    _check("dp_token_equality_mask", lib().dp_token_equality_mask(_ptr(ids), B, T, _ptr(mask), _stream(stream)))
+    return mask
+
+
+def dp_launch_count() -> int:
+    return int(lib().dp_launch_count())
+
+
+def dp_poll_status(stream=None) -> int:
+    return int(lib().dp_poll_status(_stream(stream)))

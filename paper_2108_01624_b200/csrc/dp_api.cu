@@ -1,0 +1,322 @@
+// C ABI (include/dp.h): argument validation, workspace layout and dispatch to the kernels.
+#include <atomic>
+#include <cmath>
+#include <vector>
+
+#include "dp_internal.h"
+
+namespace dpk {
+
+__device__ int g_status_word = 0;
+
+static std::atomic<long long> g_launches{0};
+void note_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+
+// Device address of the status word for the current device (looked up once per device).
+static int* status_ptr() {
+  static int* cache[64] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  if (!cache[dev]) {
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_status_word) != cudaSuccess) return nullptr;
+    cache[dev] = static_cast<int*>(p);
+  }
+  return cache[dev];
+}
+
+static bool finite_f(float x) { return std::isfinite(x); }
+static size_t elem_size(int dtype) { return dtype == DP_F32 ? 4 : 2; }
+static bool misaligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) != 0; }
+
+// Shape/pointer checks shared by the two layer-list entry points.
+static int validate_layers(const dp_layer* layers, int n_layers, bool need_acc) {
+  if (!layers || n_layers <= 0) return DP_ERR_ARG;
+  const int B = layers[0].B, T = layers[0].T;
+  if (B <= 0 || T <= 0) return DP_ERR_ARG;
+  for (int l = 0; l < n_layers; ++l) {
+    const dp_layer& L = layers[l];
+    if (L.B != B || L.T != T) return DP_ERR_ARG;
+    if (L.kind != DP_LINEAR && L.kind != DP_LAYERNORM && L.kind != DP_EMBEDDING) return DP_ERR_ARG;
+    if (L.dtype != DP_F32 && L.dtype != DP_BF16) return DP_ERR_ARG;
+    if (L.path != DP_PATH_AUTO && L.path != DP_PATH_GRAM && L.path != DP_PATH_MATERIALIZED) return DP_ERR_ARG;
+    if (L.d_in <= 0 || L.d_out <= 0 || !L.G) return DP_ERR_ARG;
+    if ((long long)B * T * (long long)(L.d_out > L.d_in && L.kind != DP_EMBEDDING ? L.d_out : L.d_in) <= 0) return DP_ERR_ARG;
+    if (misaligned(L.G, elem_size(L.dtype))) return DP_ERR_ALIGN;
+    if (L.kind == DP_EMBEDDING) {
+      if (!L.ids) return DP_ERR_ARG;
+      if (misaligned(L.ids, 4)) return DP_ERR_ALIGN;
+    } else {
+      if (!L.A) return DP_ERR_ARG;
+      if (misaligned(L.A, elem_size(L.dtype))) return DP_ERR_ALIGN;
+      if (L.kind == DP_LAYERNORM && L.d_in != L.d_out) return DP_ERR_ARG;
+    }
+    if (need_acc) {
+      if (!L.acc_w || misaligned(L.acc_w, 4)) return L.acc_w ? DP_ERR_ALIGN : DP_ERR_ARG;
+      const bool wants_b = (L.kind == DP_LINEAR && L.has_bias) || L.kind == DP_LAYERNORM;
+      if (wants_b && !L.acc_b) return DP_ERR_ARG;
+      if (L.acc_b && misaligned(L.acc_b, 4)) return DP_ERR_ALIGN;
+    }
+  }
+  return DP_OK;
+}
+
+static bool use_gram(const dp_layer& L) {
+  if (L.path == DP_PATH_GRAM) return true;
+  if (L.path == DP_PATH_MATERIALIZED) return false;
+  return (long long)L.T * (L.d_in + L.d_out) <= (long long)L.d_in * L.d_out;
+}
+
+// Workspace layout: [column-sum scratch | partial sums of the tensor-core norm kernels].
+struct WsPlan {
+  size_t colsum_bytes = 0;     // max over layers of B*2d (LayerNorm) or B*d_out (linear bias) floats
+  size_t partial_bytes = 0;    // B * partials_per_example floats
+  int partials_per_example = 0;
+  std::vector<int> umma_idx;   // layers handled by the tensor-core kernels
+  std::vector<int> umma_gram;  // 1: Gram path, 0: materialised tiles
+  size_t total() const { return align_up(colsum_bytes, 256) + align_up(partial_bytes, 256); }
+};
+
+static WsPlan plan_workspace(const dp_layer* layers, int n_layers) {
+  WsPlan p;
+  const size_t B = layers[0].B;
+  for (int l = 0; l < n_layers; ++l) {
+    const dp_layer& L = layers[l];
+    size_t need = 0;
+    if (L.kind == DP_LAYERNORM) need = B * 2 * (size_t)L.d_out * sizeof(float);
+    if (L.kind == DP_LINEAR && L.has_bias) need = B * (size_t)L.d_out * sizeof(float);
+    if (need > p.colsum_bytes) p.colsum_bytes = need;
+    if (L.kind == DP_LINEAR && umma_supported(L)) {
+      p.umma_idx.push_back(l);
+      p.umma_gram.push_back(use_gram(L) ? 1 : 0);
+    }
+  }
+  if (!p.umma_idx.empty()) {
+    p.partials_per_example = (int)umma_sqnorm_partials_per_example(layers, p.umma_idx.data(), (int)p.umma_idx.size(),
+                                                                   p.umma_gram.data());
+    p.partial_bytes = B * (size_t)p.partials_per_example * sizeof(float);
+  }
+  return p;
+}
+
+static int check_ws(const WsPlan& p, void* ws, size_t bytes) {
+  if (p.total() == 0) return DP_OK;
+  if (!ws || misaligned(ws, 256) || bytes < p.total()) return DP_ERR_WORKSPACE;
+  return DP_OK;
+}
+
+#define DP_CUDA(expr) do { if ((expr) != cudaSuccess) return DP_ERR_CUDA; } while (0)
+
+}  // namespace dpk
+
+using namespace dpk;
+
+extern "C" {
+
+size_t dp_workspace_bytes(const dp_layer* layers, int n_layers) {
+  if (validate_layers(layers, n_layers, false) != DP_OK) return 0;
+  return plan_workspace(layers, n_layers).total();
+}
+
+int dp_per_example_sqnorms(const dp_layer* layers, int n_layers, float* sqnorm, int accumulate_into,
+                           void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  int rc = validate_layers(layers, n_layers, false);
+  if (rc != DP_OK) return rc;
+  if (!sqnorm) return DP_ERR_ARG;
+  if (misaligned(sqnorm, 4)) return DP_ERR_ALIGN;
+  const WsPlan plan = plan_workspace(layers, n_layers);
+  if ((rc = check_ws(plan, workspace, workspace_bytes)) != DP_OK) return rc;
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  int* status = status_ptr();
+  if (!status) return DP_ERR_CUDA;
+  float* colsum = static_cast<float*>(workspace);
+  float* partial = reinterpret_cast<float*>(static_cast<char*>(workspace) + align_up(plan.colsum_bytes, 256));
+  const int B = layers[0].B;
+  if (!accumulate_into) DP_CUDA(launch_fill_zero(sqnorm, B, s));
+  // Tensor-core layers first (one persistent launch per path), then the bandwidth-bound layers.
+  if (!plan.umma_idx.empty()) {
+    rc = launch_umma_sqnorms(layers, plan.umma_idx.data(), (int)plan.umma_idx.size(), plan.umma_gram.data(), partial,
+                             plan.partials_per_example, 0, status, s);
+    if (rc != DP_OK) return rc;
+    DP_CUDA(launch_reduce_partials(partial, B, plan.partials_per_example, sqnorm, s));
+  }
+  size_t u = 0;
+  for (int l = 0; l < n_layers; ++l) {
+    const dp_layer& L = layers[l];
+    if (u < plan.umma_idx.size() && plan.umma_idx[u] == l) { ++u; continue; }
+    if (L.kind == DP_LINEAR) {
+      DP_CUDA(launch_linear_sqnorm_generic(L, use_gram(L), sqnorm, s));
+    } else if (L.kind == DP_LAYERNORM) {
+      DP_CUDA(launch_layernorm_colsums(L, colsum, s));
+      DP_CUDA(launch_layernorm_sqnorm(L, colsum, sqnorm, s));
+    } else {
+      DP_CUDA(launch_embedding_sqnorm(L, sqnorm, status, s));
+    }
+  }
+  return DP_OK;
+}
+
+int dp_clip_factors(const float* sqnorm, int B, float C, float* clip, void* cuda_stream) {
+  if (!sqnorm || !clip || B <= 0) return DP_ERR_ARG;
+  if (!(C > 0.0f) || !finite_f(C)) return DP_ERR_ARG;
+  if (misaligned(sqnorm, 4) || misaligned(clip, 4)) return DP_ERR_ALIGN;
+  DP_CUDA(launch_clip_factors(sqnorm, B, C, clip, static_cast<cudaStream_t>(cuda_stream)));
+  return DP_OK;
+}
+
+int dp_clipped_accumulate(const dp_layer* layers, int n_layers, const float* clip, void* workspace,
+                          size_t workspace_bytes, void* cuda_stream) {
+  int rc = validate_layers(layers, n_layers, true);
+  if (rc != DP_OK) return rc;
+  if (!clip) return DP_ERR_ARG;
+  if (misaligned(clip, 4)) return DP_ERR_ALIGN;
+  const WsPlan plan = plan_workspace(layers, n_layers);
+  if ((rc = check_ws(plan, workspace, workspace_bytes)) != DP_OK) return rc;
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  int* status = status_ptr();
+  if (!status) return DP_ERR_CUDA;
+  float* colsum = static_cast<float*>(workspace);
+  if (!plan.umma_idx.empty()) {
+    rc = launch_umma_accumulate(layers, plan.umma_idx.data(), (int)plan.umma_idx.size(), clip, status, s);
+    if (rc != DP_OK) return rc;
+  }
+  size_t u = 0;
+  for (int l = 0; l < n_layers; ++l) {
+    const dp_layer& L = layers[l];
+    const bool on_umma = u < plan.umma_idx.size() && plan.umma_idx[u] == l;
+    if (on_umma) ++u;
+    if (L.kind == DP_LINEAR) {
+      if (!on_umma) DP_CUDA(launch_linear_accum_generic(L, clip, s));
+      if (L.has_bias && !(on_umma && umma_accumulates_bias())) {
+        DP_CUDA(launch_bias_colsums(L, colsum, s));
+        DP_CUDA(launch_bias_reduce(L, colsum, clip, s));
+      }
+    } else if (L.kind == DP_LAYERNORM) {
+      DP_CUDA(launch_layernorm_colsums(L, colsum, s));
+      DP_CUDA(launch_layernorm_accum(L, colsum, clip, s));
+    } else {
+      DP_CUDA(launch_embedding_accum(L, clip, status, s));
+    }
+  }
+  return DP_OK;
+}
+
+static int make_noise_args(int64_t n, int64_t elem_offset, float sigma, float C, int64_t batch_size, uint64_t seed,
+                           uint64_t step, NoiseArgs* na) {
+  if (n < 0 || elem_offset < 0 || batch_size <= 0) return DP_ERR_ARG;
+  if (!finite_f(sigma) || sigma < 0.0f || !finite_f(C) || !(C > 0.0f)) return DP_ERR_ARG;
+  na->sigmaC = sigma * C;
+  na->inv_n = (float)(1.0 / (double)batch_size);
+  na->key0 = (uint32_t)seed;
+  na->key1 = (uint32_t)(seed >> 32);
+  na->step0 = (uint32_t)step;
+  na->step1 = (uint32_t)(step >> 32);
+  na->elem_offset = elem_offset;
+  return DP_OK;
+}
+
+static int make_adam_args(float lr, float b1, float b2, float xi, float wd, int64_t t, AdamArgs* aa) {
+  if (t < 1) return DP_ERR_ARG;
+  if (!finite_f(lr) || !finite_f(xi) || !finite_f(wd) || xi < 0.0f) return DP_ERR_ARG;
+  if (!(b1 >= 0.0f && b1 < 1.0f) || !(b2 >= 0.0f && b2 < 1.0f)) return DP_ERR_ARG;
+  aa->lr = lr; aa->beta1 = b1; aa->beta2 = b2; aa->xi = xi; aa->wd = wd;
+  aa->one_m_beta1 = (float)(1.0 - (double)b1);
+  aa->one_m_beta2 = (float)(1.0 - (double)b2);
+  aa->bias1 = (float)(1.0 / (1.0 - std::pow((double)b1, (double)t)));
+  aa->bias2 = (float)(1.0 / (1.0 - std::pow((double)b2, (double)t)));
+  return DP_OK;
+}
+
+int dp_add_noise_and_scale(float* acc, int64_t n, int64_t elem_offset, float sigma, float C, int64_t batch_size,
+                           uint64_t seed, uint64_t step, void* cuda_stream) {
+  NoiseArgs na;
+  int rc = make_noise_args(n, elem_offset, sigma, C, batch_size, seed, step, &na);
+  if (rc != DP_OK) return rc;
+  if (n == 0) return DP_OK;
+  if (!acc) return DP_ERR_ARG;
+  if (misaligned(acc, 4)) return DP_ERR_ALIGN;
+  DP_CUDA(launch_noise_scale(acc, n, na, static_cast<cudaStream_t>(cuda_stream)));
+  return DP_OK;
+}
+
+int dp_adamw_step(float* theta, float* m, float* v, const float* g, int64_t n, float lr, float beta1, float beta2,
+                  float xi, float weight_decay, int64_t t, void* cuda_stream) {
+  AdamArgs aa;
+  if (n < 0) return DP_ERR_ARG;
+  int rc = make_adam_args(lr, beta1, beta2, xi, weight_decay, t, &aa);
+  if (rc != DP_OK) return rc;
+  if (n == 0) return DP_OK;
+  if (!theta || !m || !v || !g) return DP_ERR_ARG;
+  if (misaligned(theta, 4) || misaligned(m, 4) || misaligned(v, 4) || misaligned(g, 4)) return DP_ERR_ALIGN;
+  DP_CUDA(launch_adamw(theta, m, v, g, n, aa, static_cast<cudaStream_t>(cuda_stream)));
+  return DP_OK;
+}
+
+int dp_noise_scale_adamw_step(float* theta, float* m, float* v, float* acc, int zero_acc, int64_t n,
+                              int64_t elem_offset, float sigma, float C, int64_t batch_size, uint64_t seed,
+                              uint64_t step, float lr, float beta1, float beta2, float xi, float weight_decay,
+                              int64_t t, void* cuda_stream) {
+  NoiseArgs na;
+  AdamArgs aa;
+  int rc = make_noise_args(n, elem_offset, sigma, C, batch_size, seed, step, &na);
+  if (rc != DP_OK) return rc;
+  if ((rc = make_adam_args(lr, beta1, beta2, xi, weight_decay, t, &aa)) != DP_OK) return rc;
+  if (n == 0) return DP_OK;
+  if (!theta || !m || !v || !acc) return DP_ERR_ARG;
+  if (misaligned(theta, 4) || misaligned(m, 4) || misaligned(v, 4) || misaligned(acc, 4)) return DP_ERR_ALIGN;
+  DP_CUDA(launch_noise_adamw(theta, m, v, acc, zero_acc, n, na, aa, static_cast<cudaStream_t>(cuda_stream)));
+  return DP_OK;
+}
+
+int dp_philox_u32(uint32_t* out, int64_t n_words, int64_t elem_offset, uint64_t seed, uint64_t step,
+                  void* cuda_stream) {
+  if (n_words < 0 || elem_offset < 0) return DP_ERR_ARG;
+  if (n_words == 0) return DP_OK;
+  if (!out) return DP_ERR_ARG;
+  if (misaligned(out, 4)) return DP_ERR_ALIGN;
+  NoiseArgs na = {};
+  na.key0 = (uint32_t)seed; na.key1 = (uint32_t)(seed >> 32);
+  na.step0 = (uint32_t)step; na.step1 = (uint32_t)(step >> 32);
+  na.elem_offset = elem_offset;
+  DP_CUDA(launch_philox_u32(out, n_words, na, static_cast<cudaStream_t>(cuda_stream)));
+  return DP_OK;
+}
+
+int dp_token_equality_mask(const int32_t* ids, int B, int T, uint8_t* mask, void* cuda_stream) {
+  if (!ids || !mask || B <= 0 || T <= 0) return DP_ERR_ARG;
+  if (misaligned(ids, 4)) return DP_ERR_ALIGN;
+  DP_CUDA(launch_equality_mask(ids, B, T, mask, static_cast<cudaStream_t>(cuda_stream)));
+  return DP_OK;
+}
+
+int dp_poll_status(void* cuda_stream) {
+  int* status = status_ptr();
+  if (!status) return DP_ERR_CUDA;
+  DP_CUDA(cudaStreamSynchronize(static_cast<cudaStream_t>(cuda_stream)));
+  int h = 0;
+  DP_CUDA(cudaMemcpy(&h, status, sizeof(int), cudaMemcpyDeviceToHost));
+  if (h != STATUS_OK) DP_CUDA(cudaMemset(status, 0, sizeof(int)));
+  if (h == STATUS_TIMEOUT) return DP_ERR_TIMEOUT;
+  if (h == STATUS_BAD_ID) return DP_ERR_BAD_ID;
+  return DP_OK;
+}
+
+const char* dp_status_string(int status) {
+  switch (status) {
+    case DP_OK: return "ok";
+    case DP_ERR_ARG: return "invalid argument";
+    case DP_ERR_ALIGN: return "misaligned pointer";
+    case DP_ERR_UNSUPPORTED: return "unsupported request";
+    case DP_ERR_CUDA: return "CUDA call failed";
+    case DP_ERR_TIMEOUT: return "device-side wait timed out";
+    case DP_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+    case DP_ERR_BAD_ID: return "token id out of range";
+    default: return "unknown status";
+  }
+}
+
+long long dp_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+int dp_version(void) { return 100; }
+
+}  // extern "C"

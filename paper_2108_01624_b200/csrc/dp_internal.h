@@ -1,0 +1,77 @@
+// Internal declarations shared by the translation units of libdp_b200.so.
+// Host-side launchers only; the C ABI in include/dp.h is implemented in dp_api.cu.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "../../include/dp.h"
+
+namespace dpk {
+
+// ---- small helpers -------------------------------------------------------------------------
+static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+static inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
+
+// Launch accounting: every kernel launch of the library is counted (read back by dp_launch_count).
+void note_launch(int n);
+static inline cudaError_t counted(int n) { note_launch(n); return cudaGetLastError(); }
+
+// Sticky device status word values (written with atomicCAS(0 -> code), first error wins).
+enum : int { STATUS_OK = 0, STATUS_TIMEOUT = 1, STATUS_BAD_ID = 2 };
+
+// ---- streaming kernels (dp_stream.cu) --------------------------------------------------------
+struct NoiseArgs {
+  float sigmaC;       // sigma * C
+  float inv_n;        // 1 / batch_size
+  uint32_t key0, key1;   // lo32(seed), hi32(seed)
+  uint32_t step0, step1; // lo32(step), hi32(step)
+  long long elem_offset;
+};
+struct AdamArgs {
+  float lr, beta1, beta2, one_m_beta1, one_m_beta2, bias1, bias2, xi, wd;  // bias = 1/(1-beta^t)
+};
+cudaError_t launch_clip_factors(const float* sqnorm, int B, float C, float* clip, cudaStream_t s);
+cudaError_t launch_noise_scale(float* acc, long long n, const NoiseArgs& na, cudaStream_t s);
+cudaError_t launch_adamw(float* theta, float* m, float* v, const float* g, long long n, const AdamArgs& aa,
+                         cudaStream_t s);
+cudaError_t launch_noise_adamw(float* theta, float* m, float* v, float* acc, int zero_acc, long long n,
+                               const NoiseArgs& na, const AdamArgs& aa, cudaStream_t s);
+cudaError_t launch_philox_u32(uint32_t* out, long long n, const NoiseArgs& na, cudaStream_t s);
+cudaError_t launch_equality_mask(const int32_t* ids, int B, int T, uint8_t* mask, cudaStream_t s);
+
+// ---- CUDA-core kernels for any shape and dtype (dp_generic.cu) ---------------------------------
+// Per-example squared norms; each adds into sqnorm[i] (one writer per example, launches are ordered).
+cudaError_t launch_linear_sqnorm_generic(const dp_layer& L, bool gram, float* sqnorm, cudaStream_t s);
+cudaError_t launch_linear_accum_generic(const dp_layer& L, const float* clip, cudaStream_t s);
+// LayerNorm: per-example column sums into ws[B][2d] (gain part then bias part), then either the norm
+// or the clip-weighted reduction over examples.
+cudaError_t launch_layernorm_colsums(const dp_layer& L, float* ws, cudaStream_t s);
+cudaError_t launch_layernorm_sqnorm(const dp_layer& L, const float* ws, float* sqnorm, cudaStream_t s);
+cudaError_t launch_layernorm_accum(const dp_layer& L, const float* ws, const float* clip, cudaStream_t s);
+// Embedding by grouping equal ids inside an example.
+cudaError_t launch_embedding_sqnorm(const dp_layer& L, float* sqnorm, int* status, cudaStream_t s);
+cudaError_t launch_embedding_accum(const dp_layer& L, const float* clip, int* status, cudaStream_t s);
+// Linear bias: per-example column sums of G into ws[B][d_out], then acc_b += sum_i clip_i * ws[i].
+cudaError_t launch_bias_colsums(const dp_layer& L, float* ws, cudaStream_t s);
+cudaError_t launch_bias_reduce(const dp_layer& L, const float* ws, const float* clip, cudaStream_t s);
+cudaError_t launch_fill_zero(float* p, long long n, cudaStream_t s);
+// sqnorm[i] (+)= sum of partial[i * stride + j], j < count, in a fixed order.
+cudaError_t launch_reduce_partials(const float* partial, int B, int count, float* sqnorm, cudaStream_t s);
+
+// ---- tcgen05 / TMA kernels for bf16 layers (dp_umma.cu) ----------------------------------------
+// A layer qualifies when dtype is bf16, d_in and d_out are multiples of 64 and pointers are 16-byte aligned.
+bool umma_supported(const dp_layer& L);
+// Number of fp32 partial sums the squared-norm kernels write for these layers (per example).
+// The partial buffer is [B][count] and is summed by launch_reduce_partials.
+// Whether launch_umma_accumulate also adds the bias column sums (else the caller runs the column-sum kernels).
+bool umma_accumulates_bias();
+size_t umma_sqnorm_partials_per_example(const dp_layer* layers, const int* idx, int n, const int* use_gram);
+int launch_umma_sqnorms(const dp_layer* layers, const int* idx, int n, const int* use_gram, float* partial,
+                        int partial_stride, int partial_base, int* status, cudaStream_t s);
+int launch_umma_accumulate(const dp_layer* layers, const int* idx, int n, const float* clip, int* status,
+                           cudaStream_t s);
+
+}  // namespace dpk

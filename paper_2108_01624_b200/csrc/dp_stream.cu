@@ -1,0 +1,216 @@
+// Streaming kernels: clip factors, Philox4x32-10 noise + scaling, AdamW, and the fused pass.
+// All are bandwidth-bound: one thread owns one Philox block (4 consecutive elements, one 16-byte
+// vector per array), loads are fully coalesced, and the grid is a multiple of the SM count.
+#include "dp_internal.h"
+
+namespace dpk {
+
+// ---------------------------------------------------------------------------------------------
+// Philox4x32-10 (Salmon et al., SC'11): ten rounds of
+//   (hi0,lo0) = M0*c0, (hi1,lo1) = M1*c2, c <- (hi1^c1^k0, lo1, hi0^c3^k1, lo0), key += (W0,W1).
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint4 philox4x32_10(uint4 c, uint32_t k0, uint32_t k1) {
+  const uint32_t M0 = 0xD2511F53u, M1 = 0xCD9E8D57u, W0 = 0x9E3779B9u, W1 = 0xBB67AE85u;
+#pragma unroll
+  for (int r = 0; r < 10; ++r) {
+    const uint32_t hi0 = __umulhi(M0, c.x), lo0 = M0 * c.x;
+    const uint32_t hi1 = __umulhi(M1, c.z), lo1 = M1 * c.z;
+    c = make_uint4(hi1 ^ c.y ^ k0, lo1, hi0 ^ c.w ^ k1, lo0);
+    k0 += W0;
+    k1 += W1;
+  }
+  return c;
+}
+
+__device__ __forceinline__ uint4 philox_block(unsigned long long j, const NoiseArgs& na) {
+  return philox4x32_10(make_uint4((uint32_t)j, (uint32_t)(j >> 32), na.step0, na.step1), na.key0, na.key1);
+}
+
+// Box-Muller on one word pair.  The uniforms are exact binary32 values:
+//   u1 = fl(x_a * 2^-32 + 2^-33) in (0,1],  u2 = fl(x_b * 2^-32) in [0,1].
+__device__ __forceinline__ void box_muller(uint32_t xa, uint32_t xb, float& z_even, float& z_odd) {
+  const float u1 = fmaf(__uint2float_rn(xa), 0x1p-32f, 0x1p-33f);
+  const float u2 = __uint2float_rn(xb) * 0x1p-32f;
+  const float r = sqrtf(-2.0f * logf(u1));
+  float sn, cs;
+  sincospif(2.0f * u2, &sn, &cs);
+  z_even = r * cs;
+  z_odd = r * sn;
+}
+
+__device__ __forceinline__ float4 normals4(unsigned long long j, const NoiseArgs& na) {
+  const uint4 x = philox_block(j, na);
+  float4 z;
+  box_muller(x.x, x.y, z.x, z.y);
+  box_muller(x.z, x.w, z.z, z.w);
+  return z;
+}
+
+__device__ __forceinline__ float adam_update(float& th, float& m, float& v, float g, const AdamArgs& a) {
+  m = a.beta1 * m + a.one_m_beta1 * g;
+  v = a.beta2 * v + a.one_m_beta2 * g * g;
+  const float mh = m * a.bias1;
+  const float vh = v * a.bias2;
+  th = th - a.lr * (mh / (sqrtf(vh) + a.xi) + a.wd * th);
+  return th;
+}
+
+// ---------------------------------------------------------------------------------------------
+// clip factors
+// ---------------------------------------------------------------------------------------------
+__global__ void k_clip_factors(const float* __restrict__ sqnorm, int B, float C, float* __restrict__ clip) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < B) {
+    const float n = sqnorm[i];
+    clip[i] = (n > 0.0f) ? fminf(1.0f, C / sqrtf(n)) : 1.0f;
+  }
+}
+
+cudaError_t launch_clip_factors(const float* sqnorm, int B, float C, float* clip, cudaStream_t s) {
+  k_clip_factors<<<ceil_div(B, 256), 256, 0, s>>>(sqnorm, B, C, clip);
+  return counted(1);
+}
+
+// ---------------------------------------------------------------------------------------------
+// The streaming pass.  MODE 0: noise+scale in place.  MODE 1: AdamW from g.  MODE 2: fused.
+// Thread work item = Philox block j (elements 4j .. 4j+3 of the flat parameter vector); the local
+// index of element e is e - elem_offset.  VEC: elem_offset % 4 == 0 and all pointers 16-byte
+// aligned, so a block is one float4 of each array; otherwise elements are handled one by one.
+// ---------------------------------------------------------------------------------------------
+template <int MODE, bool VEC>
+__global__ void __launch_bounds__(256)
+k_stream(float* __restrict__ theta, float* __restrict__ m, float* __restrict__ v, float* __restrict__ acc,
+         const float* __restrict__ g_in, int zero_acc, long long n, unsigned long long j0,
+         unsigned long long n_blocks, NoiseArgs na, AdamArgs aa) {
+  const unsigned long long stride = (unsigned long long)gridDim.x * blockDim.x;
+  for (unsigned long long b = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x; b < n_blocks; b += stride) {
+    const unsigned long long j = j0 + b;
+    const long long k0 = (long long)(4ull * j) - na.elem_offset;   // local index of lane 0
+    if (VEC && k0 >= 0 && k0 + 4 <= n) {
+      float4 gv;
+      if (MODE != 1) {
+        const float4 a4 = *reinterpret_cast<const float4*>(acc + k0);
+        const float4 z = normals4(j, na);
+        gv.x = (a4.x + na.sigmaC * z.x) * na.inv_n;
+        gv.y = (a4.y + na.sigmaC * z.y) * na.inv_n;
+        gv.z = (a4.z + na.sigmaC * z.z) * na.inv_n;
+        gv.w = (a4.w + na.sigmaC * z.w) * na.inv_n;
+      } else {
+        gv = *reinterpret_cast<const float4*>(g_in + k0);
+      }
+      if (MODE == 0) {
+        *reinterpret_cast<float4*>(acc + k0) = gv;
+      } else {
+        float4 t4 = *reinterpret_cast<const float4*>(theta + k0);
+        float4 m4 = *reinterpret_cast<const float4*>(m + k0);
+        float4 v4 = *reinterpret_cast<const float4*>(v + k0);
+        adam_update(t4.x, m4.x, v4.x, gv.x, aa);
+        adam_update(t4.y, m4.y, v4.y, gv.y, aa);
+        adam_update(t4.z, m4.z, v4.z, gv.z, aa);
+        adam_update(t4.w, m4.w, v4.w, gv.w, aa);
+        *reinterpret_cast<float4*>(theta + k0) = t4;
+        *reinterpret_cast<float4*>(m + k0) = m4;
+        *reinterpret_cast<float4*>(v + k0) = v4;
+        if (MODE == 2 && zero_acc) *reinterpret_cast<float4*>(acc + k0) = make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+    } else {
+      float z[4] = {0.f, 0.f, 0.f, 0.f};
+      if (MODE != 1) {
+        const float4 z4 = normals4(j, na);
+        z[0] = z4.x; z[1] = z4.y; z[2] = z4.z; z[3] = z4.w;
+      }
+#pragma unroll
+      for (int l = 0; l < 4; ++l) {
+        const long long k = k0 + l;
+        if (k < 0 || k >= n) continue;
+        float gv;
+        if (MODE != 1) gv = (acc[k] + na.sigmaC * z[l]) * na.inv_n; else gv = g_in[k];
+        if (MODE == 0) {
+          acc[k] = gv;
+        } else {
+          float t1 = theta[k], m1 = m[k], v1 = v[k];
+          adam_update(t1, m1, v1, gv, aa);
+          theta[k] = t1; m[k] = m1; v[k] = v1;
+          if (MODE == 2 && zero_acc) acc[k] = 0.0f;
+        }
+      }
+    }
+  }
+}
+
+static int stream_grid(unsigned long long n_blocks) {
+  int dev = 0, sms = 148;
+  cudaGetDevice(&dev);
+  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  const unsigned long long want = (n_blocks + 255) / 256;
+  const unsigned long long cap = (unsigned long long)sms * 16;   // 8 resident CTAs of 256 threads, two rounds
+  unsigned long long g = want < cap ? want : cap;
+  if (g >= (unsigned long long)sms) g = g / sms * sms;           // whole waves
+  return (int)(g ? g : 1);
+}
+
+static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+template <int MODE>
+static cudaError_t launch_stream(float* theta, float* m, float* v, float* acc, const float* g, int zero_acc,
+                                 long long n, const NoiseArgs& na, const AdamArgs& aa, cudaStream_t s) {
+  if (n <= 0) return cudaSuccess;
+  const unsigned long long j0 = (unsigned long long)na.elem_offset >> 2;
+  const unsigned long long j1 = ((unsigned long long)na.elem_offset + (unsigned long long)n + 3ull) >> 2;
+  const unsigned long long nb = j1 - j0;
+  bool vec = (na.elem_offset & 3) == 0;
+  if (MODE != 1) vec = vec && aligned16(acc);
+  if (MODE == 1) vec = vec && aligned16(g);
+  if (MODE != 0) vec = vec && aligned16(theta) && aligned16(m) && aligned16(v);
+  const int grid = stream_grid(nb);
+  if (vec) k_stream<MODE, true><<<grid, 256, 0, s>>>(theta, m, v, acc, g, zero_acc, n, j0, nb, na, aa);
+  else     k_stream<MODE, false><<<grid, 256, 0, s>>>(theta, m, v, acc, g, zero_acc, n, j0, nb, na, aa);
+  return counted(1);
+}
+
+cudaError_t launch_noise_scale(float* acc, long long n, const NoiseArgs& na, cudaStream_t s) {
+  AdamArgs aa = {};
+  return launch_stream<0>(nullptr, nullptr, nullptr, acc, nullptr, 0, n, na, aa, s);
+}
+cudaError_t launch_adamw(float* theta, float* m, float* v, const float* g, long long n, const AdamArgs& aa,
+                         cudaStream_t s) {
+  NoiseArgs na = {};
+  return launch_stream<1>(theta, m, v, nullptr, g, 0, n, na, aa, s);
+}
+cudaError_t launch_noise_adamw(float* theta, float* m, float* v, float* acc, int zero_acc, long long n,
+                               const NoiseArgs& na, const AdamArgs& aa, cudaStream_t s) {
+  return launch_stream<2>(theta, m, v, acc, nullptr, zero_acc, n, na, aa, s);
+}
+
+// ---------------------------------------------------------------------------------------------
+// Test utilities
+// ---------------------------------------------------------------------------------------------
+__global__ void k_philox_u32(uint32_t* __restrict__ out, long long n, NoiseArgs na) {
+  const long long stride = (long long)gridDim.x * blockDim.x;
+  for (long long k = (long long)blockIdx.x * blockDim.x + threadIdx.x; k < n; k += stride) {
+    const unsigned long long e = (unsigned long long)(na.elem_offset + k);
+    const uint4 x = philox_block(e >> 2, na);
+    const uint32_t w[4] = {x.x, x.y, x.z, x.w};
+    out[k] = w[e & 3];
+  }
+}
+cudaError_t launch_philox_u32(uint32_t* out, long long n, const NoiseArgs& na, cudaStream_t s) {
+  if (n <= 0) return cudaSuccess;
+  long long blocks = (n + 255) / 256;
+  if (blocks > 148 * 16) blocks = 148 * 16;
+  k_philox_u32<<<(int)blocks, 256, 0, s>>>(out, n, na);
+  return counted(1);
+}
+
+__global__ void k_equality_mask(const int32_t* __restrict__ ids, int T, uint8_t* __restrict__ mask) {
+  const int i = blockIdx.x;
+  const int32_t* row = ids + (size_t)i * T;
+  uint8_t* out = mask + (size_t)i * T * T;
+  for (int p = threadIdx.x; p < T * T; p += blockDim.x) out[p] = (row[p / T] == row[p % T]) ? 1 : 0;
+}
+cudaError_t launch_equality_mask(const int32_t* ids, int B, int T, uint8_t* mask, cudaStream_t s) {
+  k_equality_mask<<<B, 256, 0, s>>>(ids, T, mask);
+  return counted(1);
+}
+
+}  // namespace dpk

@@ -1,0 +1,110 @@
+"""Host-side sequencing of one DP-SGD macro-step over the C ABI (no arithmetic here).
+
+Algorithm 1's g_t needs, per microbatch, the per-example norms over ALL layers before any layer can be
+scaled, hence two passes over (A, G): norms -> clip factors -> clipped accumulate.  Noise, the division by
+the macro-batch size and the AdamW update run once per macro-batch (Section 5.3) as one fused pass.
+"""
+from __future__ import annotations
+
+from typing import List, Optional, Sequence
+
+import torch
+
+from . import binding as b
+from .synth import EMBEDDING, LAYERNORM, LINEAR, LayerData, LayerSpec
+
+
+class DPStep:
+    """Owns the flat fp32 state (theta, m, v, accumulator) for a list of layer specs.
+
+    Tensors are laid end to end in spec order (weight then bias), each start rounded up to a multiple of
+    4 elements so that every tensor is 16-byte aligned and one fused launch covers the whole vector.  The
+    flat index of an element is also its Philox element index.
+    """
+
+    def __init__(self, specs: Sequence[LayerSpec], device, C: float, sigma: float, lr: float, beta1: float,
+                 beta2: float, xi: float, weight_decay: float, seed: int = 0, theta: Optional[torch.Tensor] = None):
+        self.specs = list(specs)
+        self.device = torch.device(device)
+        self.C, self.sigma, self.lr, self.beta1, self.beta2 = C, sigma, lr, beta1, beta2
+        self.xi, self.weight_decay, self.seed = xi, weight_decay, seed
+        self.offsets: List[List[int]] = []
+        self.shapes: List[List[tuple]] = []
+        pos = 0
+        for sp in self.specs:
+            if sp.kind == LINEAR:
+                shp = [(sp.d_in, sp.d_out)] + ([(sp.d_out,)] if sp.has_bias else [])
+            elif sp.kind == LAYERNORM:
+                shp = [(sp.d_out,), (sp.d_out,)]
+            else:
+                shp = [(sp.d_in, sp.d_out)]
+            offs = []
+            for s in shp:
+                offs.append(pos)
+                n = 1
+                for x in s:
+                    n *= x
+                pos += (n + 3) // 4 * 4
+            self.offsets.append(offs)
+            self.shapes.append(shp)
+        self.n_flat = pos
+        self.acc = torch.zeros(pos, dtype=torch.float32, device=self.device)
+        self.m = torch.zeros_like(self.acc)
+        self.v = torch.zeros_like(self.acc)
+        self.theta = torch.zeros_like(self.acc) if theta is None else theta
+        self.t = 0
+        self.examples_seen = 0
+        self._ws = None
+        self._sqnorm = None
+        self._clip = None
+
+    def view(self, flat: torch.Tensor, li: int, k: int) -> torch.Tensor:
+        shp = self.shapes[li][k]
+        n = 1
+        for x in shp:
+            n *= x
+        off = self.offsets[li][k]
+        return flat[off:off + n].view(*shp)
+
+    def layer_list(self, data: Sequence[LayerData], paths: Optional[Sequence[int]] = None) -> b.LayerList:
+        """Descriptors for one microbatch; data[k] must correspond to specs[k]."""
+        out = []
+        for li, ld in enumerate(data):
+            sp = self.specs[li]
+            assert ld.spec.kind == sp.kind and ld.spec.d_out == sp.d_out
+            acc_w = self.view(self.acc, li, 0)
+            acc_b = self.view(self.acc, li, 1) if len(self.shapes[li]) > 1 else None
+            out.append(b.Layer(kind=sp.kind, G=ld.G, A=ld.A, ids=ld.ids, acc_w=acc_w, acc_b=acc_b,
+                               has_bias=sp.has_bias, vocab=sp.d_in if sp.kind == EMBEDDING else 0,
+                               path=b.DP_PATH_AUTO if paths is None else paths[li]))
+        return b.LayerList(out)
+
+    def accumulate_microbatch(self, layers: b.LayerList, stream=None):
+        """norms -> clip factors -> clipped accumulate for one microbatch (all enqueued, no sync)."""
+        B = layers.B
+        if self._sqnorm is None or self._sqnorm.numel() != B:
+            self._sqnorm = torch.empty(B, dtype=torch.float32, device=self.device)
+            self._clip = torch.empty(B, dtype=torch.float32, device=self.device)
+        need = b.dp_workspace_bytes(layers)
+        if self._ws is None or self._ws.numel() < need:
+            self._ws = torch.empty(max(need, 256), dtype=torch.uint8, device=self.device)
+        b.dp_per_example_sqnorms(layers, self._sqnorm, False, self._ws, stream)
+        b.dp_clip_factors(self._sqnorm, self.C, self._clip, stream)
+        b.dp_clipped_accumulate(layers, self._clip, self._ws, stream)
+        self.examples_seen += B
+        return self._sqnorm, self._clip
+
+    def finish_macro_batch(self, batch_size: Optional[int] = None, fused: bool = True, stream=None):
+        """Noise, division by the macro-batch size and the AdamW update; clears the accumulator."""
+        N = self.examples_seen if batch_size is None else batch_size
+        self.t += 1
+        if fused:
+            b.dp_noise_scale_adamw_step(self.theta, self.m, self.v, self.acc, True, self.sigma, self.C, N, self.seed,
+                                        self.t, self.lr, self.beta1, self.beta2, self.xi, self.weight_decay, self.t,
+                                        0, stream)
+        else:
+            b.dp_add_noise_and_scale(self.acc, self.sigma, self.C, N, self.seed, self.t, 0, stream)
+            b.dp_adamw_step(self.theta, self.m, self.v, self.acc, self.lr, self.beta1, self.beta2, self.xi,
+                            self.weight_decay, self.t, stream)
+            self.acc.zero_()
+        self.examples_seen = 0

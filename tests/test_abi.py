@@ -1,0 +1,97 @@
+"""CPU-only checks of the C-ABI library: it builds, loads, exports every declared symbol, and rejects
+bad arguments on the host before touching a device."""
+import ctypes as C
+import os
+import re
+
+import pytest
+
+from paper_2108_01624_b200 import binding as b
+from paper_2108_01624_b200 import build as builder
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    builder.build()
+    return b.lib()
+
+
+def test_every_declared_symbol_is_exported(lib):
+    header = open(os.path.join(ROOT, "include", "dp.h")).read()
+    names = re.findall(r"DP_API\s+[\w\s\*]+?\b(dp_\w+)\s*\(", header)
+    assert len(names) >= 12
+    assert sorted(names) == sorted(b.EXPORTS)
+    for n in names:
+        assert hasattr(lib, n)
+
+
+def test_status_strings_and_version(lib):
+    assert lib.dp_version() >= 100
+    assert b.status_string(0) == "ok"
+    for code in range(-7, 0):
+        assert b.status_string(code) not in ("ok", "unknown status")
+    assert b.status_string(-99) == "unknown status"
+
+
+def test_struct_layout_matches_header():
+    assert C.sizeof(b.dp_layer) == 8 * 4 + 5 * 8
+    assert b.dp_layer.A.offset == 32 and b.dp_layer.acc_b.offset == 64
+
+
+def test_host_side_argument_validation(lib):
+    """Null pointers, bad sizes and non-finite scalars are refused before any launch."""
+    ARG = -1
+    assert lib.dp_clip_factors(None, 4, 1.0, None, None) == ARG
+    assert lib.dp_clip_factors(256, 0, 1.0, 512, None) == ARG
+    assert lib.dp_clip_factors(256, 4, -1.0, 512, None) == ARG
+    assert lib.dp_clip_factors(256, 4, float("nan"), 512, None) == ARG
+    assert lib.dp_clip_factors(258, 4, 1.0, 512, None) == -2          # misaligned fp32 pointer
+    assert lib.dp_add_noise_and_scale(None, 8, 0, 1.0, 1.0, 4, 0, 0, None) == ARG
+    assert lib.dp_add_noise_and_scale(256, 8, 0, float("inf"), 1.0, 4, 0, 0, None) == ARG
+    assert lib.dp_add_noise_and_scale(256, 8, 0, 1.0, 0.0, 4, 0, 0, None) == ARG
+    assert lib.dp_add_noise_and_scale(256, 8, 0, 1.0, 1.0, 0, 0, 0, None) == ARG
+    assert lib.dp_add_noise_and_scale(256, -1, 0, 1.0, 1.0, 4, 0, 0, None) == ARG
+    assert lib.dp_add_noise_and_scale(None, 0, 0, 1.0, 1.0, 4, 0, 0, None) == 0   # empty range is a no-op
+    assert lib.dp_adamw_step(256, 256, 256, 256, 8, 1e-3, 0.9, 0.999, 1e-11, 0.0, 0, None) == ARG   # t < 1
+    assert lib.dp_adamw_step(256, 256, 256, 256, 8, 1e-3, 1.0, 0.999, 1e-11, 0.0, 1, None) == ARG   # beta1 = 1
+    assert lib.dp_adamw_step(None, 256, 256, 256, 8, 1e-3, 0.9, 0.999, 1e-11, 0.0, 1, None) == ARG
+    assert lib.dp_adamw_step(None, None, None, None, 0, 1e-3, 0.9, 0.999, 1e-11, 0.0, 1, None) == 0
+    assert lib.dp_philox_u32(None, 4, 0, 0, 0, None) == ARG
+    assert lib.dp_token_equality_mask(None, 1, 1, None, None) == ARG
+    # layer lists
+    L = (b.dp_layer * 2)()
+    assert lib.dp_per_example_sqnorms(None, 1, 256, 0, None, 0, None) == ARG
+    assert lib.dp_per_example_sqnorms(C.cast(L, C.c_void_p), 0, 256, 0, None, 0, None) == ARG
+    for k in range(2):
+        L[k].kind, L[k].dtype, L[k].B, L[k].T, L[k].d_in, L[k].d_out = 0, 0, 4, 8, 16, 16
+        L[k].A, L[k].G = 1024, 2048
+    p = C.cast(L, C.c_void_p)
+    assert lib.dp_per_example_sqnorms(p, 2, None, 0, None, 0, None) == ARG       # no output
+    L[1].B = 5
+    assert lib.dp_per_example_sqnorms(p, 2, 256, 0, None, 0, None) == ARG       # B differs between layers
+    L[1].B = 4
+    L[1].A = None
+    assert lib.dp_per_example_sqnorms(p, 2, 256, 0, None, 0, None) == ARG       # linear layer without A
+    L[1].A = 1026
+    assert lib.dp_per_example_sqnorms(p, 2, 256, 0, None, 0, None) == -2        # fp32 A not 4-byte aligned
+    L[1].A = 1024
+    L[1].kind = 7
+    assert lib.dp_per_example_sqnorms(p, 2, 256, 0, None, 0, None) == ARG       # unknown kind
+    L[1].kind = 2
+    assert lib.dp_per_example_sqnorms(p, 2, 256, 0, None, 0, None) == ARG       # embedding without ids
+    L[1].kind = 0
+    assert lib.dp_clipped_accumulate(p, 2, 256, None, 0, None) == ARG           # accumulators missing
+    assert lib.dp_workspace_bytes(p, 2) == 0                                    # nothing here needs scratch
+    L[0].has_bias = 1
+    assert lib.dp_workspace_bytes(p, 2) >= 4 * 16 * 4                           # bias column sums [B, d_out]
+    L[0].acc_w, L[0].acc_b, L[1].acc_w = 4096, 8192, 4096
+    assert lib.dp_clipped_accumulate(p, 2, 256, None, 0, None) == -6            # workspace missing
+
+
+def test_missing_library_fails_loudly(monkeypatch, tmp_path):
+    monkeypatch.setattr(b, "_lib", None)
+    monkeypatch.setattr(b, "LIB_PATH", str(tmp_path / "nope.so"))
+    with pytest.raises(ImportError):
+        b.lib()

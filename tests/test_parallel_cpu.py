@@ -1,0 +1,96 @@
+"""world_size-2 (and 3) gloo runs on CPU of the data-parallel macro-step's host logic: sharding, the
+accumulator reduction, shard-local noise + AdamW keyed by the global element index, and the gather."""
+import os
+import socket
+import sys
+
+import numpy as np
+import pytest
+import torch
+import torch.multiprocessing as mp
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+class _State:
+    def __init__(self, n, acc):
+        self.acc = acc.clone()
+        self.theta = torch.linspace(-1, 1, n, dtype=torch.float64)
+        self.m = torch.zeros(n, dtype=torch.float64)
+        self.v = torch.zeros(n, dtype=torch.float64)
+        self.t, self.examples_seen = 0, 0
+        self.sigma, self.C, self.seed = 1.3, 0.5, 11
+        self.lr, self.beta1, self.beta2, self.xi, self.weight_decay = 1e-2, 0.9, 0.999, 1e-11, 0.5
+
+
+def _oracle_update(state):
+    from oracle import dp_oracle as O
+
+    def fn(theta, m, v, acc, elem_offset, batch_size, t):
+        g = O.add_noise_and_scale(acc.numpy(), state.sigma, state.C, batch_size, state.seed, t, elem_offset)
+        th, mm, vv = O.adamw_step(theta.numpy(), m.numpy(), v.numpy(), g, state.lr, state.beta1, state.beta2,
+                                  state.xi, state.weight_decay, t)
+        theta.copy_(torch.from_numpy(th)); m.copy_(torch.from_numpy(mm)); v.copy_(torch.from_numpy(vv))
+        acc.zero_()
+    return fn
+
+
+def _worker(rank, world, port, n, out_dir):
+    sys.path.insert(0, ROOT)
+    import torch.distributed as dist
+    from paper_2108_01624_b200.parallel import ShardedUpdate
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    g = torch.Generator().manual_seed(100 + rank)
+    local_acc = torch.randn(n, generator=g, dtype=torch.float64)
+    st = _State(n, local_acc)
+    sh = ShardedUpdate(st, dist, world, rank, update_fn=_oracle_update(st))
+    for step in range(2):
+        st.acc.copy_(local_acc * (step + 1))
+        st.examples_seen = 64 * world
+        sh.finish_macro_batch()
+    torch.save({"theta": st.theta, "acc": st.acc, "lo": sh.lo, "hi": sh.hi, "m": st.m}, f"{out_dir}/r{rank}.pt")
+    dist.destroy_process_group()
+
+
+def _free_port():
+    s = socket.socket()
+    s.bind(("127.0.0.1", 0))
+    p = s.getsockname()[1]
+    s.close()
+    return p
+
+
+@pytest.mark.parametrize("world,n", [(2, 1003), (3, 64)])
+def test_sharded_update_equals_single_process(world, n, tmp_path):
+    from oracle import dp_oracle as O
+    mp.spawn(_worker, args=(world, _free_port(), n, str(tmp_path)), nprocs=world, join=True)
+    outs = [torch.load(f"{tmp_path}/r{r}.pt") for r in range(world)]
+    # single-process reference: summed accumulators, one update over the whole vector
+    accs = [torch.randn(n, generator=torch.Generator().manual_seed(100 + r), dtype=torch.float64) for r in range(world)]
+    st = _State(n, sum(accs))
+    fn = _oracle_update(st)
+    for step in range(2):
+        st.t += 1
+        acc = (sum(accs) * (step + 1)).clone()
+        fn(st.theta, st.m, st.v, acc, 0, 64 * world, st.t)
+    for r, o in enumerate(outs):
+        np.testing.assert_allclose(o["theta"].numpy(), st.theta.numpy(), rtol=1e-12, atol=1e-14)
+        assert float(o["acc"].abs().max()) == 0.0
+        np.testing.assert_allclose(o["m"][o["lo"]:o["hi"]].numpy(), st.m[o["lo"]:o["hi"]].numpy(), rtol=1e-12)
+    covered = sorted((o["lo"], o["hi"]) for o in outs)
+    assert covered[0][0] == 0 and covered[-1][1] == n
+    assert all(a[1] == b[0] for a, b in zip(covered[:-1], covered[1:]))
+    assert all(lo % 4 == 0 for lo, _ in covered)
+
+
+def test_shard_bounds_cover_and_align():
+    from paper_2108_01624_b200.parallel import shard_bounds
+    for n in (1, 5, 64, 1003, 333_563_904):
+        for world in (1, 2, 3, 8):
+            spans = [shard_bounds(n, world, r) for r in range(world)]
+            assert spans[0][0] == 0 and spans[-1][1] == n
+            for (a, b_), (c, d) in zip(spans[:-1], spans[1:]):
+                assert b_ == c and a <= b_
+            assert all(lo % 4 == 0 or lo == n for lo, _ in spans)

@@ -1,0 +1,180 @@
+"""GPU parity at BERT shapes: a BERT-Base block in full, the 24-layer BERT-Large stack with its Zipf token
+embedding (checker on an 8-example subset plus sampled accumulator entries at the full launch size), the
+T=512 crossover layer under all three path settings, and the mega-batch accumulation invariants."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2108_01624_b200 import DPStep, synth
+
+from .helpers import (LINEAR, O, b, gpu_norms_clip, make_layer_list, rel_l2, to_np, to_oracle_layers)
+
+pytestmark = pytest.mark.gpu
+
+if not torch.cuda.is_available():
+    pytest.skip("needs a CUDA device", allow_module_level=True)
+
+DEV = "cuda:0"
+CLIP_TOL = 1e-3
+BF16_TOL = 2e-2
+
+
+def _subset(data, rows):
+    return [synth.LayerData(ld.spec, G=ld.G[rows].contiguous(), A=None if ld.A is None else ld.A[rows].contiguous(),
+                            ids=None if ld.ids is None else ld.ids[rows].contiguous()) for ld in data]
+
+
+def _sampled_entries_check(data, accs, clip, n_samples, seed):
+    """acc_w[p,q] = sum_r clip[r/T] A[r,p] G[r,q] recomputed in fp64 on the host for random (p,q)."""
+    rng = np.random.default_rng(seed)
+    c = to_np(clip)
+    for ld, acc in zip(data, accs):
+        if ld.spec.kind != LINEAR:
+            continue
+        B, T, _ = ld.G.shape
+        w = np.repeat(c, T)
+        errs, mags = [], []
+        for _ in range(n_samples):
+            p, q = int(rng.integers(ld.spec.d_in)), int(rng.integers(ld.spec.d_out))
+            a = to_np(ld.A[:, :, p]).reshape(-1)
+            g = to_np(ld.G[:, :, q]).reshape(-1)
+            ref = float(np.sum(w * a * g))
+            errs.append(abs(float(acc[0][p, q]) - ref))
+            mags.append(abs(ref))
+        scale = float(np.sqrt(np.mean(np.square(mags)))) + 1e-30
+        assert max(errs) <= BF16_TOL * scale, f"{ld.spec.name}: {max(errs):.3e} vs rms {scale:.3e}"
+        if ld.spec.has_bias:
+            q = int(rng.integers(ld.spec.d_out))
+            ref = float(np.sum(w * to_np(ld.G[:, :, q]).reshape(-1)))
+            assert abs(float(acc[1][q]) - ref) <= BF16_TOL * (abs(ref) + scale)
+
+
+def test_bert_base_block_full_batch():
+    wl = synth.workload("bert_base_layer")
+    data = synth.generate(wl, seed=0, device=DEV)
+    ll, accs = make_layer_list(data, DEV)
+    n, c, ws = gpu_norms_clip(ll, wl.C)
+    b.dp_clipped_accumulate(ll, c, ws)
+    assert b.dp_poll_status() == 0
+    ol = to_oracle_layers(data)
+    n_ref = O.per_example_sqnorms(ol)
+    c_ref = O.clip_factors(n_ref, wl.C)
+    frac = float(np.mean(c_ref < 1.0))
+    assert 0.2 < frac < 0.8                      # the input recipe makes some examples clip and some not
+    np.testing.assert_allclose(to_np(c), c_ref, rtol=CLIP_TOL)
+    np.testing.assert_allclose(to_np(n), n_ref, rtol=2 * CLIP_TOL)
+    ref = O.clipped_accumulate(ol, c_ref, O.zero_accumulators(ol))
+    for ld, acc, racc in zip(data, accs, ref):
+        for x, y in zip(acc, racc):
+            assert rel_l2(to_np(x), y) <= BF16_TOL, ld.spec.name
+    # every clipped contribution is bounded by C: ||sum|| <= (number of examples) * C
+    tot = np.sqrt(sum(float((x.double() ** 2).sum()) for acc in accs for x in acc))
+    assert tot <= wl.B * wl.C * (1 + 1e-3)
+
+
+@pytest.mark.parametrize("n_layers", [24])
+def test_bert_large_stack_subset_and_samples(n_layers):
+    wl = synth.workload("bert_large")
+    specs = wl.specs[:6 * n_layers] + [wl.specs[-1]]
+    data = synth.generate(wl, seed=0, device=DEV, specs=specs)
+    assert len(data) == 6 * n_layers + 1
+    ll, accs = make_layer_list(data, DEV)
+    n, c, ws = gpu_norms_clip(ll, wl.C)
+    b.dp_clipped_accumulate(ll, c, ws)
+    torch.cuda.synchronize()
+    assert b.dp_poll_status() == 0
+    # (a) checker on examples 0..7, all layers and the embedding
+    rows = slice(0, 8)
+    sub = _subset(data, rows)
+    ol = to_oracle_layers(sub)
+    n_ref = O.per_example_sqnorms(ol)
+    c_ref = O.clip_factors(n_ref, wl.C)
+    np.testing.assert_allclose(to_np(n[rows]), n_ref, rtol=2 * CLIP_TOL)
+    np.testing.assert_allclose(to_np(c[rows]), c_ref, rtol=CLIP_TOL)
+    # (b) full launch size: sampled accumulator entries in fp64
+    _sampled_entries_check(data, accs, c, n_samples=6, seed=1)
+    # (c) the 8-example subset through the GPU path, element by element against the checker
+    ll8, acc8 = make_layer_list(sub, DEV)
+    n8, c8, ws8 = gpu_norms_clip(ll8, wl.C)
+    b.dp_clipped_accumulate(ll8, c8, ws8)
+    np.testing.assert_allclose(to_np(c8), c_ref, rtol=CLIP_TOL)
+    ref = O.clipped_accumulate(ol, c_ref, O.zero_accumulators(ol))
+    for ld, acc, racc in zip(sub, acc8, ref):
+        for x, y in zip(acc, racc):
+            assert rel_l2(to_np(x), y) <= BF16_TOL, ld.spec.name
+    # embedding ids follow the Zipf recipe: id 0 is the most frequent by far
+    ids = data[-1].ids
+    assert float((ids == 0).float().mean()) > 0.10
+
+
+def test_long_sequence_crossover_all_paths():
+    wl = synth.workload("bert_large_layer_t512")
+    data = synth.generate(wl, seed=0, device=DEV)
+    sub = _subset(data, slice(0, 4))
+    ol = to_oracle_layers(sub)
+    n_ref = O.per_example_sqnorms(ol)
+    c_ref = O.clip_factors(n_ref, wl.C)
+    norms = {}
+    for path in (b.DP_PATH_AUTO, b.DP_PATH_GRAM, b.DP_PATH_MATERIALIZED):
+        ll, accs = make_layer_list(data, DEV, [path] * len(data))
+        n, c, ws = gpu_norms_clip(ll, wl.C)
+        norms[path] = to_np(n)
+        np.testing.assert_allclose(norms[path][:4], n_ref, rtol=2 * CLIP_TOL)
+        np.testing.assert_allclose(to_np(c[:4]), c_ref, rtol=CLIP_TOL)
+    np.testing.assert_allclose(norms[b.DP_PATH_GRAM], norms[b.DP_PATH_MATERIALIZED], rtol=2 * CLIP_TOL)
+    np.testing.assert_allclose(norms[b.DP_PATH_AUTO], norms[b.DP_PATH_GRAM], rtol=2 * CLIP_TOL)
+    # clipped sum of the 4-example subset, element by element
+    ll4, acc4 = make_layer_list(sub, DEV)
+    n4, c4, ws4 = gpu_norms_clip(ll4, wl.C)
+    b.dp_clipped_accumulate(ll4, c4, ws4)
+    ref = O.clipped_accumulate(ol, c_ref, O.zero_accumulators(ol))
+    for ld, acc, racc in zip(sub, acc4, ref):
+        for x, y in zip(acc, racc):
+            assert rel_l2(to_np(x), y) <= BF16_TOL, ld.spec.name
+    # and sampled entries at the full B = 64 launch
+    ll, accs = make_layer_list(data, DEV)
+    n, c, ws = gpu_norms_clip(ll, wl.C)
+    b.dp_clipped_accumulate(ll, c, ws)
+    _sampled_entries_check(data, accs, c, n_samples=6, seed=2)
+
+
+def test_mega_batch_accumulation_invariants():
+    """K distinct microbatches against the checker, then the loop invariants: the same microbatch M times
+    gives M times the single result, and ||acc|| <= N * C."""
+    wl = synth.workload("bert_base_layer")
+    B = 16
+    step = DPStep(wl.specs, DEV, wl.C, wl.sigma, wl.lr, wl.beta1, wl.beta2, wl.xi, wl.weight_decay, seed=3)
+    ref = None
+    for mb in range(4):
+        data = synth.generate(wl, seed=1, device=DEV, microbatch=mb, B=B)
+        step.accumulate_microbatch(step.layer_list(data))
+        ol = to_oracle_layers(data)
+        ref = O.zero_accumulators(ol) if ref is None else ref
+        O.clipped_accumulate(ol, O.clip_factors(O.per_example_sqnorms(ol), wl.C), ref)
+    assert step.examples_seen == 4 * B
+    for li in range(len(wl.specs)):
+        for k in range(len(ref[li])):
+            assert rel_l2(to_np(step.view(step.acc, li, k)), ref[li][k]) <= BF16_TOL
+    assert float(step.acc.double().norm()) <= 4 * B * wl.C * (1 + 1e-3)
+    # same microbatch M times
+    single = DPStep(wl.specs, DEV, wl.C, wl.sigma, wl.lr, wl.beta1, wl.beta2, wl.xi, wl.weight_decay)
+    many = DPStep(wl.specs, DEV, wl.C, wl.sigma, wl.lr, wl.beta1, wl.beta2, wl.xi, wl.weight_decay)
+    data = synth.generate(wl, seed=2, device=DEV, B=B)
+    single.accumulate_microbatch(single.layer_list(data))
+    M = 8
+    ll = many.layer_list(data)
+    for _ in range(M):
+        many.accumulate_microbatch(ll)
+    assert rel_l2(to_np(many.acc), M * to_np(single.acc)) <= 1e-5
+    # finish: fused noise + AdamW against the checker on the whole flat vector
+    acc_before = to_np(many.acc)
+    th0 = synth.initial_weights(many.n_flat, 0, DEV)
+    many.theta.copy_(th0)
+    many.finish_macro_batch()
+    assert float(many.acc.abs().max()) == 0.0 and many.examples_seen == 0 and many.t == 1
+    g = O.add_noise_and_scale(acc_before, wl.sigma, wl.C, M * B, seed=0, step=1, elem_offset=0)
+    rt, rm, rv = O.adamw_step(to_np(th0), 0 * acc_before, 0 * acc_before, g, wl.lr, wl.beta1, wl.beta2, wl.xi,
+                              wl.weight_decay, 1)
+    assert rel_l2(to_np(many.m), rm) <= 1e-5 and rel_l2(to_np(many.v), rv) <= 1e-5
+    d, rd = to_np(many.theta) - to_np(th0), rt - to_np(th0)
+    assert np.max(np.abs(d - rd)) <= 1e-4 * np.max(np.abs(rd)) + 1e-7 * float(th0.abs().max())

@@ -1,0 +1,168 @@
+"""GPU parity for the layer passes (per-example norms, clip factors, clipped accumulate) against the CPU
+checker, from the tiny fp32 layer up to BERT-shaped bf16 blocks, including ragged and degenerate cases."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2108_01624_b200 import synth
+
+from .helpers import (EMBEDDING, LAYERNORM, LINEAR, LayerSpec, O, b, gpu_norms_clip, make_layer_list, random_layers,
+                      rel_l2, rel_max, to_np, to_oracle_layers)
+
+pytestmark = pytest.mark.gpu
+
+if not torch.cuda.is_available():
+    pytest.skip("needs a CUDA device", allow_module_level=True)
+
+DEV = "cuda:0"
+CLIP_TOL = 1e-3       # clip factors: relative error bound
+F32_TOL = 1e-4        # fp32-input paths
+BF16_TOL = 2e-2       # bf16-input / fp32-accumulate clipped sums, relative L2
+
+
+def check_against_checker(data, C, paths=None, sum_tol=BF16_TOL, rows=None):
+    """Runs norms -> clip -> accumulate on the GPU and compares all three with the checker."""
+    ll, accs = make_layer_list(data, DEV, paths)
+    n, c, ws = gpu_norms_clip(ll, C)
+    b.dp_clipped_accumulate(ll, c, ws)
+    assert b.dp_poll_status() == 0
+    ol = to_oracle_layers(data)
+    n_ref = O.per_example_sqnorms(ol)
+    c_ref = O.clip_factors(n_ref, C)
+    np.testing.assert_allclose(to_np(n), n_ref, rtol=2 * CLIP_TOL)
+    np.testing.assert_allclose(to_np(c), c_ref, rtol=CLIP_TOL)
+    ref = O.clipped_accumulate(ol, c_ref, O.zero_accumulators(ol))
+    for ld, acc, racc in zip(data, accs, ref):
+        for k, (x, y) in enumerate(zip(acc, racc)):
+            assert x.shape == y.shape
+            err = rel_l2(to_np(x), y)
+            assert err <= sum_tol, f"{ld.spec.name or ld.spec.kind}[{k}] rel L2 {err:.3e}"
+    return n_ref, c_ref, accs
+
+
+# ------------------------------------------------------------------ the tiny fp32 layer, end to end
+
+@pytest.mark.parametrize("path", [b.DP_PATH_AUTO, b.DP_PATH_GRAM, b.DP_PATH_MATERIALIZED])
+def test_tiny_linear_fp32_full_step(path):
+    wl = synth.workload("tiny_linear")
+    data = synth.generate(wl, seed=0, device=DEV)
+    n_ref, c_ref, accs = check_against_checker(data, wl.C, [path], sum_tol=F32_TOL)
+    assert np.all(c_ref < 1.0)                    # unit-variance inputs: every example clips at C = 1
+    # noise + AdamW on the 64x64 weight and the bias, laid end to end
+    rng = np.random.default_rng(0)
+    W0 = (rng.standard_normal((64, 64)) * 0.02).astype(np.float32)
+    ol = to_oracle_layers(data)
+    g_ref, _ = O.privatised_gradient([ol], wl.C, wl.sigma, seed=0, step=1)
+    flat = torch.cat([accs[0][0].reshape(-1), accs[0][1].reshape(-1)])
+    b.dp_add_noise_and_scale(flat, wl.sigma, wl.C, wl.B, 0, 1, 0)
+    g_ref_flat = np.concatenate([g_ref[0][0].ravel(), g_ref[0][1].ravel()])
+    assert rel_max(to_np(flat), g_ref_flat) <= F32_TOL
+    theta = torch.cat([torch.from_numpy(W0).reshape(-1), torch.zeros(64)]).to(DEV)
+    th0 = to_np(theta)
+    m, v = torch.zeros_like(theta), torch.zeros_like(theta)
+    b.dp_adamw_step(theta, m, v, flat, wl.lr, wl.beta1, wl.beta2, wl.xi, wl.weight_decay, 1)
+    rt, rm, rv = O.adamw_step(th0, np.zeros_like(th0), np.zeros_like(th0), g_ref_flat, wl.lr, wl.beta1, wl.beta2,
+                              wl.xi, wl.weight_decay, 1)
+    assert rel_max(to_np(m), rm) <= F32_TOL and rel_max(to_np(v), rv) <= F32_TOL
+    d, rd = to_np(theta) - th0, rt - th0
+    assert np.max(np.abs(d - rd)) <= F32_TOL * np.max(np.abs(rd)) + 1e-7 * np.max(np.abs(th0))
+
+
+# ------------------------------------------------------------------ small mixed models, ragged shapes
+
+SMALL = [LayerSpec(LINEAR, 128, 192, True, "fc1"), LayerSpec(LINEAR, 192, 64, False, "fc2"),
+         LayerSpec(LAYERNORM, 128, 128, False, "ln"), LayerSpec(EMBEDDING, 50, 64, False, "emb")]
+ODD = [LayerSpec(LINEAR, 72, 40, True, "fc_odd"), LayerSpec(LINEAR, 33, 17, True, "fc_unaligned"),
+       LayerSpec(LAYERNORM, 100, 100, False, "ln_odd"), LayerSpec(EMBEDDING, 11, 24, False, "emb_dup")]
+
+
+@pytest.mark.parametrize("dtype,tol", [(torch.float32, F32_TOL), (torch.bfloat16, BF16_TOL)])
+@pytest.mark.parametrize("specs,B,T", [(SMALL, 6, 40), (SMALL, 3, 128), (SMALL, 2, 200), (ODD, 5, 19), (ODD, 1, 1)])
+@pytest.mark.parametrize("path", [b.DP_PATH_AUTO, b.DP_PATH_GRAM, b.DP_PATH_MATERIALIZED])
+def test_small_models_all_paths(dtype, tol, specs, B, T, path):
+    data = random_layers(specs, B, T, dtype, DEV, seed=B * 1000 + T, g_scale=0.02, vocab_dup=7)
+    ol = to_oracle_layers(data)
+    C = float(np.sqrt(np.median(O.per_example_sqnorms(ol))))       # about half the examples clip
+    check_against_checker(data, C, [path] * len(specs), sum_tol=tol)
+
+
+def test_accumulates_in_place_over_microbatches():
+    """Two microbatches into the same accumulators equal the checker's sum; linear in the microbatch."""
+    accs = None
+    ref = None
+    for mb in range(2):
+        data = random_layers(SMALL, 4, 64, torch.bfloat16, DEV, seed=50 + mb, g_scale=0.02)
+        ll, accs = make_layer_list(data, DEV, accs=accs)
+        n, c, ws = gpu_norms_clip(ll, 0.5)
+        b.dp_clipped_accumulate(ll, c, ws)
+        ol = to_oracle_layers(data)
+        ref = O.zero_accumulators(ol) if ref is None else ref
+        O.clipped_accumulate(ol, O.clip_factors(O.per_example_sqnorms(ol), 0.5), ref)
+    for acc, racc in zip(accs, ref):
+        for x, y in zip(acc, racc):
+            assert rel_l2(to_np(x), y) <= BF16_TOL
+
+
+def test_sqnorm_accumulate_into_splits_the_model():
+    data = random_layers(SMALL, 4, 64, torch.bfloat16, DEV, seed=8, g_scale=0.02)
+    ll_all, _ = make_layer_list(data, DEV)
+    n_all, _, _ = gpu_norms_clip(ll_all, 1.0)
+    n_split = torch.empty(4, dtype=torch.float32, device=DEV)
+    for k, part in enumerate((data[:2], data[2:])):
+        ll, _ = make_layer_list(part, DEV)
+        b.dp_per_example_sqnorms(ll, n_split, accumulate_into=(k > 0), workspace=b.alloc_workspace(ll))
+    np.testing.assert_allclose(to_np(n_split), to_np(n_all), rtol=1e-5)
+
+
+def test_zero_gradient_example_is_left_unscaled():
+    data = random_layers(SMALL[:3], 3, 32, torch.bfloat16, DEV, seed=4, g_scale=0.02)
+    for ld in data:
+        ld.G[1].zero_()
+    ll, accs = make_layer_list(data, DEV)
+    n, c, ws = gpu_norms_clip(ll, 1e-3)
+    assert float(n[1]) == 0.0 and float(c[1]) == 1.0
+    b.dp_clipped_accumulate(ll, c, ws)
+    assert all(torch.isfinite(x).all() for acc in accs for x in acc)
+
+
+def test_no_clipping_equals_batch_gradient():
+    """C -> infinity: every c_i = 1 and the clipped sum is the plain batch gradient A^T G."""
+    data = random_layers(SMALL, 5, 96, torch.bfloat16, DEV, seed=21, g_scale=0.02)
+    ll, accs = make_layer_list(data, DEV)
+    n, c, ws = gpu_norms_clip(ll, 1e30)
+    assert torch.all(c == 1.0)
+    b.dp_clipped_accumulate(ll, c, ws)
+    A = to_np(data[0].A).reshape(-1, 128)
+    G = to_np(data[0].G).reshape(-1, 192)
+    assert rel_l2(to_np(accs[0][0]), A.T @ G) <= 1e-5
+    assert rel_l2(to_np(accs[0][1]), G.sum(0)) <= 1e-5
+
+
+def test_out_of_range_token_id_is_skipped_and_reported():
+    data = random_layers([SMALL[3]], 2, 16, torch.float32, DEV, seed=2)
+    data[0].ids[0, 3] = 50          # == V
+    data[0].ids[1, 0] = -1
+    ll, accs = make_layer_list(data, DEV)
+    n, c, ws = gpu_norms_clip(ll, 1e30)
+    b.dp_clipped_accumulate(ll, c, ws)
+    assert b.dp_poll_status() == -7
+    assert b.dp_poll_status() == 0                     # sticky word is cleared by the poll
+    ids = data[0].ids.cpu().numpy()
+    G = to_np(data[0].G)
+    E = np.zeros((50, 64))
+    for i in range(2):
+        for t in range(16):
+            if 0 <= ids[i, t] < 50:
+                E[ids[i, t]] += G[i, t]
+    assert rel_l2(to_np(accs[0][0]), E) <= 1e-6
+
+
+def test_workspace_too_small_is_refused():
+    data = random_layers(SMALL, 2, 16, torch.bfloat16, DEV, seed=2)
+    ll, _ = make_layer_list(data, DEV)
+    need = b.dp_workspace_bytes(ll)
+    assert need > 0
+    n = torch.empty(2, dtype=torch.float32, device=DEV)
+    with pytest.raises(b.DpError) as e:
+        b.dp_per_example_sqnorms(ll, n, False, torch.empty(need - 1, dtype=torch.uint8, device=DEV))
+    assert e.value.code == -6

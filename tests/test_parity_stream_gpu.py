@@ -1,0 +1,174 @@
+"""GPU parity: Philox words, equality masks, noise + scaling, AdamW, fused pass -- all through the C ABI,
+element by element against the CPU checker on the same seeded inputs."""
+import numpy as np
+import pytest
+import torch
+
+from .helpers import O, b, rel_l2, rel_max, to_np
+
+pytestmark = pytest.mark.gpu
+
+if not torch.cuda.is_available():
+    pytest.skip("needs a CUDA device", allow_module_level=True)
+
+DEV = "cuda:0"
+F32_TOL = 1e-4        # fp32 paths: relative error bound stated for this step
+
+
+@pytest.mark.parametrize("n,off,seed,step", [
+    (10007, 0, 0, 0),
+    (4099, 5, 0xDEADBEEF12345678, (7 << 32) | 11),
+    (2051, (1 << 34) + 3, 1, 2),        # block index crosses into the second counter word
+    (1, 2, 3, 4),
+])
+def test_philox_words_bit_exact(n, off, seed, step):
+    out = torch.empty(n, dtype=torch.int32, device=DEV)
+    b.dp_philox_u32(out, off, seed, step)
+    got = out.cpu().numpy().view(np.uint32)
+    assert np.array_equal(got, O.philox_u32(n, off, seed, step))
+
+
+def test_philox_independent_of_launch_split():
+    whole = torch.empty(100_000, dtype=torch.int32, device=DEV)
+    b.dp_philox_u32(whole, 13, 99, 5)
+    parts = [torch.empty(k, dtype=torch.int32, device=DEV) for k in (1, 33_333, 66_666)]
+    off = 13
+    for p in parts:
+        b.dp_philox_u32(p, off, 99, 5)
+        off += p.numel()
+    assert torch.equal(whole, torch.cat(parts))
+
+
+def test_token_equality_mask_bit_exact():
+    g = torch.Generator().manual_seed(3)
+    ids = torch.randint(0, 9, (5, 37), generator=g, dtype=torch.int32)
+    mask = torch.empty(5, 37, 37, dtype=torch.uint8, device=DEV)
+    b.dp_token_equality_mask(ids.to(DEV), mask)
+    ref = (ids[:, :, None] == ids[:, None, :]).to(torch.uint8)
+    assert torch.equal(mask.cpu(), ref)
+
+
+@pytest.mark.parametrize("n,off", [(1 << 20, 0), ((1 << 20) + 3, 0), (50_001, 7), (5, 2), (3, 1)])
+def test_noise_and_scale_matches_checker(n, off):
+    rng = np.random.default_rng(n + off)
+    S = rng.standard_normal(n).astype(np.float32) * 3
+    sigma, C, N, seed, step = 1.1, 0.7, 4096, 0xABCDEF0123, 3
+    base = torch.zeros(n + 8, dtype=torch.float32, device=DEV)
+    # a deliberately misaligned view when off is odd-ish: exercises the element-wise tail path
+    acc = base[(off % 4):(off % 4) + n]
+    acc.copy_(torch.from_numpy(S))
+    b.dp_add_noise_and_scale(acc, sigma, C, N, seed, step, elem_offset=off)
+    ref = O.add_noise_and_scale(S.astype(np.float64), sigma, C, N, seed, step, elem_offset=off)
+    got = to_np(acc)
+    assert rel_max(got, ref) <= F32_TOL
+    assert rel_l2(got, ref) <= 1e-5
+    # the noise itself: recover z and compare with the fp64 normals
+    z = (got * N - S.astype(np.float64)) / (sigma * C)
+    zr = O.standard_normals(n, off, seed, step)
+    assert np.max(np.abs(z - zr)) <= 2e-5 * max(1.0, np.max(np.abs(zr))) + 6e-6 * np.max(np.abs(S)) / (sigma * C)
+    # untouched guard elements
+    assert float(base[(off % 4) + n:].abs().max()) == 0.0
+
+
+def test_noise_same_draw_for_any_partition():
+    n = 70_001
+    a = torch.zeros(n, dtype=torch.float32, device=DEV)
+    b.dp_add_noise_and_scale(a, 1.0, 1.0, 1, 42, 9, elem_offset=0)
+    parts = torch.zeros(n, dtype=torch.float32, device=DEV)
+    cuts = [0, 1, 4, 4099, 30_000, n]
+    for lo, hi in zip(cuts[:-1], cuts[1:]):
+        b.dp_add_noise_and_scale(parts[lo:hi], 1.0, 1.0, 1, 42, 9, elem_offset=lo)
+    assert torch.equal(a, parts)
+    # another step gives another draw
+    c = torch.zeros(n, dtype=torch.float32, device=DEV)
+    b.dp_add_noise_and_scale(c, 1.0, 1.0, 1, 42, 10, elem_offset=0)
+    assert not torch.equal(a, c)
+    z = to_np(a)
+    assert abs(z.mean()) < 5 / np.sqrt(n) and abs(z.var() - 1) < 5 * np.sqrt(2 / n)
+
+
+def _adam_case(n, seed):
+    rng = np.random.default_rng(seed)
+    th = rng.standard_normal(n).astype(np.float32) * 0.02
+    m = rng.standard_normal(n).astype(np.float32) * 1e-3
+    v = (rng.standard_normal(n).astype(np.float32) * 1e-3) ** 2
+    g = rng.standard_normal(n).astype(np.float32) * 1e-3
+    g[::97] = 0.0
+    return th, m, v, g
+
+
+def _check_adam(got, ref, old_theta):
+    th, m, v = got
+    rt, rm, rv = ref
+    assert rel_max(m, rm) <= F32_TOL and rel_max(v, rv) <= F32_TOL
+    assert rel_max(th, rt) <= F32_TOL
+    d, rd = th - old_theta, rt - old_theta
+    # the update itself, not hidden behind theta: relative with a floor from fp32 rounding of theta
+    floor = 1e-7 * np.max(np.abs(old_theta)) + 1e-7 * np.max(np.abs(rd))
+    assert np.max(np.abs(d - rd)) <= F32_TOL * np.max(np.abs(rd)) + floor
+
+
+@pytest.mark.parametrize("hp", [
+    dict(lr=1e-3, b1=0.9, b2=0.999, xi=1e-11, wd=0.01, t=1),
+    dict(lr=6.0902e-4, b1=0.75, b2=0.9, xi=1e-11, wd=1.0, t=7),      # the paper's tuned values (Table 1)
+    dict(lr=6.0902e-4, b1=0.9, b2=0.999, xi=1e-11, wd=0.5, t=20000),
+])
+@pytest.mark.parametrize("n", [1 << 18, 1001])
+def test_adamw_matches_checker(hp, n):
+    th, m, v, g = _adam_case(n, n)
+    if hp["t"] == 1:
+        m[:] = 0
+        v[:] = 0
+    dth, dm, dv, dg = (torch.from_numpy(x.copy()).to(DEV) for x in (th, m, v, g))
+    b.dp_adamw_step(dth, dm, dv, dg, hp["lr"], hp["b1"], hp["b2"], hp["xi"], hp["wd"], hp["t"])
+    ref = O.adamw_step(th.astype(np.float64), m, v, g, hp["lr"], hp["b1"], hp["b2"], hp["xi"], hp["wd"], hp["t"])
+    _check_adam((to_np(dth), to_np(dm), to_np(dv)), ref, th.astype(np.float64))
+    assert torch.equal(dg.cpu(), torch.from_numpy(g))       # g is read-only
+
+
+def test_adamw_zero_state_zero_gradient_stays_finite():
+    n = 64
+    th = torch.ones(n, device=DEV)
+    z = torch.zeros(n, device=DEV)
+    m, v = z.clone(), z.clone()
+    b.dp_adamw_step(th, m, v, z, 1e-2, 0.9, 0.999, 1e-11, 0.5, 1)
+    assert torch.isfinite(th).all()
+    np.testing.assert_allclose(to_np(th), 1 - 1e-2 * 0.5, rtol=1e-6)
+
+
+@pytest.mark.parametrize("n,off", [(1 << 19, 0), (77_777, 0), (4097, 6)])
+def test_fused_pass_matches_split_calls_and_checker(n, off):
+    th, m, v, _ = _adam_case(n, 5)
+    rng = np.random.default_rng(9)
+    S = rng.standard_normal(n).astype(np.float32) * 50
+    hp = dict(lr=6.0902e-4, b1=0.9, b2=0.999, xi=1e-11, wd=0.5, t=3)
+    sigma, C, N, seed, step = 1.0, 1.0, 2048, 77, 3
+    # fused
+    f = [torch.from_numpy(x.copy()).to(DEV) for x in (th, m, v, S)]
+    b.dp_noise_scale_adamw_step(f[0], f[1], f[2], f[3], True, sigma, C, N, seed, step, hp["lr"], hp["b1"], hp["b2"],
+                                hp["xi"], hp["wd"], hp["t"], elem_offset=off)
+    assert float(f[3].abs().max()) == 0.0                   # accumulator cleared
+    # split
+    s = [torch.from_numpy(x.copy()).to(DEV) for x in (th, m, v, S)]
+    b.dp_add_noise_and_scale(s[3], sigma, C, N, seed, step, elem_offset=off)
+    b.dp_adamw_step(s[0], s[1], s[2], s[3], hp["lr"], hp["b1"], hp["b2"], hp["xi"], hp["wd"], hp["t"])
+    for x, y in zip(f[:3], s[:3]):
+        assert rel_max(to_np(x), to_np(y)) <= 1e-6
+    g = O.add_noise_and_scale(S.astype(np.float64), sigma, C, N, seed, step, elem_offset=off)
+    ref = O.adamw_step(th.astype(np.float64), m, v, g, hp["lr"], hp["b1"], hp["b2"], hp["xi"], hp["wd"], hp["t"])
+    _check_adam(tuple(to_np(x) for x in f[:3]), ref, th.astype(np.float64))
+    # zero_acc = 0 leaves the accumulator as it was
+    k = [torch.from_numpy(x.copy()).to(DEV) for x in (th, m, v, S)]
+    b.dp_noise_scale_adamw_step(k[0], k[1], k[2], k[3], False, sigma, C, N, seed, step, hp["lr"], hp["b1"],
+                                hp["b2"], hp["xi"], hp["wd"], hp["t"], elem_offset=off)
+    assert torch.equal(k[3].cpu(), torch.from_numpy(S))
+    assert torch.equal(k[0], f[0])
+
+
+def test_clip_factors_special_values():
+    C = 3.2429e-3
+    n = torch.tensor([0.0, C * C, 4 * C * C, 0.25 * C * C, 1e30, 1e-30], dtype=torch.float32, device=DEV)
+    c = torch.empty_like(n)
+    b.dp_clip_factors(n, C, c)
+    ref = O.clip_factors(to_np(n), C)
+    np.testing.assert_allclose(to_np(c), ref, rtol=1e-6)
