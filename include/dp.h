@@ -90,7 +90,7 @@ DP_API int dp_per_example_sqnorms(const dp_layer* layers /*HOST*/, int n_layers,
 
 /* c_i = min(1, C / sqrt(sqnorm_i)), c_i = 1 when sqnorm_i = 0: the factor of clip(., C) in
  * Algorithm 1.  C > 0. */
-DP_API int dp_clip_factors(const float* sqnorm, int B, float C, float* clip, void* cuda_stream);
+DP_API int dp_clip_factors(const float* sqnorm, int B, double C, float* clip, void* cuda_stream);
 
 /* acc += sum_i clip_i * g_i for every layer: the sum of clipped gradients of Algorithm 1,
  * accumulated over microbatches as in Section 5.3.  clip[B] fp32 from dp_clip_factors. */
@@ -101,21 +101,22 @@ DP_API int dp_clipped_accumulate(const dp_layer* layers /*HOST*/, int n_layers, 
  * z_e depends only on (seed, step, e) with e = elem_offset + index: Philox4x32-10 block e >> 2 with
  * counter (lo(e>>2), hi(e>>2), lo(step), hi(step)) and key (lo(seed), hi(seed)); Box-Muller on the word
  * pairs (x0,x1), (x2,x3).  n >= 0 elements; sigma >= 0, C > 0, batch_size > 0. */
-DP_API int dp_add_noise_and_scale(float* acc, int64_t n, int64_t elem_offset, float sigma, float C,
+DP_API int dp_add_noise_and_scale(float* acc, int64_t n, int64_t elem_offset, double sigma, double C,
                            int64_t batch_size, uint64_t seed, uint64_t step, void* cuda_stream);
 
 /* Adam with bias correction and decoupled weight decay (Algorithm 1):
  *   m <- b1 m + (1-b1) g;  v <- b2 v + (1-b2) g^2;
  *   theta <- theta - lr * ( (m/(1-b1^t)) / (sqrt(v/(1-b2^t)) + xi) + weight_decay * theta ),  t >= 1.
- * The bias corrections are formed on the host in double precision. */
-DP_API int dp_adamw_step(float* theta, float* m, float* v, const float* g, int64_t n, float lr, float beta1,
-                  float beta2, float xi, float weight_decay, int64_t t, void* cuda_stream);
+ * Scalars are doubles so that 1-beta and the bias corrections 1/(1-beta^t) are formed on the host in double
+ * precision before being rounded once to fp32 for the kernel. */
+DP_API int dp_adamw_step(float* theta, float* m, float* v, const float* g, int64_t n, double lr, double beta1,
+                  double beta2, double xi, double weight_decay, int64_t t, void* cuda_stream);
 
 /* The two calls above in one pass over memory (same arithmetic, same Philox indexing): reads acc, theta,
  * m, v and writes theta, m, v; with zero_acc != 0 it also clears acc for the next macro-batch. */
 DP_API int dp_noise_scale_adamw_step(float* theta, float* m, float* v, float* acc, int zero_acc, int64_t n,
-                              int64_t elem_offset, float sigma, float C, int64_t batch_size, uint64_t seed,
-                              uint64_t step, float lr, float beta1, float beta2, float xi, float weight_decay,
+                              int64_t elem_offset, double sigma, double C, int64_t batch_size, uint64_t seed,
+                              uint64_t step, double lr, double beta1, double beta2, double xi, double weight_decay,
                               int64_t t, void* cuda_stream);
 
 /* Test utility: out[k] = the raw Philox word of element elem_offset + k (lane (e & 3) of block e >> 2). */

@@ -50,7 +50,7 @@ def lib() -> C.CDLL:
             raise ImportError(f"{LIB_PATH} not found: run `python -m paper_2108_01624_b200.build` (needs nvcc). "
                               "There is no fallback implementation.")
         L = C.CDLL(LIB_PATH)
-        vp, i32, i64, u64, f32, sz = C.c_void_p, C.c_int, C.c_int64, C.c_uint64, C.c_float, C.c_size_t
+        vp, i32, i64, u64, f32, sz = C.c_void_p, C.c_int, C.c_int64, C.c_uint64, C.c_double, C.c_size_t
         L.dp_workspace_bytes.restype = sz
         L.dp_workspace_bytes.argtypes = [vp, i32]
         L.dp_per_example_sqnorms.argtypes = [vp, i32, vp, i32, vp, sz, vp]

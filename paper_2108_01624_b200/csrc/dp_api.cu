@@ -25,7 +25,6 @@ static int* status_ptr() {
   return cache[dev];
 }
 
-static bool finite_f(float x) { return std::isfinite(x); }
 static size_t elem_size(int dtype) { return dtype == DP_F32 ? 4 : 2; }
 static bool misaligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) != 0; }
 
@@ -143,7 +142,16 @@ int dp_per_example_sqnorms(const dp_layer* layers, int n_layers, float* sqnorm, 
   size_t u = 0;
   for (int l = 0; l < n_layers; ++l) {
     const dp_layer& L = layers[l];
-    if (u < plan.umma_idx.size() && plan.umma_idx[u] == l) { ++u; continue; }
+    if (u < plan.umma_idx.size() && plan.umma_idx[u] == l) {
+      // The materialised-tile kernel covers the weight gradient only; the bias part |sum_t G_i[t,:]|^2 is a
+      // bandwidth-bound column sum (the Gram kernel has it built in as the +1 on the token Gram of A).
+      if (!plan.umma_gram[u] && L.has_bias) {
+        DP_CUDA(launch_bias_colsums(L, colsum, s));
+        DP_CUDA(launch_rows_sqsum(colsum, B, L.d_out, sqnorm, s));
+      }
+      ++u;
+      continue;
+    }
     if (L.kind == DP_LINEAR) {
       DP_CUDA(launch_linear_sqnorm_generic(L, use_gram(L), sqnorm, s));
     } else if (L.kind == DP_LAYERNORM) {
@@ -156,11 +164,11 @@ int dp_per_example_sqnorms(const dp_layer* layers, int n_layers, float* sqnorm, 
   return DP_OK;
 }
 
-int dp_clip_factors(const float* sqnorm, int B, float C, float* clip, void* cuda_stream) {
+int dp_clip_factors(const float* sqnorm, int B, double C, float* clip, void* cuda_stream) {
   if (!sqnorm || !clip || B <= 0) return DP_ERR_ARG;
-  if (!(C > 0.0f) || !finite_f(C)) return DP_ERR_ARG;
+  if (!(C > 0.0) || !std::isfinite(C)) return DP_ERR_ARG;
   if (misaligned(sqnorm, 4) || misaligned(clip, 4)) return DP_ERR_ALIGN;
-  DP_CUDA(launch_clip_factors(sqnorm, B, C, clip, static_cast<cudaStream_t>(cuda_stream)));
+  DP_CUDA(launch_clip_factors(sqnorm, B, (float)C, clip, static_cast<cudaStream_t>(cuda_stream)));
   return DP_OK;
 }
 
@@ -201,11 +209,11 @@ int dp_clipped_accumulate(const dp_layer* layers, int n_layers, const float* cli
   return DP_OK;
 }
 
-static int make_noise_args(int64_t n, int64_t elem_offset, float sigma, float C, int64_t batch_size, uint64_t seed,
+static int make_noise_args(int64_t n, int64_t elem_offset, double sigma, double C, int64_t batch_size, uint64_t seed,
                            uint64_t step, NoiseArgs* na) {
   if (n < 0 || elem_offset < 0 || batch_size <= 0) return DP_ERR_ARG;
-  if (!finite_f(sigma) || sigma < 0.0f || !finite_f(C) || !(C > 0.0f)) return DP_ERR_ARG;
-  na->sigmaC = sigma * C;
+  if (!std::isfinite(sigma) || sigma < 0.0 || !std::isfinite(C) || !(C > 0.0)) return DP_ERR_ARG;
+  na->sigmaC = (float)(sigma * C);
   na->inv_n = (float)(1.0 / (double)batch_size);
   na->key0 = (uint32_t)seed;
   na->key1 = (uint32_t)(seed >> 32);
@@ -215,19 +223,19 @@ static int make_noise_args(int64_t n, int64_t elem_offset, float sigma, float C,
   return DP_OK;
 }
 
-static int make_adam_args(float lr, float b1, float b2, float xi, float wd, int64_t t, AdamArgs* aa) {
+static int make_adam_args(double lr, double b1, double b2, double xi, double wd, int64_t t, AdamArgs* aa) {
   if (t < 1) return DP_ERR_ARG;
-  if (!finite_f(lr) || !finite_f(xi) || !finite_f(wd) || xi < 0.0f) return DP_ERR_ARG;
-  if (!(b1 >= 0.0f && b1 < 1.0f) || !(b2 >= 0.0f && b2 < 1.0f)) return DP_ERR_ARG;
-  aa->lr = lr; aa->beta1 = b1; aa->beta2 = b2; aa->xi = xi; aa->wd = wd;
-  aa->one_m_beta1 = (float)(1.0 - (double)b1);
-  aa->one_m_beta2 = (float)(1.0 - (double)b2);
-  aa->bias1 = (float)(1.0 / (1.0 - std::pow((double)b1, (double)t)));
-  aa->bias2 = (float)(1.0 / (1.0 - std::pow((double)b2, (double)t)));
+  if (!std::isfinite(lr) || !std::isfinite(xi) || !std::isfinite(wd) || xi < 0.0) return DP_ERR_ARG;
+  if (!(b1 >= 0.0 && b1 < 1.0) || !(b2 >= 0.0 && b2 < 1.0)) return DP_ERR_ARG;
+  aa->lr = (float)lr; aa->beta1 = (float)b1; aa->beta2 = (float)b2; aa->xi = (float)xi; aa->wd = (float)wd;
+  aa->one_m_beta1 = (float)(1.0 - b1);
+  aa->one_m_beta2 = (float)(1.0 - b2);
+  aa->bias1 = (float)(1.0 / (1.0 - std::pow(b1, (double)t)));
+  aa->bias2 = (float)(1.0 / (1.0 - std::pow(b2, (double)t)));
   return DP_OK;
 }
 
-int dp_add_noise_and_scale(float* acc, int64_t n, int64_t elem_offset, float sigma, float C, int64_t batch_size,
+int dp_add_noise_and_scale(float* acc, int64_t n, int64_t elem_offset, double sigma, double C, int64_t batch_size,
                            uint64_t seed, uint64_t step, void* cuda_stream) {
   NoiseArgs na;
   int rc = make_noise_args(n, elem_offset, sigma, C, batch_size, seed, step, &na);
@@ -239,8 +247,8 @@ int dp_add_noise_and_scale(float* acc, int64_t n, int64_t elem_offset, float sig
   return DP_OK;
 }
 
-int dp_adamw_step(float* theta, float* m, float* v, const float* g, int64_t n, float lr, float beta1, float beta2,
-                  float xi, float weight_decay, int64_t t, void* cuda_stream) {
+int dp_adamw_step(float* theta, float* m, float* v, const float* g, int64_t n, double lr, double beta1, double beta2,
+                  double xi, double weight_decay, int64_t t, void* cuda_stream) {
   AdamArgs aa;
   if (n < 0) return DP_ERR_ARG;
   int rc = make_adam_args(lr, beta1, beta2, xi, weight_decay, t, &aa);
@@ -253,8 +261,8 @@ int dp_adamw_step(float* theta, float* m, float* v, const float* g, int64_t n, f
 }
 
 int dp_noise_scale_adamw_step(float* theta, float* m, float* v, float* acc, int zero_acc, int64_t n,
-                              int64_t elem_offset, float sigma, float C, int64_t batch_size, uint64_t seed,
-                              uint64_t step, float lr, float beta1, float beta2, float xi, float weight_decay,
+                              int64_t elem_offset, double sigma, double C, int64_t batch_size, uint64_t seed,
+                              uint64_t step, double lr, double beta1, double beta2, double xi, double weight_decay,
                               int64_t t, void* cuda_stream) {
   NoiseArgs na;
   AdamArgs aa;

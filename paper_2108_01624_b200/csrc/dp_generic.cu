@@ -299,9 +299,12 @@ __global__ void __launch_bounds__(256) k_rows_sqsum(const float* __restrict__ ws
   t = block_sum(t, red);
   if (threadIdx.x == 0) sqnorm[blockIdx.x] += t;
 }
-cudaError_t launch_layernorm_sqnorm(const dp_layer& L, const float* ws, float* sqnorm, cudaStream_t s) {
-  k_rows_sqsum<<<L.B, 256, 0, s>>>(ws, 2 * L.d_out, sqnorm);
+cudaError_t launch_rows_sqsum(const float* ws, int B, int width, float* sqnorm, cudaStream_t s) {
+  k_rows_sqsum<<<B, 256, 0, s>>>(ws, width, sqnorm);
   return counted(1);
+}
+cudaError_t launch_layernorm_sqnorm(const dp_layer& L, const float* ws, float* sqnorm, cudaStream_t s) {
+  return launch_rows_sqsum(ws, L.B, 2 * L.d_out, sqnorm, s);
 }
 
 // dst[j] += sum_i clip[i] * ws[i][off + j], j < d; rows of ws are `width` apart.  64 columns x 4 example groups.

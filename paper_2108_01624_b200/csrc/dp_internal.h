@@ -49,6 +49,8 @@ cudaError_t launch_linear_accum_generic(const dp_layer& L, const float* clip, cu
 // LayerNorm: per-example column sums into ws[B][2d] (gain part then bias part), then either the norm
 // or the clip-weighted reduction over examples.
 cudaError_t launch_layernorm_colsums(const dp_layer& L, float* ws, cudaStream_t s);
+// sqnorm[i] += sum_j ws[i][j]^2, j < width (rows of ws are `width` apart).
+cudaError_t launch_rows_sqsum(const float* ws, int B, int width, float* sqnorm, cudaStream_t s);
 cudaError_t launch_layernorm_sqnorm(const dp_layer& L, const float* ws, float* sqnorm, cudaStream_t s);
 cudaError_t launch_layernorm_accum(const dp_layer& L, const float* ws, const float* clip, cudaStream_t s);
 // Embedding by grouping equal ids inside an example.

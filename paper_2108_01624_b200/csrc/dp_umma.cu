@@ -1,9 +1,668 @@
-// placeholder until the tcgen05 kernels land
+// tcgen05 / TMEM / TMA kernels for bf16 linear layers (sm_100a).
+//
+//   k_gram_sqnorm  per-example squared norm by the token-Gram identity
+//                  |A_i^T G_i|_F^2 + |1^T G_i|^2 = < A_i A_i^T + [bias] 1 1^T , G_i G_i^T >.
+//                  Both 128x128 fp32 Grams of a token-block pair live in TMEM (2 x 128 columns,
+//                  double-buffered); operands are K-major 128x64 tiles fetched by TMA.
+//   k_tile<ACCUM>  acc_w^T tile (128 of d_out x 256 of d_in) += sum over tokens of G^T diag(c) A: one
+//                  128x256x16 UMMA per 16 tokens, both operands MN-major straight from the row-major
+//                  activations.  The per-example factor c is applied to the 128-wide G tile in shared
+//                  memory by four transform warps (fp32 multiply, one bf16 rounding), which also form
+//                  the bias column sums, so A and G are read from HBM exactly once.
+//   k_tile<SQNORM> the materialised-tile norm: the same tiles for ONE example, squared and summed.
+//
+// All three are persistent kernels (grid = number of SMs) over a work list decoded on the device from
+// per-layer tile counts; roles are warp-specialised (TMA producer / MMA issuer / epilogue / transform).
+#include <cuda.h>
+
+#include <vector>
+
 #include "dp_internal.h"
+#include "dp_ptx.cuh"
+
 namespace dpk {
-bool umma_supported(const dp_layer&) { return false; }
-bool umma_accumulates_bias() { return false; }
-size_t umma_sqnorm_partials_per_example(const dp_layer*, const int*, int, const int*) { return 0; }
-int launch_umma_sqnorms(const dp_layer*, const int*, int, const int*, float*, int, int, int*, cudaStream_t) { return DP_ERR_UNSUPPORTED; }
-int launch_umma_accumulate(const dp_layer*, const int*, int, const float*, int*, cudaStream_t) { return DP_ERR_UNSUPPORTED; }
+using namespace ptx;
+
+constexpr int kMaxLayers = 96;
+
+struct alignas(64) UmmaLayer {
+  CUtensorMap mapG;   // [B, T, d_out] bf16
+  CUtensorMap mapA;   // [B, T, d_in]  bf16
+  float* acc_w;
+  float* acc_b;
+  int d_out, d_in;
+  int tiles_m, tiles_n;   // tile kernels: 128-wide tiles over d_out, 256-wide tiles over d_in
+  int item_start;         // first work item of this layer within the launch
+  int partial_base;       // first per-example partial slot of this layer
+  int has_bias, pad;
+};
+
+struct UmmaParams {
+  UmmaLayer L[kMaxLayers];
+  int n_layers, total_items, B, T;
+  int box_rows;           // token rows per TMA box (min(tile rows, T))
+  int splits;             // accumulate: number of example ranges a tile is split into
+  int partial_stride, pad;
+  const float* clip;
+  float* partial;
+  int* status;
+};
+static_assert(sizeof(UmmaParams) <= 32000, "kernel parameter block too large");
+
+__device__ __forceinline__ int find_layer(const UmmaParams& P, int item) {
+  int l = 0;
+  while (l + 1 < P.n_layers && item >= P.L[l + 1].item_start) ++l;
+  return l;
 }
+
+__device__ __forceinline__ uint8_t* align1024(uint8_t* p) {
+  return reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(p) + 1023) & ~uintptr_t(1023));
+}
+
+// =================================================================================================
+// Gram kernel
+// =================================================================================================
+constexpr int G_SLOTS = 12;
+constexpr int G_SLOT_BYTES = 128 * 128;          // 128 tokens x 64 bf16 features, 128-byte swizzle
+constexpr int G_THREADS = 192;                   // warp 0: TMA, warp 1: MMA, warps 2..5: epilogue
+constexpr uint32_t G_IDESC = idesc_bf16_f32(128, 128, false, false);
+
+struct GramCtl {
+  uint64_t full[G_SLOTS], empty[G_SLOTS], tmem_full[2], tmem_empty[2], drain;
+  uint32_t tmem_base;
+  int abort;
+};
+constexpr int G_SMEM = 1024 + G_SLOTS * G_SLOT_BYTES + (int)sizeof(GramCtl);
+
+// item -> (layer, example, token-block pair r <= c)
+__device__ __forceinline__ void gram_decode(const UmmaParams& P, int item, int npairs, int nblk, int& l, int& i, int& pair,
+                                            int& r, int& c) {
+  l = find_layer(P, item);
+  const int rem = item - P.L[l].item_start;
+  i = rem / npairs;
+  pair = rem - i * npairs;
+  int p = pair;
+  r = 0;
+  while (p >= nblk - r) { p -= nblk - r; ++r; }
+  c = r + p;
+}
+
+__global__ void __launch_bounds__(G_THREADS, 1) k_gram_sqnorm(const __grid_constant__ UmmaParams P) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* tiles = align1024(smem_raw);
+  GramCtl* S = reinterpret_cast<GramCtl*>(tiles + G_SLOTS * G_SLOT_BYTES);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  volatile int* abort_flag = &S->abort;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < G_SLOTS; ++s) { mbar_init(&S->full[s], 1); mbar_init(&S->empty[s], 1); }
+    for (int b = 0; b < 2; ++b) { mbar_init(&S->tmem_full[b], 1); mbar_init(&S->tmem_empty[b], 4); }
+    mbar_init(&S->drain, 1);
+    S->abort = 0;
+    fence_mbar_init();
+  }
+  if (P.box_rows < 128) {   // rows the TMA box never writes must read as zero tokens
+    for (int k = threadIdx.x; k < G_SLOTS * G_SLOT_BYTES / 16; k += G_THREADS)
+      reinterpret_cast<uint4*>(tiles)[k] = make_uint4(0, 0, 0, 0);
+    fence_proxy_async_smem();
+  }
+  if (warp == 1) { tmem_alloc(&S->tmem_base, 512); tmem_relinquish(); }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = S->tmem_base;
+  const int nblk = (P.T + 127) / 128, npairs = nblk * (nblk + 1) / 2;
+  const uint32_t box_bytes = (uint32_t)P.box_rows * 128u;
+
+  if (warp == 0) {
+    if (lane == 0) {   // ---------------- TMA producer ----------------
+      uint32_t it = 0;
+      bool alive = true;
+      for (int item = blockIdx.x; item < P.total_items && alive; item += gridDim.x) {
+        int l, i, pair, r, c;
+        gram_decode(P, item, npairs, nblk, l, i, pair, r, c);
+        const UmmaLayer& L = P.L[l];
+        for (int which = 0; which < 2 && alive; ++which) {
+          const CUtensorMap* map = which ? &L.mapG : &L.mapA;
+          const int d = which ? L.d_out : L.d_in;
+          for (int k0 = 0; k0 < d && alive; k0 += 64) {
+            for (int half = 0; half < (r == c ? 1 : 2); ++half) {
+              const uint32_t slot = it % G_SLOTS, ph = (it / G_SLOTS) & 1u;
+              if (!mbar_wait(&S->empty[slot], ph ^ 1u, abort_flag, P.status)) { alive = false; break; }
+              mbar_arrive_expect_tx(&S->full[slot], box_bytes);
+              tma_load_3d(tiles + slot * G_SLOT_BYTES, map, &S->full[slot], k0, (half ? c : r) * 128, i);
+              ++it;
+            }
+          }
+        }
+      }
+      // Leave no copy in flight: every issued slot must have landed before shared memory is released.
+      const uint32_t pending = it < (uint32_t)G_SLOTS ? it : (uint32_t)G_SLOTS;
+      for (uint32_t k = 0; k < pending; ++k) {
+        const uint32_t j = it - 1 - k;
+        mbar_wait_drain(&S->full[j % G_SLOTS], (j / G_SLOTS) & 1u, P.status);
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {   // ---------------- MMA issuer ----------------
+      uint32_t it = 0, tile_it = 0;
+      bool alive = true;
+      for (int item = blockIdx.x; item < P.total_items && alive; item += gridDim.x, ++tile_it) {
+        int l, i, pair, r, c;
+        gram_decode(P, item, npairs, nblk, l, i, pair, r, c);
+        const UmmaLayer& L = P.L[l];
+        const uint32_t buf = tile_it & 1u, tph = (tile_it >> 1) & 1u;
+        if (!mbar_wait(&S->tmem_empty[buf], tph ^ 1u, abort_flag, P.status)) { alive = false; break; }
+        tc_fence_after();
+        for (int which = 0; which < 2 && alive; ++which) {
+          const int d = which ? L.d_out : L.d_in;
+          const uint32_t d_tmem = tmem_base + buf * 256u + (uint32_t)which * 128u;
+          for (int k0 = 0; k0 < d; k0 += 64) {
+            const uint32_t sr = it % G_SLOTS, pr = (it / G_SLOTS) & 1u;
+            ++it;
+            if (!mbar_wait(&S->full[sr], pr, abort_flag, P.status)) { alive = false; break; }
+            uint32_t sc = sr;
+            if (r != c) {
+              sc = it % G_SLOTS;
+              const uint32_t pc = (it / G_SLOTS) & 1u;
+              ++it;
+              if (!mbar_wait(&S->full[sc], pc, abort_flag, P.status)) { alive = false; break; }
+            }
+            tc_fence_after();
+            const uint32_t ar = smem_u32(tiles + sr * G_SLOT_BYTES), ac = smem_u32(tiles + sc * G_SLOT_BYTES);
+#pragma unroll
+            for (int k4 = 0; k4 < 4; ++k4) {
+              umma_bf16(d_tmem, smem_desc_sw128(ar + k4 * 32, 16, 1024), smem_desc_sw128(ac + k4 * 32, 16, 1024),
+                        G_IDESC, (k0 | k4) ? 1u : 0u);
+            }
+            umma_commit(&S->empty[sr]);
+            if (r != c) umma_commit(&S->empty[sc]);
+          }
+        }
+        if (alive) umma_commit(&S->tmem_full[buf]);
+      }
+      // Drain: all issued MMAs must have completed before TMEM and shared memory are released.
+      umma_commit(&S->drain);
+      mbar_wait_drain(&S->drain, 0u, P.status);
+    }
+  } else {   // ---------------- epilogue warps 2..5 ----------------
+    const uint32_t q = (uint32_t)warp & 3u;
+    uint32_t tile_it = 0;
+    bool alive = true;
+    for (int item = blockIdx.x; item < P.total_items; item += gridDim.x, ++tile_it) {
+      int l, i, pair, r, c;
+      gram_decode(P, item, npairs, nblk, l, i, pair, r, c);
+      const UmmaLayer& L = P.L[l];
+      const uint32_t buf = tile_it & 1u, tph = (tile_it >> 1) & 1u;
+      if (alive) alive = __all_sync(0xffffffffu, mbar_wait(&S->tmem_full[buf], tph, abort_flag, P.status));
+      if (!alive) continue;
+      tc_fence_after();
+      const float bias1 = L.has_bias ? 1.0f : 0.0f;
+      float sum = 0.0f;
+#pragma unroll 1
+      for (int ch = 0; ch < 4; ++ch) {
+        uint32_t pv[32], qv[32];
+        const uint32_t ta = tmem_base + ((q * 32u) << 16) + buf * 256u + (uint32_t)ch * 32u;
+        tmem_ld_32x32(ta, pv);
+        tmem_ld_32x32(ta + 128u, qv);
+        tmem_ld_wait();
+#pragma unroll
+        for (int j = 0; j < 32; ++j) sum = fmaf(__uint_as_float(pv[j]) + bias1, __uint_as_float(qv[j]), sum);
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&S->tmem_empty[buf]);
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) sum += __shfl_down_sync(0xffffffffu, sum, o);
+      if (lane == 0)
+        P.partial[(size_t)i * P.partial_stride + L.partial_base + pair * 4 + (int)q] = (r == c) ? sum : 2.0f * sum;
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    __syncwarp();
+    tc_fence_after();
+    tmem_dealloc(tmem_base, 512);
+  }
+}
+
+// =================================================================================================
+// Tile kernel: 128 (d_out) x 256 (d_in) output tiles, K = tokens
+// =================================================================================================
+constexpr int T_STAGES = 4;
+constexpr int T_ATOM_BYTES = 64 * 128;                 // 64 tokens x 64 bf16 features
+constexpr int T_M_BYTES = 2 * T_ATOM_BYTES;            // G tile: 128 features of d_out
+constexpr int T_N_BYTES = 4 * T_ATOM_BYTES;            // A tile: 256 features of d_in
+constexpr int T_STAGE_BYTES = T_M_BYTES + T_N_BYTES;   // 48 KB
+constexpr uint32_t T_IDESC = idesc_bf16_f32(128, 256, true, true);
+
+struct TileCtl {
+  uint64_t full[T_STAGES], empty[T_STAGES], ready[T_STAGES], tmem_full[2], tmem_empty[2], drain;
+  uint32_t tmem_base;
+  int abort;
+  float colsum[8][128];
+};
+constexpr int T_SMEM = 1024 + T_STAGES * T_STAGE_BYTES + (int)sizeof(TileCtl);
+
+struct TileItem { int l, m0, n0, e0, e1, nt, slot; };
+
+template <bool ACCUM>
+__device__ __forceinline__ TileItem tile_decode(const UmmaParams& P, int item) {
+  TileItem t;
+  t.l = find_layer(P, item);
+  const UmmaLayer& L = P.L[t.l];
+  const int rem = item - L.item_start, tiles = L.tiles_m * L.tiles_n;
+  const int outer = rem / tiles, tile = rem - outer * tiles;
+  const int mt = tile / L.tiles_n;
+  t.nt = tile - mt * L.tiles_n;
+  t.m0 = mt * 128;
+  t.n0 = t.nt * 256;
+  if (ACCUM) {            // outer = split index over example ranges
+    t.e0 = (int)((long long)outer * P.B / P.splits);
+    t.e1 = (int)((long long)(outer + 1) * P.B / P.splits);
+    t.slot = 0;
+  } else {                // outer = example
+    t.e0 = outer;
+    t.e1 = outer + 1;
+    t.slot = L.partial_base + tile * 4;
+  }
+  return t;
+}
+
+template <bool ACCUM>
+__global__ void __launch_bounds__(ACCUM ? 320 : 192, 1) k_tile(const __grid_constant__ UmmaParams P) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* tiles = align1024(smem_raw);
+  TileCtl* S = reinterpret_cast<TileCtl*>(tiles + T_STAGES * T_STAGE_BYTES);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  volatile int* abort_flag = &S->abort;
+  constexpr int NT = ACCUM ? 320 : 192;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < T_STAGES; ++s) {
+      mbar_init(&S->full[s], 1);
+      mbar_init(&S->empty[s], 1);
+      mbar_init(&S->ready[s], 128);
+    }
+    for (int b = 0; b < 2; ++b) { mbar_init(&S->tmem_full[b], 1); mbar_init(&S->tmem_empty[b], 4); }
+    mbar_init(&S->drain, 1);
+    S->abort = 0;
+    fence_mbar_init();
+  }
+  if (P.box_rows < 64) {
+    for (int k = threadIdx.x; k < T_STAGES * T_STAGE_BYTES / 16; k += NT)
+      reinterpret_cast<uint4*>(tiles)[k] = make_uint4(0, 0, 0, 0);
+    fence_proxy_async_smem();
+  }
+  if (warp == 1) { tmem_alloc(&S->tmem_base, 512); tmem_relinquish(); }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = S->tmem_base;
+  const int n_tb = (P.T + 63) / 64;
+  const uint32_t box_bytes = (uint32_t)P.box_rows * 128u;
+
+  if (warp == 0) {
+    if (lane == 0) {   // ---------------- TMA producer ----------------
+      uint32_t it = 0;
+      bool alive = true;
+      for (int item = blockIdx.x; item < P.total_items && alive; item += gridDim.x) {
+        const TileItem t = tile_decode<ACCUM>(P, item);
+        const UmmaLayer& L = P.L[t.l];
+        for (int e = t.e0; e < t.e1 && alive; ++e) {
+          for (int tb = 0; tb < n_tb; ++tb) {
+            const uint32_t slot = it % T_STAGES, ph = (it / T_STAGES) & 1u;
+            if (!mbar_wait(&S->empty[slot], ph ^ 1u, abort_flag, P.status)) { alive = false; break; }
+            uint8_t* st = tiles + slot * T_STAGE_BYTES;
+            mbar_arrive_expect_tx(&S->full[slot], 6u * box_bytes);
+#pragma unroll
+            for (int a = 0; a < 2; ++a) tma_load_3d(st + a * T_ATOM_BYTES, &L.mapG, &S->full[slot], t.m0 + a * 64, tb * 64, e);
+#pragma unroll
+            for (int a = 0; a < 4; ++a)
+              tma_load_3d(st + T_M_BYTES + a * T_ATOM_BYTES, &L.mapA, &S->full[slot], t.n0 + a * 64, tb * 64, e);
+            ++it;
+          }
+        }
+      }
+      const uint32_t pending = it < (uint32_t)T_STAGES ? it : (uint32_t)T_STAGES;
+      for (uint32_t k = 0; k < pending; ++k) {
+        const uint32_t j = it - 1 - k;
+        mbar_wait_drain(&S->full[j % T_STAGES], (j / T_STAGES) & 1u, P.status);
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {   // ---------------- MMA issuer ----------------
+      uint32_t it = 0, tile_it = 0;
+      bool alive = true;
+      for (int item = blockIdx.x; item < P.total_items && alive; item += gridDim.x, ++tile_it) {
+        const TileItem t = tile_decode<ACCUM>(P, item);
+        const uint32_t buf = tile_it & 1u, tph = (tile_it >> 1) & 1u;
+        if (!mbar_wait(&S->tmem_empty[buf], tph ^ 1u, abort_flag, P.status)) { alive = false; break; }
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + buf * 256u;
+        uint32_t first = 0;
+        for (int e = t.e0; e < t.e1 && alive; ++e) {
+          for (int tb = 0; tb < n_tb; ++tb) {
+            const uint32_t slot = it % T_STAGES, ph = (it / T_STAGES) & 1u;
+            ++it;
+            if (!mbar_wait(ACCUM ? &S->ready[slot] : &S->full[slot], ph, abort_flag, P.status)) { alive = false; break; }
+            tc_fence_after();
+            const uint32_t am = smem_u32(tiles + slot * T_STAGE_BYTES), an = am + T_M_BYTES;
+#pragma unroll
+            for (int k4 = 0; k4 < 4; ++k4) {
+              umma_bf16(d_tmem, smem_desc_sw128(am + k4 * 2048, T_ATOM_BYTES, 1024),
+                        smem_desc_sw128(an + k4 * 2048, T_ATOM_BYTES, 1024), T_IDESC, first | (uint32_t)k4);
+            }
+            first = 1;
+            umma_commit(&S->empty[slot]);
+          }
+        }
+        if (alive) umma_commit(&S->tmem_full[buf]);
+      }
+      umma_commit(&S->drain);
+      mbar_wait_drain(&S->drain, 0u, P.status);
+    }
+  } else if (warp < 6) {   // ---------------- epilogue warps 2..5 ----------------
+    const uint32_t q = (uint32_t)warp & 3u;
+    uint32_t tile_it = 0;
+    bool alive = true;
+    for (int item = blockIdx.x; item < P.total_items; item += gridDim.x, ++tile_it) {
+      const TileItem t = tile_decode<ACCUM>(P, item);
+      const UmmaLayer& L = P.L[t.l];
+      const uint32_t buf = tile_it & 1u, tph = (tile_it >> 1) & 1u;
+      if (alive) alive = __all_sync(0xffffffffu, mbar_wait(&S->tmem_full[buf], tph, abort_flag, P.status));
+      if (!alive) continue;
+      tc_fence_after();
+      const int m = t.m0 + (int)q * 32 + lane;
+      float sum = 0.0f;
+#pragma unroll 1
+      for (int ch = 0; ch < 8; ++ch) {
+        uint32_t v[32];
+        tmem_ld_32x32(tmem_base + ((q * 32u) << 16) + buf * 256u + (uint32_t)ch * 32u, v);
+        tmem_ld_wait();
+        if (ACCUM) {
+          const int nb = t.n0 + ch * 32;
+          if (m < L.d_out && nb < L.d_in) {
+            float* p = L.acc_w + (size_t)nb * L.d_out + m;
+            const int nv = (L.d_in - nb) < 32 ? (L.d_in - nb) : 32;
+            if (P.splits > 1) {
+#pragma unroll
+              for (int j = 0; j < 32; ++j)
+                if (j < nv) atomicAdd(p + (size_t)j * L.d_out, __uint_as_float(v[j]));
+            } else {
+              float old[32];
+#pragma unroll
+              for (int j = 0; j < 32; ++j) old[j] = (j < nv) ? p[(size_t)j * L.d_out] : 0.0f;
+#pragma unroll
+              for (int j = 0; j < 32; ++j)
+                if (j < nv) p[(size_t)j * L.d_out] = old[j] + __uint_as_float(v[j]);
+            }
+          }
+        } else {
+#pragma unroll
+          for (int j = 0; j < 32; ++j) sum = fmaf(__uint_as_float(v[j]), __uint_as_float(v[j]), sum);
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&S->tmem_empty[buf]);
+      if (!ACCUM) {
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) sum += __shfl_down_sync(0xffffffffu, sum, o);
+        if (lane == 0) P.partial[(size_t)t.e0 * P.partial_stride + t.slot + (int)q] = sum;
+      }
+    }
+  } else if (ACCUM) {   // ---------------- transform warps 6..9: scale the G tile, bias column sums ----------------
+    const int tt = threadIdx.x - 192;                 // 0..127
+    const int a = tt >> 6, kk = (tt & 63) >> 3, jp = tt & 7;
+    uint32_t it = 0;
+    bool alive = true;
+    for (int item = blockIdx.x; item < P.total_items; item += gridDim.x) {
+      const TileItem t = tile_decode<true>(P, item);
+      const UmmaLayer& L = P.L[t.l];
+      const bool need_bias = L.has_bias && t.nt == 0;
+      float col[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) col[u] = 0.0f;
+      for (int e = t.e0; e < t.e1; ++e) {
+        const float cf = alive ? __ldg(P.clip + e) : 1.0f;
+        for (int tb = 0; tb < n_tb; ++tb) {
+          const uint32_t slot = it % T_STAGES, ph = (it / T_STAGES) & 1u;
+          ++it;
+          if (alive && !mbar_wait(&S->full[slot], ph, abort_flag, P.status)) alive = false;
+          if (!alive) continue;
+          if (cf != 1.0f || need_bias) {
+            uint8_t* base = tiles + slot * T_STAGE_BYTES + a * T_ATOM_BYTES + kk * 128 + jp * 16;
+#pragma unroll
+            for (int i8 = 0; i8 < 8; ++i8) {
+              uint4* p = reinterpret_cast<uint4*>(base + i8 * 1024);
+              uint4 w = *p;
+              uint32_t x[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+              for (int u = 0; u < 4; ++u) {
+                const float lo = __uint_as_float(x[u] << 16) * cf;
+                const float hi = __uint_as_float(x[u] & 0xffff0000u) * cf;
+                col[2 * u] += lo;
+                col[2 * u + 1] += hi;
+                const __nv_bfloat162 pk = __floats2bfloat162_rn(lo, hi);
+                x[u] = *reinterpret_cast<const uint32_t*>(&pk);
+              }
+              if (cf != 1.0f) *p = make_uint4(x[0], x[1], x[2], x[3]);
+            }
+            fence_proxy_async_smem();
+          }
+          mbar_arrive(&S->ready[slot]);
+        }
+      }
+      if (need_bias) {      // uniform over the 128 transform threads; executed even after an abort
+        const int j = jp ^ kk;                        // logical 16-byte chunk under the 128-byte swizzle
+#pragma unroll
+        for (int u = 0; u < 8; ++u) S->colsum[kk][a * 64 + j * 8 + u] = col[u];
+        asm volatile("bar.sync 2, 128;" ::: "memory");
+        const int mcol = t.m0 + tt;
+        if (alive && mcol < L.d_out) {
+          float s = 0.0f;
+#pragma unroll
+          for (int r8 = 0; r8 < 8; ++r8) s += S->colsum[r8][tt];
+          if (P.splits > 1) atomicAdd(L.acc_b + mcol, s); else L.acc_b[mcol] += s;
+        }
+        asm volatile("bar.sync 2, 128;" ::: "memory");
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    __syncwarp();
+    tc_fence_after();
+    tmem_dealloc(tmem_base, 512);
+  }
+}
+
+// =================================================================================================
+// Host side: tensor maps, work lists, launches
+// =================================================================================================
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// The driver entry point is resolved at run time so that the library loads on machines without a driver.
+static EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+// bf16 tensor [B, T, d] viewed as (x = feature, y = token, z = example); box = 64 features x box_rows tokens,
+// 128-byte swizzle, out-of-range elements read as zero.
+static bool encode_map(CUtensorMap* map, const void* base, int B, int T, int d, int box_rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[3] = {(cuuint64_t)d, (cuuint64_t)T, (cuuint64_t)B};
+  const cuuint64_t strides[2] = {(cuuint64_t)d * 2, (cuuint64_t)T * d * 2};
+  const cuuint32_t box[3] = {64u, (cuuint32_t)box_rows, 1u};
+  const cuuint32_t estr[3] = {1u, 1u, 1u};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+bool umma_supported(const dp_layer& L) {
+  if (L.kind != DP_LINEAR || L.dtype != DP_BF16) return false;
+  if (L.d_in % 64 != 0 || L.d_out % 64 != 0) return false;
+  if ((reinterpret_cast<uintptr_t>(L.A) | reinterpret_cast<uintptr_t>(L.G)) & 15u) return false;
+  if ((long long)L.T * (L.d_in > L.d_out ? L.d_in : L.d_out) * 2 >= (1ll << 40)) return false;
+  return true;
+}
+bool umma_accumulates_bias() { return true; }
+
+static int gram_pairs(int T) { const int nb = (T + 127) / 128; return nb * (nb + 1) / 2; }
+static int tile_count(const dp_layer& L) { return ceil_div(L.d_out, 128) * ceil_div(L.d_in, 256); }
+
+size_t umma_sqnorm_partials_per_example(const dp_layer* layers, const int* idx, int n, const int* use_gram) {
+  size_t c = 0;
+  for (int k = 0; k < n; ++k) c += 4 * (size_t)(use_gram[k] ? gram_pairs(layers[idx[k]].T) : tile_count(layers[idx[k]]));
+  return c;
+}
+
+static int sm_count() {
+  static int sms = 0;
+  if (!sms) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (sms <= 0) sms = 148;
+  }
+  return sms;
+}
+
+template <typename K>
+static bool ensure_smem(K kernel, int bytes) {
+  return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) == cudaSuccess;
+}
+
+static bool fill_layer(UmmaLayer& U, const dp_layer& L, int box_rows) {
+  if (!encode_map(&U.mapG, L.G, L.B, L.T, L.d_out, box_rows)) return false;
+  if (!encode_map(&U.mapA, L.A, L.B, L.T, L.d_in, box_rows)) return false;
+  U.acc_w = L.acc_w;
+  U.acc_b = L.acc_b;
+  U.d_out = L.d_out;
+  U.d_in = L.d_in;
+  U.tiles_m = ceil_div(L.d_out, 128);
+  U.tiles_n = ceil_div(L.d_in, 256);
+  U.has_bias = L.has_bias;
+  U.pad = 0;
+  return true;
+}
+
+int launch_umma_sqnorms(const dp_layer* layers, const int* idx, int n, const int* use_gram, float* partial,
+                        int partial_stride, int partial_base, int* status, cudaStream_t s) {
+  if (n <= 0) return DP_OK;
+  const int B = layers[idx[0]].B, T = layers[idx[0]].T;
+  static bool attr_ok = ensure_smem(k_gram_sqnorm, G_SMEM) && ensure_smem(k_tile<false>, T_SMEM);
+  if (!attr_ok) return DP_ERR_CUDA;
+  // Partial slots are assigned in the caller's layer order, whichever kernel fills them.
+  std::vector<int> base(n);
+  int pos = partial_base;
+  for (int k = 0; k < n; ++k) {
+    base[k] = pos;
+    pos += 4 * (use_gram[k] ? gram_pairs(T) : tile_count(layers[idx[k]]));
+  }
+  for (int pass = 0; pass < 2; ++pass) {             // pass 0: Gram layers, pass 1: materialised tiles
+    const bool gram = pass == 0;
+    int k = 0;
+    while (k < n) {
+      UmmaParams P;
+      P.n_layers = 0;
+      long long items = 0;
+      for (; k < n && P.n_layers < kMaxLayers; ++k) {
+        if ((use_gram[k] != 0) != gram) continue;
+        const dp_layer& L = layers[idx[k]];
+        const long long add = (long long)B * (gram ? gram_pairs(T) : tile_count(L));
+        if (items + add > 0x7fffffffll) break;
+        UmmaLayer& U = P.L[P.n_layers];
+        if (!fill_layer(U, L, gram ? (T < 128 ? T : 128) : (T < 64 ? T : 64))) return DP_ERR_CUDA;
+        U.item_start = (int)items;
+        U.partial_base = base[k];
+        items += add;
+        ++P.n_layers;
+      }
+      if (P.n_layers == 0) continue;
+      P.total_items = (int)items;
+      P.B = B;
+      P.T = T;
+      P.box_rows = gram ? (T < 128 ? T : 128) : (T < 64 ? T : 64);
+      P.splits = 1;
+      P.partial_stride = partial_stride;
+      P.pad = 0;
+      P.clip = nullptr;
+      P.partial = partial;
+      P.status = status;
+      const int grid = P.total_items < sm_count() ? P.total_items : sm_count();
+      if (gram) k_gram_sqnorm<<<grid, G_THREADS, G_SMEM, s>>>(P);
+      else      k_tile<false><<<grid, 192, T_SMEM, s>>>(P);
+      if (counted(1) != cudaSuccess) return DP_ERR_CUDA;
+    }
+  }
+  return DP_OK;
+}
+
+int launch_umma_accumulate(const dp_layer* layers, const int* idx, int n, const float* clip, int* status,
+                           cudaStream_t s) {
+  if (n <= 0) return DP_OK;
+  const int B = layers[idx[0]].B, T = layers[idx[0]].T;
+  static bool attr_ok = ensure_smem(k_tile<true>, T_SMEM);
+  if (!attr_ok) return DP_ERR_CUDA;
+  const int sms = sm_count();
+  for (int k0 = 0; k0 < n; k0 += kMaxLayers) {
+    const int nl = (n - k0) < kMaxLayers ? (n - k0) : kMaxLayers;
+    long long tiles = 0;
+    for (int k = 0; k < nl; ++k) tiles += tile_count(layers[idx[k0 + k]]);
+    // Split the example range when the tiles alone cannot fill the machine: pick the smallest split count
+    // (<= 8, <= B) whose last wave is at least 85% full.  Split tiles combine through fp32 atomics.
+    int splits = 1;
+    if (tiles < 4ll * sms) {
+      double best = 0.0;
+      for (int sp = 1; sp <= 8 && sp <= B; ++sp) {
+        const long long it = tiles * sp;
+        const double eff = (double)it / (double)((it + sms - 1) / sms * sms);
+        if (eff > best + 1e-9) { best = eff; splits = sp; }
+        if (eff >= 0.85) { splits = sp; break; }
+      }
+    }
+    UmmaParams P;
+    long long items = 0;
+    for (int k = 0; k < nl; ++k) {
+      const dp_layer& L = layers[idx[k0 + k]];
+      UmmaLayer& U = P.L[k];
+      if (!fill_layer(U, L, T < 64 ? T : 64)) return DP_ERR_CUDA;
+      U.item_start = (int)items;
+      U.partial_base = 0;
+      items += (long long)tile_count(L) * splits;
+    }
+    P.n_layers = nl;
+    P.total_items = (int)items;
+    P.B = B;
+    P.T = T;
+    P.box_rows = T < 64 ? T : 64;
+    P.splits = splits;
+    P.partial_stride = 0;
+    P.pad = 0;
+    P.clip = clip;
+    P.partial = nullptr;
+    P.status = status;
+    const int grid = P.total_items < sms ? P.total_items : sms;
+    k_tile<true><<<grid, 320, T_SMEM, s>>>(P);
+    if (counted(1) != cudaSuccess) return DP_ERR_CUDA;
+  }
+  return DP_OK;
+}
+
+}  // namespace dpk
