@@ -188,6 +188,8 @@ def main():
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--blocks", type=int, default=24,
+                    help="encoder blocks of the stack (24 = the benchmark workload; fewer only for profiler captures)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
@@ -214,6 +216,8 @@ def main():
         dist.barrier()
 
     wl = synth.workload(WORKLOAD)
+    if args.blocks != 24:
+        wl.specs = wl.specs[:6 * args.blocks] + [wl.specs[-1]]
     data = synth.generate(wl, seed=1000 + rank, device=dev)
     step = pkg.DPStep(wl.specs, dev, wl.C, wl.sigma, wl.lr, wl.beta1, wl.beta2, wl.xi, wl.weight_decay, seed=0)
     step.theta.copy_(synth.initial_weights(step.n_flat, 0, dev))
@@ -315,7 +319,8 @@ def main():
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
                 "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
                 "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-                "config": {"workload": WORKLOAD, "B": B, "T": T, "layers": len(wl.specs), "params": n_params,
+                "config": {"workload": WORKLOAD if args.blocks == 24 else f"{WORKLOAD}[first {args.blocks} blocks only]",
+                           "B": B, "T": T, "layers": len(wl.specs), "params": n_params,
                            "microbatches_per_step": 1, "parallelism": f"dp{world}",
                            "l2": "inputs (32 GB per microbatch) far exceed L2; no flush"},
                 "phases_ms": {"norms+clip": phases[0], "accumulate_linear": phases[1],
