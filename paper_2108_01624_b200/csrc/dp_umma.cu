@@ -481,6 +481,272 @@ __global__ void __launch_bounds__(ACCUM ? 320 : 192, 1) k_tile(const __grid_cons
 }
 
 // =================================================================================================
+// Clipped-accumulate kernel: 256 (d_out) x 256 (d_in) output tiles, K = tokens, 32 tokens per stage.
+// Two 128x256x16 UMMAs (the two 128-row halves of the G tile) share each 256-wide A tile, so a stage of
+// 32 KB feeds 512 tensor-pipe cycles and a 6-stage ring covers the L2/HBM latency.  The whole 512-column
+// TMEM holds the one fp32 accumulator; at the end of a tile all eight non-producer warps drain it.
+// =================================================================================================
+constexpr int A_STAGES = 6;
+constexpr int A_BK = 32;
+constexpr int A_ATOM_BYTES = A_BK * 128;                // 32 tokens x 64 bf16 features
+constexpr int A_M_BYTES = 4 * A_ATOM_BYTES;             // G tile: 256 features of d_out
+constexpr int A_N_BYTES = 4 * A_ATOM_BYTES;             // A tile: 256 features of d_in
+constexpr int A_STAGE_BYTES = A_M_BYTES + A_N_BYTES;    // 32 KB
+constexpr int A_THREADS = 320;
+
+struct AccumCtl {
+  uint64_t full[A_STAGES], empty[A_STAGES], ready[A_STAGES], tmem_full, tmem_empty, drain;
+  uint32_t tmem_base;
+  int abort;
+  float colsum[8][256];
+};
+constexpr int A_SMEM = 1024 + A_STAGES * A_STAGE_BYTES + (int)sizeof(AccumCtl);
+
+struct AccumItem { int l, m0, n0, e0, e1, nt; };
+
+__device__ __forceinline__ AccumItem accum_decode(const UmmaParams& P, int item) {
+  AccumItem t;
+  t.l = find_layer(P, item);
+  const UmmaLayer& L = P.L[t.l];
+  const int rem = item - L.item_start, tiles = L.tiles_m * L.tiles_n;
+  const int split = rem / tiles, tile = rem - split * tiles;
+  const int mt = tile / L.tiles_n;
+  t.nt = tile - mt * L.tiles_n;
+  t.m0 = mt * 256;
+  t.n0 = t.nt * 256;
+  t.e0 = (int)((long long)split * P.B / P.splits);
+  t.e1 = (int)((long long)(split + 1) * P.B / P.splits);
+  return t;
+}
+
+// acc_w[(n0 + j) * d_out + m] += tile value; one lane owns row m (a d_out index), 32 columns per chunk.
+__device__ __forceinline__ void accum_store_chunk(const UmmaLayer& L, int m, int nb, const uint32_t (&v)[32], bool atomic) {
+  if (m >= L.d_out || nb >= L.d_in) return;
+  float* p = L.acc_w + (size_t)nb * L.d_out + m;
+  const int nv = (L.d_in - nb) < 32 ? (L.d_in - nb) : 32;
+  if (atomic) {
+#pragma unroll
+    for (int j = 0; j < 32; ++j)
+      if (j < nv) atomicAdd(p + (size_t)j * L.d_out, __uint_as_float(v[j]));
+  } else {
+    float old[32];
+#pragma unroll
+    for (int j = 0; j < 32; ++j) old[j] = (j < nv) ? p[(size_t)j * L.d_out] : 0.0f;
+#pragma unroll
+    for (int j = 0; j < 32; ++j)
+      if (j < nv) p[(size_t)j * L.d_out] = old[j] + __uint_as_float(v[j]);
+  }
+}
+
+__global__ void __launch_bounds__(A_THREADS, 1) k_accum(const __grid_constant__ UmmaParams P) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* tiles = align1024(smem_raw);
+  AccumCtl* S = reinterpret_cast<AccumCtl*>(tiles + A_STAGES * A_STAGE_BYTES);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  volatile int* abort_flag = &S->abort;
+  constexpr uint32_t IDESC = idesc_bf16_f32(128, 256, true, true);
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < A_STAGES; ++s) {
+      mbar_init(&S->full[s], 1);
+      mbar_init(&S->empty[s], 1);
+      mbar_init(&S->ready[s], 64);
+    }
+    mbar_init(&S->tmem_full, 1);
+    mbar_init(&S->tmem_empty, 8);
+    mbar_init(&S->drain, 1);
+    S->abort = 0;
+    fence_mbar_init();
+  }
+  if (P.box_rows < A_BK) {
+    for (int k = threadIdx.x; k < A_STAGES * A_STAGE_BYTES / 16; k += A_THREADS)
+      reinterpret_cast<uint4*>(tiles)[k] = make_uint4(0, 0, 0, 0);
+    fence_proxy_async_smem();
+  }
+  if (warp == 1) { tmem_alloc(&S->tmem_base, 512); tmem_relinquish(); }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = S->tmem_base;
+  const int n_tb = (P.T + A_BK - 1) / A_BK;
+  const uint32_t box_bytes = (uint32_t)P.box_rows * 128u;
+  const bool atomic = P.splits > 1;
+
+  if (warp == 0) {
+    if (lane == 0) {   // ---------------- TMA producer ----------------
+      uint32_t it = 0;
+      bool alive = true;
+      for (int item = blockIdx.x; item < P.total_items && alive; item += gridDim.x) {
+        const AccumItem t = accum_decode(P, item);
+        const UmmaLayer& L = P.L[t.l];
+        for (int e = t.e0; e < t.e1 && alive; ++e) {
+          for (int tb = 0; tb < n_tb; ++tb) {
+            const uint32_t slot = it % A_STAGES, ph = (it / A_STAGES) & 1u;
+            if (!mbar_wait(&S->empty[slot], ph ^ 1u, abort_flag, P.status)) { alive = false; break; }
+            uint8_t* st = tiles + slot * A_STAGE_BYTES;
+            mbar_arrive_expect_tx(&S->full[slot], 8u * box_bytes);
+#pragma unroll
+            for (int a = 0; a < 4; ++a)
+              tma_load_3d(st + a * A_ATOM_BYTES, &L.mapG, &S->full[slot], t.m0 + a * 64, tb * A_BK, e);
+#pragma unroll
+            for (int a = 0; a < 4; ++a)
+              tma_load_3d(st + A_M_BYTES + a * A_ATOM_BYTES, &L.mapA, &S->full[slot], t.n0 + a * 64, tb * A_BK, e);
+            ++it;
+          }
+        }
+      }
+      const uint32_t pending = it < (uint32_t)A_STAGES ? it : (uint32_t)A_STAGES;
+      for (uint32_t k = 0; k < pending; ++k) {
+        const uint32_t j = it - 1 - k;
+        mbar_wait_drain(&S->full[j % A_STAGES], (j / A_STAGES) & 1u, P.status);
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {   // ---------------- MMA issuer ----------------
+      uint32_t it = 0, tile_it = 0;
+      bool alive = true;
+      for (int item = blockIdx.x; item < P.total_items && alive; item += gridDim.x, ++tile_it) {
+        const AccumItem t = accum_decode(P, item);
+        if (!mbar_wait(&S->tmem_empty, (tile_it & 1u) ^ 1u, abort_flag, P.status)) { alive = false; break; }
+        tc_fence_after();
+        uint32_t acc = 0;
+        for (int e = t.e0; e < t.e1 && alive; ++e) {
+          for (int tb = 0; tb < n_tb; ++tb) {
+            const uint32_t slot = it % A_STAGES, ph = (it / A_STAGES) & 1u;
+            ++it;
+            if (!mbar_wait(&S->ready[slot], ph, abort_flag, P.status)) { alive = false; break; }
+            tc_fence_after();
+            const uint32_t am = smem_u32(tiles + slot * A_STAGE_BYTES), an = am + A_M_BYTES;
+#pragma unroll
+            for (int k2 = 0; k2 < 2; ++k2) {
+              const uint64_t bdesc = smem_desc_sw128(an + k2 * 2048, A_ATOM_BYTES, 1024);
+#pragma unroll
+              for (int h = 0; h < 2; ++h) {
+                umma_bf16(tmem_base + (uint32_t)h * 256u,
+                          smem_desc_sw128(am + h * 2 * A_ATOM_BYTES + k2 * 2048, A_ATOM_BYTES, 1024), bdesc, IDESC,
+                          acc | (uint32_t)k2);
+              }
+            }
+            acc = 1;
+            umma_commit(&S->empty[slot]);
+          }
+        }
+        if (alive) umma_commit(&S->tmem_full);
+      }
+      umma_commit(&S->drain);
+      mbar_wait_drain(&S->drain, 0u, P.status);
+    }
+  } else {   // ---------------- warps 2..9: scale the G tile (and bias column sums), then drain the accumulator
+    // The scaling of a stage is a chain of waits (data landed -> read -> write -> proxy fence -> signal) whose
+    // latency exceeds the 512 tensor-pipe cycles a stage feeds, so four groups of two warps work on four
+    // consecutive stages at once: group g owns the stages with index % 4 == g.
+    const uint32_t q = (uint32_t)warp & 3u;
+    const int h = warp >= 6 ? 1 : 0;                  // which 128-row half of the tile this warp drains
+    const int tt = threadIdx.x - 64;                  // 0..255
+    const uint32_t grp = (uint32_t)tt >> 6;           // 0..3
+    const int kk = (tt & 63) >> 3, jp = tt & 7;       // row & 7, physical 16-byte chunk
+    uint32_t it = 0, tile_it = 0;
+    bool alive = true;
+    for (int item = blockIdx.x; item < P.total_items; item += gridDim.x, ++tile_it) {
+      const AccumItem t = accum_decode(P, item);
+      const UmmaLayer& L = P.L[t.l];
+      const bool need_bias = L.has_bias && t.nt == 0;
+      float col[4][8];
+#pragma unroll
+      for (int a = 0; a < 4; ++a)
+#pragma unroll
+        for (int u = 0; u < 8; ++u) col[a][u] = 0.0f;
+      for (int e = t.e0; e < t.e1; ++e) {
+        const float cf = alive ? __ldg(P.clip + e) : 1.0f;
+        // c = c_hi + c_lo in bf16: x*c_hi + x*c_lo keeps the factor to ~2^-17 with two packed instructions
+        const __nv_bfloat16 chi = __float2bfloat16_rn(cf);
+        const __nv_bfloat162 chi2 = __halves2bfloat162(chi, chi);
+        const __nv_bfloat16 clo = __float2bfloat16_rn(cf - __bfloat162float(chi));
+        const __nv_bfloat162 clo2 = __halves2bfloat162(clo, clo);
+        for (int tb = 0; tb < n_tb; ++tb) {
+          const uint32_t slot = it % A_STAGES, ph = (it / A_STAGES) & 1u, mine = (it & 3u) == grp;
+          ++it;
+          if (!mine) continue;
+          if (alive && !mbar_wait(&S->full[slot], ph, abort_flag, P.status)) alive = false;
+          if (!alive) continue;
+          if (cf != 1.0f || need_bias) {
+            uint8_t* base = tiles + slot * A_STAGE_BYTES + kk * 128 + jp * 16;
+#pragma unroll
+            for (int a = 0; a < 4; ++a) {
+#pragma unroll
+              for (int i4 = 0; i4 < 4; ++i4) {        // rows kk, kk+8, kk+16, kk+24 of atom a
+                uint4* p = reinterpret_cast<uint4*>(base + a * A_ATOM_BYTES + i4 * 1024);
+                uint4 w = *p;
+                uint32_t x[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                  if (need_bias) {
+                    col[a][2 * u] = fmaf(__uint_as_float(x[u] << 16), cf, col[a][2 * u]);
+                    col[a][2 * u + 1] = fmaf(__uint_as_float(x[u] & 0xffff0000u), cf, col[a][2 * u + 1]);
+                  }
+                  const __nv_bfloat162 xv = *reinterpret_cast<const __nv_bfloat162*>(&x[u]);
+                  const __nv_bfloat162 yv = __hfma2(xv, clo2, __hmul2(xv, chi2));
+                  x[u] = *reinterpret_cast<const uint32_t*>(&yv);
+                }
+                if (cf != 1.0f) *p = make_uint4(x[0], x[1], x[2], x[3]);
+              }
+            }
+            fence_proxy_async_smem();
+          }
+          mbar_arrive(&S->ready[slot]);
+        }
+      }
+      if (need_bias) {      // uniform over the 256 threads of warps 2..9; executed even after an abort
+        const int j = jp ^ kk;                        // logical 16-byte chunk under the 128-byte swizzle
+#pragma unroll 1
+        for (uint32_t g2 = 0; g2 < 4; ++g2) {         // groups add their sums one after another: fixed order
+          if (grp == g2) {
+#pragma unroll
+            for (int a = 0; a < 4; ++a)
+#pragma unroll
+              for (int u = 0; u < 8; ++u) {
+                float* dst = &S->colsum[kk][a * 64 + j * 8 + u];
+                *dst = (g2 == 0 ? 0.0f : *dst) + col[a][u];
+              }
+          }
+          asm volatile("bar.sync 2, 256;" ::: "memory");
+        }
+        const int mcol = t.m0 + tt;
+        if (alive && mcol < L.d_out) {
+          float sacc = 0.0f;
+#pragma unroll
+          for (int r8 = 0; r8 < 8; ++r8) sacc += S->colsum[r8][tt];
+          if (atomic) atomicAdd(L.acc_b + mcol, sacc); else L.acc_b[mcol] += sacc;
+        }
+        asm volatile("bar.sync 2, 256;" ::: "memory");
+      }
+      // ---- drain the accumulator: rows [h*128 + q*32, +32) of the tile
+      if (alive) alive = __all_sync(0xffffffffu, mbar_wait(&S->tmem_full, tile_it & 1u, abort_flag, P.status));
+      if (!alive) continue;
+      tc_fence_after();
+      const int m = t.m0 + h * 128 + (int)q * 32 + lane;
+#pragma unroll 1
+      for (int ch = 0; ch < 8; ++ch) {
+        uint32_t v[32];
+        tmem_ld_32x32(tmem_base + ((q * 32u) << 16) + (uint32_t)h * 256u + (uint32_t)ch * 32u, v);
+        tmem_ld_wait();
+        accum_store_chunk(L, m, t.n0 + ch * 32, v, atomic);
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&S->tmem_empty);
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    __syncwarp();
+    tc_fence_after();
+    tmem_dealloc(tmem_base, 512);
+  }
+}
+
+// =================================================================================================
 // Host side: tensor maps, work lists, launches
 // =================================================================================================
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -525,6 +791,7 @@ bool umma_accumulates_bias() { return true; }
 
 static int gram_pairs(int T) { const int nb = (T + 127) / 128; return nb * (nb + 1) / 2; }
 static int tile_count(const dp_layer& L) { return ceil_div(L.d_out, 128) * ceil_div(L.d_in, 256); }
+static int accum_tile_count(const dp_layer& L) { return ceil_div(L.d_out, 256) * ceil_div(L.d_in, 256); }
 
 size_t umma_sqnorm_partials_per_example(const dp_layer* layers, const int* idx, int n, const int* use_gram) {
   size_t c = 0;
@@ -618,13 +885,13 @@ int launch_umma_accumulate(const dp_layer* layers, const int* idx, int n, const 
                            cudaStream_t s) {
   if (n <= 0) return DP_OK;
   const int B = layers[idx[0]].B, T = layers[idx[0]].T;
-  static bool attr_ok = ensure_smem(k_tile<true>, T_SMEM);
+  static bool attr_ok = ensure_smem(k_accum, A_SMEM);
   if (!attr_ok) return DP_ERR_CUDA;
   const int sms = sm_count();
   for (int k0 = 0; k0 < n; k0 += kMaxLayers) {
     const int nl = (n - k0) < kMaxLayers ? (n - k0) : kMaxLayers;
     long long tiles = 0;
-    for (int k = 0; k < nl; ++k) tiles += tile_count(layers[idx[k0 + k]]);
+    for (int k = 0; k < nl; ++k) tiles += accum_tile_count(layers[idx[k0 + k]]);
     // Split the example range when the tiles alone cannot fill the machine: pick the smallest split count
     // (<= 8, <= B) whose last wave is at least 85% full.  Split tiles combine through fp32 atomics.
     int splits = 1;
@@ -642,16 +909,17 @@ int launch_umma_accumulate(const dp_layer* layers, const int* idx, int n, const 
     for (int k = 0; k < nl; ++k) {
       const dp_layer& L = layers[idx[k0 + k]];
       UmmaLayer& U = P.L[k];
-      if (!fill_layer(U, L, T < 64 ? T : 64)) return DP_ERR_CUDA;
+      if (!fill_layer(U, L, T < A_BK ? T : A_BK)) return DP_ERR_CUDA;
+      U.tiles_m = ceil_div(L.d_out, 256);
       U.item_start = (int)items;
       U.partial_base = 0;
-      items += (long long)tile_count(L) * splits;
+      items += (long long)accum_tile_count(L) * splits;
     }
     P.n_layers = nl;
     P.total_items = (int)items;
     P.B = B;
     P.T = T;
-    P.box_rows = T < 64 ? T : 64;
+    P.box_rows = T < A_BK ? T : A_BK;
     P.splits = splits;
     P.partial_stride = 0;
     P.pad = 0;
@@ -659,7 +927,7 @@ int launch_umma_accumulate(const dp_layer* layers, const int* idx, int n, const 
     P.partial = nullptr;
     P.status = status;
     const int grid = P.total_items < sms ? P.total_items : sms;
-    k_tile<true><<<grid, 320, T_SMEM, s>>>(P);
+    k_accum<<<grid, A_THREADS, A_SMEM, s>>>(P);
     if (counted(1) != cudaSuccess) return DP_ERR_CUDA;
   }
   return DP_OK;
