@@ -66,25 +66,31 @@ static bool use_gram(const dp_layer& L) {
   return (long long)L.T * (L.d_in + L.d_out) <= (long long)L.d_in * L.d_out;
 }
 
-// Workspace layout: [column-sum scratch | partial sums of the tensor-core norm kernels].
+// Workspace layout: [per-example column sums of every LayerNorm / bias task | partial sums of the tensor-core
+// norm kernels].  The two layer-list calls plan the same layout, so one workspace serves both.
 struct WsPlan {
-  size_t colsum_bytes = 0;     // max over layers of B*2d (LayerNorm) or B*d_out (linear bias) floats
+  size_t colsum_bytes = 0;
   size_t partial_bytes = 0;    // B * partials_per_example floats
   int partials_per_example = 0;
   std::vector<int> umma_idx;   // layers handled by the tensor-core kernels
   std::vector<int> umma_gram;  // 1: Gram path, 0: materialised tiles
+  std::vector<size_t> col_off; // per layer: byte offset of its column-sum block (or SIZE_MAX if it has none)
   size_t total() const { return align_up(colsum_bytes, 256) + align_up(partial_bytes, 256); }
 };
 
 static WsPlan plan_workspace(const dp_layer* layers, int n_layers) {
   WsPlan p;
   const size_t B = layers[0].B;
+  p.col_off.assign(n_layers, (size_t)-1);
   for (int l = 0; l < n_layers; ++l) {
     const dp_layer& L = layers[l];
     size_t need = 0;
     if (L.kind == DP_LAYERNORM) need = B * 2 * (size_t)L.d_out * sizeof(float);
     if (L.kind == DP_LINEAR && L.has_bias) need = B * (size_t)L.d_out * sizeof(float);
-    if (need > p.colsum_bytes) p.colsum_bytes = need;
+    if (need) {
+      p.col_off[l] = p.colsum_bytes;
+      p.colsum_bytes += align_up(need, 256);
+    }
     if (L.kind == DP_LINEAR && umma_supported(L)) {
       p.umma_idx.push_back(l);
       p.umma_gram.push_back(use_gram(L) ? 1 : 0);
@@ -128,7 +134,6 @@ int dp_per_example_sqnorms(const dp_layer* layers, int n_layers, float* sqnorm, 
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
   int* status = status_ptr();
   if (!status) return DP_ERR_CUDA;
-  float* colsum = static_cast<float*>(workspace);
   float* partial = reinterpret_cast<float*>(static_cast<char*>(workspace) + align_up(plan.colsum_bytes, 256));
   const int B = layers[0].B;
   if (!accumulate_into) DP_CUDA(launch_fill_zero(sqnorm, B, s));
@@ -139,27 +144,32 @@ int dp_per_example_sqnorms(const dp_layer* layers, int n_layers, float* sqnorm, 
     if (rc != DP_OK) return rc;
     DP_CUDA(launch_reduce_partials(partial, B, plan.partials_per_example, sqnorm, s));
   }
+  // Bandwidth-bound layers: LayerNorm column sums (and the bias part of materialised-tile layers) in one
+  // batched launch, then one reduction; generic linear layers and embeddings one launch each.
+  std::vector<ColTaskHost> tasks;
   size_t u = 0;
   for (int l = 0; l < n_layers; ++l) {
     const dp_layer& L = layers[l];
+    float* out = plan.col_off[l] == (size_t)-1 ? nullptr
+                                                : reinterpret_cast<float*>(static_cast<char*>(workspace) + plan.col_off[l]);
     if (u < plan.umma_idx.size() && plan.umma_idx[u] == l) {
       // The materialised-tile kernel covers the weight gradient only; the bias part |sum_t G_i[t,:]|^2 is a
-      // bandwidth-bound column sum (the Gram kernel has it built in as the +1 on the token Gram of A).
-      if (!plan.umma_gram[u] && L.has_bias) {
-        DP_CUDA(launch_bias_colsums(L, colsum, s));
-        DP_CUDA(launch_rows_sqsum(colsum, B, L.d_out, sqnorm, s));
-      }
+      // column sum (the Gram kernel has it built in as the +1 on the token Gram of A).
+      if (!plan.umma_gram[u] && L.has_bias) tasks.push_back({&L, false, out});
       ++u;
       continue;
     }
     if (L.kind == DP_LINEAR) {
       DP_CUDA(launch_linear_sqnorm_generic(L, use_gram(L), sqnorm, s));
     } else if (L.kind == DP_LAYERNORM) {
-      DP_CUDA(launch_layernorm_colsums(L, colsum, s));
-      DP_CUDA(launch_layernorm_sqnorm(L, colsum, sqnorm, s));
+      tasks.push_back({&L, true, out});
     } else {
       DP_CUDA(launch_embedding_sqnorm(L, sqnorm, status, s));
     }
+  }
+  if (!tasks.empty()) {
+    DP_CUDA(launch_colsums_batched(tasks.data(), (int)tasks.size(), s));
+    DP_CUDA(launch_rows_sqsum_batched(tasks.data(), (int)tasks.size(), sqnorm, s));
   }
   return DP_OK;
 }
@@ -183,28 +193,30 @@ int dp_clipped_accumulate(const dp_layer* layers, int n_layers, const float* cli
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
   int* status = status_ptr();
   if (!status) return DP_ERR_CUDA;
-  float* colsum = static_cast<float*>(workspace);
   if (!plan.umma_idx.empty()) {
     rc = launch_umma_accumulate(layers, plan.umma_idx.data(), (int)plan.umma_idx.size(), clip, status, s);
     if (rc != DP_OK) return rc;
   }
+  std::vector<ColTaskHost> tasks;
   size_t u = 0;
   for (int l = 0; l < n_layers; ++l) {
     const dp_layer& L = layers[l];
+    float* out = plan.col_off[l] == (size_t)-1 ? nullptr
+                                                : reinterpret_cast<float*>(static_cast<char*>(workspace) + plan.col_off[l]);
     const bool on_umma = u < plan.umma_idx.size() && plan.umma_idx[u] == l;
     if (on_umma) ++u;
     if (L.kind == DP_LINEAR) {
       if (!on_umma) DP_CUDA(launch_linear_accum_generic(L, clip, s));
-      if (L.has_bias && !(on_umma && umma_accumulates_bias())) {
-        DP_CUDA(launch_bias_colsums(L, colsum, s));
-        DP_CUDA(launch_bias_reduce(L, colsum, clip, s));
-      }
+      if (L.has_bias && !(on_umma && umma_accumulates_bias())) tasks.push_back({&L, false, out});
     } else if (L.kind == DP_LAYERNORM) {
-      DP_CUDA(launch_layernorm_colsums(L, colsum, s));
-      DP_CUDA(launch_layernorm_accum(L, colsum, clip, s));
+      tasks.push_back({&L, true, out});
     } else {
       DP_CUDA(launch_embedding_accum(L, clip, status, s));
     }
+  }
+  if (!tasks.empty()) {
+    DP_CUDA(launch_colsums_batched(tasks.data(), (int)tasks.size(), s));
+    DP_CUDA(launch_weighted_rows_sum_batched(tasks.data(), (int)tasks.size(), clip, s));
   }
   return DP_OK;
 }

@@ -223,8 +223,8 @@ template <typename T> struct VecLoad<T, 1> {
 };
 
 template <typename T, int VEC, bool WITH_X>
-__global__ void __launch_bounds__(512)
-k_colsums(const T* __restrict__ X, const T* __restrict__ G, int Tn, int d, float* __restrict__ out) {
+__device__ __forceinline__ void
+k_colsums_body(const T* __restrict__ X, const T* __restrict__ G, int Tn, int d, float* __restrict__ out) {
   __shared__ float sh[3][128][2 * VEC];
   const int i = blockIdx.x;
   const int lane = threadIdx.x & 127, tg = threadIdx.x >> 7;
@@ -267,71 +267,139 @@ k_colsums(const T* __restrict__ X, const T* __restrict__ G, int Tn, int d, float
   }
 }
 
-template <typename T, int VEC>
-static cudaError_t colsums_launch(const void* X, const void* G, int B, int Tn, int d, bool with_x, float* out,
-                                  cudaStream_t s) {
-  if (with_x) k_colsums<T, VEC, true><<<B, 512, 0, s>>>(static_cast<const T*>(X), static_cast<const T*>(G), Tn, d, out);
-  else        k_colsums<T, VEC, false><<<B, 512, 0, s>>>(nullptr, static_cast<const T*>(G), Tn, d, out);
-  return counted(1);
+// ---- batched over layers: one launch covers every LayerNorm (or bias) task of a call ------------------------
+constexpr int kMaxColTasks = 64;
+struct ColTask {
+  const void* X;     // normalised input (WITH_X) or nullptr
+  const void* G;
+  float* out;        // [B][width] per-example column sums
+  float* acc0;       // accumulate target of columns [0, d)
+  float* acc1;       // accumulate target of columns [d, 2d) (WITH_X only)
+  int d, width;
+};
+struct ColBatch {
+  ColTask t[kMaxColTasks];
+  int n, B, T, pad;
+};
+
+template <typename T, int VEC, bool WITH_X>
+__global__ void __launch_bounds__(512) k_colsums_b(const __grid_constant__ ColBatch P) {
+  const ColTask& t = P.t[blockIdx.y];
+  k_colsums_body<T, VEC, WITH_X>(static_cast<const T*>(t.X), static_cast<const T*>(t.G), P.T, t.d, t.out);
 }
 
-static cudaError_t colsums_dispatch(const dp_layer& L, bool with_x, float* out, cudaStream_t s) {
+// sqnorm[i] += sum over tasks and columns of out[i][j]^2 (fixed order).
+__global__ void __launch_bounds__(256) k_rows_sqsum_b(const __grid_constant__ ColBatch P, float* __restrict__ sqnorm) {
+  __shared__ float red[32];
+  float tot = 0.0f;
+  for (int k = 0; k < P.n; ++k) {
+    const float* w = P.t[k].out + (size_t)blockIdx.x * P.t[k].width;
+    for (int j = threadIdx.x; j < P.t[k].width; j += 256) tot = fmaf(w[j], w[j], tot);
+  }
+  tot = block_sum(tot, red);
+  if (threadIdx.x == 0) sqnorm[blockIdx.x] += tot;
+}
+
+// acc[j] += sum_i clip[i] * out[i][j] for task blockIdx.y; 64 columns x 4 example groups per CTA.
+__global__ void __launch_bounds__(256)
+k_weighted_rows_sum_b(const __grid_constant__ ColBatch P, const float* __restrict__ clip) {
+  __shared__ float sh[4][64];
+  const ColTask& t = P.t[blockIdx.y];
+  const int c = threadIdx.x & 63, g = threadIdx.x >> 6;
+  const int j = blockIdx.x * 64 + c;
+  float a = 0.0f;
+  if (j < t.width)
+    for (int i = g; i < P.B; i += 4) a = fmaf(__ldg(clip + i), t.out[(size_t)i * t.width + j], a);
+  sh[g][c] = a;
+  __syncthreads();
+  if (g == 0 && j < t.width) {
+    const float v = (sh[0][c] + sh[1][c]) + (sh[2][c] + sh[3][c]);
+    if (j < t.d) t.acc0[j] += v; else t.acc1[j - t.d] += v;
+  }
+}
+
+// variant key of a task: dtype, vector width, with_x
+static int col_variant(const dp_layer& L, bool with_x) {
   const int d = L.d_out;
   const bool al = ((reinterpret_cast<uintptr_t>(L.G) | (with_x ? reinterpret_cast<uintptr_t>(L.A) : 0)) & 15u) == 0;
-  if (L.dtype == DP_F32) {
-    if (al && d % 4 == 0) return colsums_launch<float, 4>(L.A, L.G, L.B, L.T, d, with_x, out, s);
-    return colsums_launch<float, 1>(L.A, L.G, L.B, L.T, d, with_x, out, s);
+  int v;
+  if (L.dtype == DP_F32) v = (al && d % 4 == 0) ? 0 : 1; else v = (al && d % 8 == 0) ? 2 : 3;
+  return v * 2 + (with_x ? 1 : 0);
+}
+
+template <typename T, int VEC>
+static void colsums_b_launch(const ColBatch& P, bool with_x, cudaStream_t s) {
+  dim3 grid(P.B, P.n);
+  if (with_x) k_colsums_b<T, VEC, true><<<grid, 512, 0, s>>>(P); else k_colsums_b<T, VEC, false><<<grid, 512, 0, s>>>(P);
+}
+
+static ColTask make_task(const ColTaskHost& h) {
+  const dp_layer& L = *h.L;
+  ColTask t;
+  t.X = h.with_x ? L.A : nullptr;
+  t.G = L.G;
+  t.out = h.out;
+  t.d = L.d_out;
+  t.width = (h.with_x ? 2 : 1) * L.d_out;
+  t.acc0 = h.with_x ? L.acc_w : L.acc_b;
+  t.acc1 = h.with_x ? L.acc_b : nullptr;
+  return t;
+}
+
+cudaError_t launch_colsums_batched(const ColTaskHost* tasks, int n, cudaStream_t s) {
+  // group by kernel variant, at most kMaxColTasks per launch
+  for (int variant = 0; variant < 8; ++variant) {
+    ColBatch P;
+    P.n = 0;
+    for (int k = 0; k <= n; ++k) {
+      const bool take = k < n && col_variant(*tasks[k].L, tasks[k].with_x) == variant;
+      if (take) {
+        P.t[P.n++] = make_task(tasks[k]);
+        P.B = tasks[k].L->B;
+        P.T = tasks[k].L->T;
+      }
+      if (P.n == kMaxColTasks || (k == n && P.n > 0)) {
+        const bool wx = variant & 1;
+        switch (variant >> 1) {
+          case 0: colsums_b_launch<float, 4>(P, wx, s); break;
+          case 1: colsums_b_launch<float, 1>(P, wx, s); break;
+          case 2: colsums_b_launch<__nv_bfloat16, 8>(P, wx, s); break;
+          default: colsums_b_launch<__nv_bfloat16, 1>(P, wx, s); break;
+        }
+        if (counted(1) != cudaSuccess) return cudaGetLastError();
+        P.n = 0;
+      }
+    }
   }
-  if (al && d % 8 == 0) return colsums_launch<__nv_bfloat16, 8>(L.A, L.G, L.B, L.T, d, with_x, out, s);
-  return colsums_launch<__nv_bfloat16, 1>(L.A, L.G, L.B, L.T, d, with_x, out, s);
+  return cudaSuccess;
 }
 
-cudaError_t launch_layernorm_colsums(const dp_layer& L, float* ws, cudaStream_t s) {
-  return colsums_dispatch(L, true, ws, s);
+template <typename F>
+static cudaError_t for_each_batch(const ColTaskHost* tasks, int n, F launch) {
+  for (int k0 = 0; k0 < n; k0 += kMaxColTasks) {
+    ColBatch P;
+    P.n = (n - k0) < kMaxColTasks ? (n - k0) : kMaxColTasks;
+    for (int k = 0; k < P.n; ++k) P.t[k] = make_task(tasks[k0 + k]);
+    P.B = tasks[k0].L->B;
+    P.T = tasks[k0].L->T;
+    launch(P);
+    const cudaError_t e = counted(1);
+    if (e != cudaSuccess) return e;
+  }
+  return cudaSuccess;
 }
 
-// sqnorm[i] += sum_j ws[i][j]^2, j < width.
-__global__ void __launch_bounds__(256) k_rows_sqsum(const float* __restrict__ ws, int width, float* __restrict__ sqnorm) {
-  __shared__ float red[32];
-  const float* w = ws + (size_t)blockIdx.x * width;
-  float t = 0.0f;
-  for (int j = threadIdx.x; j < width; j += 256) t = fmaf(w[j], w[j], t);
-  t = block_sum(t, red);
-  if (threadIdx.x == 0) sqnorm[blockIdx.x] += t;
-}
-cudaError_t launch_rows_sqsum(const float* ws, int B, int width, float* sqnorm, cudaStream_t s) {
-  k_rows_sqsum<<<B, 256, 0, s>>>(ws, width, sqnorm);
-  return counted(1);
-}
-cudaError_t launch_layernorm_sqnorm(const dp_layer& L, const float* ws, float* sqnorm, cudaStream_t s) {
-  return launch_rows_sqsum(ws, L.B, 2 * L.d_out, sqnorm, s);
+cudaError_t launch_rows_sqsum_batched(const ColTaskHost* tasks, int n, float* sqnorm, cudaStream_t s) {
+  return for_each_batch(tasks, n, [&](const ColBatch& P) { k_rows_sqsum_b<<<P.B, 256, 0, s>>>(P, sqnorm); });
 }
 
-// dst[j] += sum_i clip[i] * ws[i][off + j], j < d; rows of ws are `width` apart.  64 columns x 4 example groups.
-__global__ void __launch_bounds__(256)
-k_weighted_rows_sum(const float* __restrict__ ws, int B, int width, int off, int d, const float* __restrict__ clip,
-                    float* __restrict__ dst) {
-  __shared__ float sh[4][64];
-  const int j = blockIdx.x * 64 + (threadIdx.x & 63), g = threadIdx.x >> 6;
-  float t = 0.0f;
-  if (j < d)
-    for (int i = g; i < B; i += 4) t = fmaf(__ldg(clip + i), ws[(size_t)i * width + off + j], t);
-  sh[g][threadIdx.x & 63] = t;
-  __syncthreads();
-  if (g == 0 && j < d) dst[j] += (sh[0][threadIdx.x] + sh[1][threadIdx.x]) + (sh[2][threadIdx.x] + sh[3][threadIdx.x]);
-}
-cudaError_t launch_layernorm_accum(const dp_layer& L, const float* ws, const float* clip, cudaStream_t s) {
-  const int d = L.d_out;
-  k_weighted_rows_sum<<<ceil_div(d, 64), 256, 0, s>>>(ws, L.B, 2 * d, 0, d, clip, L.acc_w);
-  k_weighted_rows_sum<<<ceil_div(d, 64), 256, 0, s>>>(ws, L.B, 2 * d, d, d, clip, L.acc_b);
-  return counted(2);
-}
-// Linear bias: ws[B][d_out] scratch is supplied through L.acc_w == nullptr convention is NOT used;
-// the caller passes the scratch explicitly.
-cudaError_t launch_bias_colsums(const dp_layer& L, float* ws, cudaStream_t s) { return colsums_dispatch(L, false, ws, s); }
-cudaError_t launch_bias_reduce(const dp_layer& L, const float* ws, const float* clip, cudaStream_t s) {
-  k_weighted_rows_sum<<<ceil_div(L.d_out, 64), 256, 0, s>>>(ws, L.B, L.d_out, 0, L.d_out, clip, L.acc_b);
-  return counted(1);
+cudaError_t launch_weighted_rows_sum_batched(const ColTaskHost* tasks, int n, const float* clip, cudaStream_t s) {
+  return for_each_batch(tasks, n, [&](const ColBatch& P) {
+    int wmax = 0;
+    for (int k = 0; k < P.n; ++k) wmax = P.t[k].width > wmax ? P.t[k].width : wmax;
+    dim3 grid(ceil_div(wmax, 64), P.n);
+    k_weighted_rows_sum_b<<<grid, 256, 0, s>>>(P, clip);
+  });
 }
 
 __global__ void k_fill_zero(float* __restrict__ p, long long n) {

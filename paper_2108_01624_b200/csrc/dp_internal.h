@@ -46,19 +46,17 @@ cudaError_t launch_equality_mask(const int32_t* ids, int B, int T, uint8_t* mask
 // Per-example squared norms; each adds into sqnorm[i] (one writer per example, launches are ordered).
 cudaError_t launch_linear_sqnorm_generic(const dp_layer& L, bool gram, float* sqnorm, cudaStream_t s);
 cudaError_t launch_linear_accum_generic(const dp_layer& L, const float* clip, cudaStream_t s);
-// LayerNorm: per-example column sums into ws[B][2d] (gain part then bias part), then either the norm
-// or the clip-weighted reduction over examples.
-cudaError_t launch_layernorm_colsums(const dp_layer& L, float* ws, cudaStream_t s);
-// sqnorm[i] += sum_j ws[i][j]^2, j < width (rows of ws are `width` apart).
-cudaError_t launch_rows_sqsum(const float* ws, int B, int width, float* sqnorm, cudaStream_t s);
-cudaError_t launch_layernorm_sqnorm(const dp_layer& L, const float* ws, float* sqnorm, cudaStream_t s);
-cudaError_t launch_layernorm_accum(const dp_layer& L, const float* ws, const float* clip, cudaStream_t s);
+// Column-sum tasks, batched over layers.  A task yields out[B][width]: for a LayerNorm (with_x) the gain part
+// sum_t x*G then the bias part sum_t G (width 2d); for a linear bias (no x) sum_t G (width d_out).
+struct ColTaskHost { const dp_layer* L; bool with_x; float* out; };
+cudaError_t launch_colsums_batched(const ColTaskHost* tasks, int n, cudaStream_t s);
+// sqnorm[i] += sum over tasks, columns of out[i][j]^2.
+cudaError_t launch_rows_sqsum_batched(const ColTaskHost* tasks, int n, float* sqnorm, cudaStream_t s);
+// LayerNorm: acc_w += sum_i clip_i * gain part, acc_b += ... bias part.  Linear bias: acc_b += sum_i clip_i * out[i].
+cudaError_t launch_weighted_rows_sum_batched(const ColTaskHost* tasks, int n, const float* clip, cudaStream_t s);
 // Embedding by grouping equal ids inside an example.
 cudaError_t launch_embedding_sqnorm(const dp_layer& L, float* sqnorm, int* status, cudaStream_t s);
 cudaError_t launch_embedding_accum(const dp_layer& L, const float* clip, int* status, cudaStream_t s);
-// Linear bias: per-example column sums of G into ws[B][d_out], then acc_b += sum_i clip_i * ws[i].
-cudaError_t launch_bias_colsums(const dp_layer& L, float* ws, cudaStream_t s);
-cudaError_t launch_bias_reduce(const dp_layer& L, const float* ws, const float* clip, cudaStream_t s);
 cudaError_t launch_fill_zero(float* p, long long n, cudaStream_t s);
 // sqnorm[i] (+)= sum of partial[i * stride + j], j < count, in a fixed order.
 cudaError_t launch_reduce_partials(const float* partial, int B, int count, float* sqnorm, cudaStream_t s);

@@ -485,6 +485,9 @@ __global__ void __launch_bounds__(ACCUM ? 320 : 192, 1) k_tile(const __grid_cons
 // Two 128x256x16 UMMAs (the two 128-row halves of the G tile) share each 256-wide A tile, so a stage of
 // 32 KB feeds 512 tensor-pipe cycles and a 6-stage ring covers the L2/HBM latency.  The whole 512-column
 // TMEM holds the one fp32 accumulator; at the end of a tile all eight non-producer warps drain it.
+// What bounds the kernel is the shared-memory data pipe (one 128-byte wavefront per cycle, shared by TMA
+// writes, UMMA operand reads and ld/st.shared): per stage 384 operand + 256 TMA wavefronts, plus up to 256
+// for scaling the G tile in place (skipped for examples whose clip factor is 1).
 // =================================================================================================
 constexpr int A_STAGES = 6;
 constexpr int A_BK = 32;
@@ -550,7 +553,7 @@ __global__ void __launch_bounds__(A_THREADS, 1) k_accum(const __grid_constant__ 
     for (int s = 0; s < A_STAGES; ++s) {
       mbar_init(&S->full[s], 1);
       mbar_init(&S->empty[s], 1);
-      mbar_init(&S->ready[s], 64);
+      mbar_init(&S->ready[s], 256);
     }
     mbar_init(&S->tmem_full, 1);
     mbar_init(&S->tmem_empty, 8);
@@ -637,25 +640,19 @@ __global__ void __launch_bounds__(A_THREADS, 1) k_accum(const __grid_constant__ 
       mbar_wait_drain(&S->drain, 0u, P.status);
     }
   } else {   // ---------------- warps 2..9: scale the G tile (and bias column sums), then drain the accumulator
-    // The scaling of a stage is a chain of waits (data landed -> read -> write -> proxy fence -> signal) whose
-    // latency exceeds the 512 tensor-pipe cycles a stage feeds, so four groups of two warps work on four
-    // consecutive stages at once: group g owns the stages with index % 4 == g.
     const uint32_t q = (uint32_t)warp & 3u;
     const int h = warp >= 6 ? 1 : 0;                  // which 128-row half of the tile this warp drains
     const int tt = threadIdx.x - 64;                  // 0..255
-    const uint32_t grp = (uint32_t)tt >> 6;           // 0..3
-    const int kk = (tt & 63) >> 3, jp = tt & 7;       // row & 7, physical 16-byte chunk
+    const int ta = tt >> 6, kk = (tt & 63) >> 3, jp = tt & 7;   // atom, row & 7, physical 16-byte chunk
     uint32_t it = 0, tile_it = 0;
     bool alive = true;
     for (int item = blockIdx.x; item < P.total_items; item += gridDim.x, ++tile_it) {
       const AccumItem t = accum_decode(P, item);
       const UmmaLayer& L = P.L[t.l];
       const bool need_bias = L.has_bias && t.nt == 0;
-      float col[4][8];
+      float col[8];
 #pragma unroll
-      for (int a = 0; a < 4; ++a)
-#pragma unroll
-        for (int u = 0; u < 8; ++u) col[a][u] = 0.0f;
+      for (int u = 0; u < 8; ++u) col[u] = 0.0f;
       for (int e = t.e0; e < t.e1; ++e) {
         const float cf = alive ? __ldg(P.clip + e) : 1.0f;
         // c = c_hi + c_lo in bf16: x*c_hi + x*c_lo keeps the factor to ~2^-17 with two packed instructions
@@ -664,32 +661,28 @@ __global__ void __launch_bounds__(A_THREADS, 1) k_accum(const __grid_constant__ 
         const __nv_bfloat16 clo = __float2bfloat16_rn(cf - __bfloat162float(chi));
         const __nv_bfloat162 clo2 = __halves2bfloat162(clo, clo);
         for (int tb = 0; tb < n_tb; ++tb) {
-          const uint32_t slot = it % A_STAGES, ph = (it / A_STAGES) & 1u, mine = (it & 3u) == grp;
+          const uint32_t slot = it % A_STAGES, ph = (it / A_STAGES) & 1u;
           ++it;
-          if (!mine) continue;
           if (alive && !mbar_wait(&S->full[slot], ph, abort_flag, P.status)) alive = false;
           if (!alive) continue;
           if (cf != 1.0f || need_bias) {
-            uint8_t* base = tiles + slot * A_STAGE_BYTES + kk * 128 + jp * 16;
+            uint8_t* base = tiles + slot * A_STAGE_BYTES + ta * A_ATOM_BYTES + kk * 128 + jp * 16;
 #pragma unroll
-            for (int a = 0; a < 4; ++a) {
+            for (int i4 = 0; i4 < 4; ++i4) {          // rows kk, kk+8, kk+16, kk+24 of atom ta
+              uint4* p = reinterpret_cast<uint4*>(base + i4 * 1024);
+              uint4 w = *p;
+              uint32_t x[4] = {w.x, w.y, w.z, w.w};
 #pragma unroll
-              for (int i4 = 0; i4 < 4; ++i4) {        // rows kk, kk+8, kk+16, kk+24 of atom a
-                uint4* p = reinterpret_cast<uint4*>(base + a * A_ATOM_BYTES + i4 * 1024);
-                uint4 w = *p;
-                uint32_t x[4] = {w.x, w.y, w.z, w.w};
-#pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                  if (need_bias) {
-                    col[a][2 * u] = fmaf(__uint_as_float(x[u] << 16), cf, col[a][2 * u]);
-                    col[a][2 * u + 1] = fmaf(__uint_as_float(x[u] & 0xffff0000u), cf, col[a][2 * u + 1]);
-                  }
-                  const __nv_bfloat162 xv = *reinterpret_cast<const __nv_bfloat162*>(&x[u]);
-                  const __nv_bfloat162 yv = __hfma2(xv, clo2, __hmul2(xv, chi2));
-                  x[u] = *reinterpret_cast<const uint32_t*>(&yv);
+              for (int u = 0; u < 4; ++u) {
+                if (need_bias) {
+                  col[2 * u] = fmaf(__uint_as_float(x[u] << 16), cf, col[2 * u]);
+                  col[2 * u + 1] = fmaf(__uint_as_float(x[u] & 0xffff0000u), cf, col[2 * u + 1]);
                 }
-                if (cf != 1.0f) *p = make_uint4(x[0], x[1], x[2], x[3]);
+                const __nv_bfloat162 xv = *reinterpret_cast<const __nv_bfloat162*>(&x[u]);
+                const __nv_bfloat162 yv = __hfma2(xv, clo2, __hmul2(xv, chi2));
+                x[u] = *reinterpret_cast<const uint32_t*>(&yv);
               }
+              if (cf != 1.0f) *p = make_uint4(x[0], x[1], x[2], x[3]);
             }
             fence_proxy_async_smem();
           }
@@ -698,19 +691,9 @@ __global__ void __launch_bounds__(A_THREADS, 1) k_accum(const __grid_constant__ 
       }
       if (need_bias) {      // uniform over the 256 threads of warps 2..9; executed even after an abort
         const int j = jp ^ kk;                        // logical 16-byte chunk under the 128-byte swizzle
-#pragma unroll 1
-        for (uint32_t g2 = 0; g2 < 4; ++g2) {         // groups add their sums one after another: fixed order
-          if (grp == g2) {
 #pragma unroll
-            for (int a = 0; a < 4; ++a)
-#pragma unroll
-              for (int u = 0; u < 8; ++u) {
-                float* dst = &S->colsum[kk][a * 64 + j * 8 + u];
-                *dst = (g2 == 0 ? 0.0f : *dst) + col[a][u];
-              }
-          }
-          asm volatile("bar.sync 2, 256;" ::: "memory");
-        }
+        for (int u = 0; u < 8; ++u) S->colsum[kk][ta * 64 + j * 8 + u] = col[u];
+        asm volatile("bar.sync 2, 256;" ::: "memory");
         const int mcol = t.m0 + tt;
         if (alive && mcol < L.d_out) {
           float sacc = 0.0f;
