@@ -60,10 +60,14 @@ constexpr int kStatusTimeout = 1;
 
 // Waits for the phase with the given parity.  Returns false if the limit ran out or another thread
 // of the CTA has already given up (abort flag); the caller then leaves its loop.
+// SLEEP_NS > 0 backs off between polls (for waiters that are not on the critical path: polling warps cost
+// issue slots and power that the tensor pipe could use).
+template <int SLEEP_NS = 0>
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status) {
   if (mbar_try_wait(bar, parity)) return true;
   const unsigned long long t0 = globaltimer_ns();
   for (uint32_t spin = 1;; ++spin) {
+    if (SLEEP_NS > 0) __nanosleep(SLEEP_NS);
     if (mbar_try_wait(bar, parity)) return true;
     if ((spin & 63u) == 0u) {
       if (*abort_flag) return false;
