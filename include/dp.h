@@ -126,6 +126,28 @@ DP_API int dp_philox_u32(uint32_t* out, int64_t n_words, int64_t elem_offset, ui
 /* Test utility: mask[i,t,s] = (ids[i,t] == ids[i,s]) as bytes, the first factor of the embedding Gram. */
 DP_API int dp_token_equality_mask(const int32_t* ids, int B, int T, uint8_t* mask, void* cuda_stream);
 
+/* Floats of fixed device scratch behind dp_layernorm_sqnorms_static (4 MiB, held by every GPU that loads the
+ * library until the process exits). */
+#define DP_STATIC_SCRATCH_FLOATS (1u << 20)
+
+/* (No counterpart in the paper: a variant for callers that cannot supply scratch memory.)
+ * Squared L2 norms of ONE LayerNorm layer's per-example gain and bias gradients, like dp_per_example_sqnorms
+ * restricted to that layer, but with the per-example column sums kept in a fixed array inside the library
+ * instead of a caller-provided workspace.  It exists for callers that cannot call cudaMalloc -- code running
+ * under a memory manager that owns the whole device, or where cudaMalloc's device-wide synchronisation is not
+ * acceptable -- and it calls no cudaMalloc, cudaFree or allocating library routine itself.
+ *   layer   HOST pointer to one dp_layer of kind DP_LAYERNORM (A = normalised input, G, B, T, d as usual;
+ *           accumulators ignored).  Inputs and the output stay caller-owned device memory.
+ *   sqnorm  [B] fp32, overwritten (accumulate_into = 0) or added to (1).
+ * Limit: B * 2 * d <= DP_STATIC_SCRATCH_FLOATS, otherwise DP_ERR_WORKSPACE (nothing is launched).
+ * The first call on a device looks up the array's device address (cudaGetSymbolAddress, with that device
+ * current); make that first call before any stream capture begins.
+ * All calls on a device share the one array, which keeps the previous call's contents; every call overwrites
+ * the part it reads, so nothing needs clearing, but two calls that overlap on the GPU (different streams) race
+ * on it: serialise them. */
+DP_API int dp_layernorm_sqnorms_static(const dp_layer* layer /*HOST*/, float* sqnorm, int accumulate_into,
+                                       void* cuda_stream);
+
 /* Waits for the stream, then returns and clears the sticky device-side status (DP_OK, DP_ERR_TIMEOUT
  * or DP_ERR_BAD_ID).  Device code never traps: a wait that runs out or an id out of range is recorded
  * here and the offending work is skipped. */

@@ -23,7 +23,8 @@ _KINDS = {"linear": DP_LINEAR, "layernorm": DP_LAYERNORM, "embedding": DP_EMBEDD
 
 EXPORTS = ["dp_workspace_bytes", "dp_per_example_sqnorms", "dp_clip_factors", "dp_clipped_accumulate",
            "dp_add_noise_and_scale", "dp_adamw_step", "dp_noise_scale_adamw_step", "dp_philox_u32",
-           "dp_token_equality_mask", "dp_poll_status", "dp_launch_count", "dp_status_string", "dp_version"]
+           "dp_token_equality_mask", "dp_layernorm_sqnorms_static", "dp_poll_status", "dp_launch_count",
+           "dp_status_string", "dp_version"]
 
 
 class dp_layer(C.Structure):
@@ -62,6 +63,7 @@ def lib() -> C.CDLL:
                                                 f32, f32, f32, f32, f32, i64, vp]
         L.dp_philox_u32.argtypes = [vp, i64, i64, u64, u64, vp]
         L.dp_token_equality_mask.argtypes = [vp, i32, i32, vp, vp]
+        L.dp_layernorm_sqnorms_static.argtypes = [vp, vp, i32, vp]
         L.dp_poll_status.argtypes = [vp]
         L.dp_status_string.restype = C.c_char_p
         L.dp_status_string.argtypes = [i32]
@@ -223,6 +225,19 @@ def dp_token_equality_mask(ids: torch.Tensor, mask: torch.Tensor, stream=None) -
     B, T = ids.shape
     _check("dp_token_equality_mask", lib().dp_token_equality_mask(_ptr(ids), B, T, _ptr(mask), _stream(stream)))
     return mask
+
+
+STATIC_SCRATCH_FLOATS = 1 << 20
+
+
+def dp_layernorm_sqnorms_static(layers: LayerList, sqnorm: torch.Tensor, accumulate_into: bool = False,
+                                stream=None) -> torch.Tensor:
+    """Norms of the single LayerNorm layer in `layers` with the library's fixed scratch (no workspace)."""
+    if len(layers) != 1:
+        raise ValueError("exactly one LayerNorm layer expected")
+    _check("dp_layernorm_sqnorms_static",
+           lib().dp_layernorm_sqnorms_static(layers.ptr, _ptr(sqnorm), int(accumulate_into), _stream(stream)))
+    return sqnorm
 
 
 def dp_launch_count() -> int:

@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libdp_b200.so")
-SOURCES = ["dp_api.cu", "dp_stream.cu", "dp_generic.cu", "dp_umma.cu"]
+SOURCES = ["dp_api.cu", "dp_stream.cu", "dp_generic.cu", "dp_umma.cu", "dp_noalloc.cu"]
 
 
 def _nvcc() -> str:
