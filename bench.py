@@ -29,6 +29,10 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
+# DRAM bytes (read + write) of one k_accum launch over the 24-block stack, from the ncu capture summarised in
+# profiles/k_accum_2blocks_full.md (2-block case x 12).  Set to None whenever that kernel changes.
+ACCUM_TRAFFIC_BYTES = 40.7e9
+
 METRIC = "dp_sgd_examples_per_s_bert_large"
 UNIT = "examples/s"
 WORKLOAD = "bert_large"
@@ -292,11 +296,14 @@ def main():
     T, B = wl.T, wl.B
     flops_acc = sum(2.0 * B * T * wl.specs[k].d_in * wl.specs[k].d_out for k in lin_idx)
     ach_tf = flops_acc / (phases[1] * 1e-3) / 1e12
+    bytes_acc = sum(2.0 * B * T * (wl.specs[k].d_in + wl.specs[k].d_out)
+                    + 8.0 * wl.specs[k].d_in * wl.specs[k].d_out for k in lin_idx)
     roofline = {"kernel": "clipped-accumulate GEMM (all linear layers, one call)", "bound": "tensor",
                 "achieved": ach_tf, "peak": peaks["tf_sustained"], "unit": "TFLOP/s",
                 "frac": ach_tf / peaks["tf_sustained"], "frac_of_burst": ach_tf / peaks["tf_burst"],
                 "peak_source": peaks["source"] + " (sustained bf16; kernel timed inside a long step)",
-                "traffic": None}
+                "traffic": ACCUM_TRAFFIC_BYTES if args.blocks == 24 else None,
+                "algorithmic_bytes": bytes_acc}
     bytes_norm = sum(2.0 * B * T * (wl.specs[k].d_in + wl.specs[k].d_out) for k in lin_idx) \
         + sum(2.0 * 2 * B * T * wl.specs[k].d_out for k in rest_idx if wl.specs[k].kind == "layernorm") \
         + sum(2.0 * B * T * wl.specs[k].d_out + 4.0 * B * T for k in rest_idx if wl.specs[k].kind == "embedding")
