@@ -58,7 +58,8 @@ typedef enum { DP_F32 = 0, DP_BF16 = 1 } dp_dtype;
  *                 for an embedding the first factor is the token-id equality mask.
  *   MATERIALIZED  tiles of A_i^T G_i formed on chip, squared and summed; for an embedding,
  *                 rows with equal ids are summed first.
- *   AUTO          GRAM iff T * (d_in + d_out) < d_in * d_out, the flop count of either way. */
+ *   AUTO          linear: GRAM iff T * (d_in + d_out) <= d_in * d_out, the flop count of either way;
+ *                 embedding: GRAM whenever the tensor-core kernel accepts the layer (bf16, d_out % 64 == 0). */
 typedef enum { DP_PATH_AUTO = 0, DP_PATH_GRAM = 1, DP_PATH_MATERIALIZED = 2 } dp_path;
 
 /* One trainable layer of one microbatch.  B and T must be equal across the layers of a call. */
@@ -152,6 +153,11 @@ DP_API int dp_layernorm_sqnorms_static(const dp_layer* layer /*HOST*/, float* sq
  * or DP_ERR_BAD_ID).  Device code never traps: a wait that runs out or an id out of range is recorded
  * here and the offending work is skipped. */
 DP_API int dp_poll_status(void* cuda_stream);
+
+/* Diagnostic: after dp_poll_status returned DP_ERR_TIMEOUT, info[0..4] = {wait site tag, block index, stage or
+ * tile counter, barrier parity, thread index} of the first bounded device-side wait that gave up (HOST array).
+ * Synchronises the device. */
+DP_API int dp_last_timeout_info(int info[5]);
 
 /* Number of kernels this library has launched in the calling process so far (host-side counter). */
 DP_API long long dp_launch_count(void);

@@ -23,7 +23,7 @@ _KINDS = {"linear": DP_LINEAR, "layernorm": DP_LAYERNORM, "embedding": DP_EMBEDD
 
 EXPORTS = ["dp_workspace_bytes", "dp_per_example_sqnorms", "dp_clip_factors", "dp_clipped_accumulate",
            "dp_add_noise_and_scale", "dp_adamw_step", "dp_noise_scale_adamw_step", "dp_philox_u32",
-           "dp_token_equality_mask", "dp_layernorm_sqnorms_static", "dp_poll_status", "dp_launch_count",
+           "dp_token_equality_mask", "dp_layernorm_sqnorms_static", "dp_poll_status", "dp_last_timeout_info", "dp_launch_count",
            "dp_status_string", "dp_version"]
 
 
@@ -238,6 +238,12 @@ def dp_layernorm_sqnorms_static(layers: LayerList, sqnorm: torch.Tensor, accumul
     _check("dp_layernorm_sqnorms_static",
            lib().dp_layernorm_sqnorms_static(layers.ptr, _ptr(sqnorm), int(accumulate_into), _stream(stream)))
     return sqnorm
+
+
+def dp_last_timeout_info():
+    info = (C.c_int * 5)()
+    _check("dp_last_timeout_info", lib().dp_last_timeout_info(info))
+    return list(info)
 
 
 def dp_launch_count() -> int:

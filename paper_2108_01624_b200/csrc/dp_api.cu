@@ -7,7 +7,8 @@
 
 namespace dpk {
 
-__device__ int g_status_word = 0;
+// [0] sticky status code; [1..5] where the first bounded wait gave up (tag, block, aux, parity, thread).
+__device__ int g_status_word[8] = {0, 0, 0, 0, 0, 0, 0, 0};
 
 static std::atomic<long long> g_launches{0};
 void note_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
@@ -94,6 +95,9 @@ static WsPlan plan_workspace(const dp_layer* layers, int n_layers) {
     if (L.kind == DP_LINEAR && umma_supported(L)) {
       p.umma_idx.push_back(l);
       p.umma_gram.push_back(use_gram(L) ? 1 : 0);
+    } else if (L.kind == DP_EMBEDDING && L.path != DP_PATH_MATERIALIZED && umma_supported(L)) {
+      p.umma_idx.push_back(l);     // norms only: token-id equality mask times G G^T in the Gram kernel
+      p.umma_gram.push_back(1);
     }
   }
   if (!p.umma_idx.empty()) {
@@ -193,8 +197,11 @@ int dp_clipped_accumulate(const dp_layer* layers, int n_layers, const float* cli
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
   int* status = status_ptr();
   if (!status) return DP_ERR_CUDA;
-  if (!plan.umma_idx.empty()) {
-    rc = launch_umma_accumulate(layers, plan.umma_idx.data(), (int)plan.umma_idx.size(), clip, status, s);
+  std::vector<int> lin_idx;      // the tensor-core accumulate takes linear layers only
+  for (int l : plan.umma_idx)
+    if (layers[l].kind == DP_LINEAR) lin_idx.push_back(l);
+  if (!lin_idx.empty()) {
+    rc = launch_umma_accumulate(layers, lin_idx.data(), (int)lin_idx.size(), clip, status, s);
     if (rc != DP_OK) return rc;
   }
   std::vector<ColTaskHost> tasks;
@@ -318,6 +325,13 @@ int dp_poll_status(void* cuda_stream) {
   if (h != STATUS_OK) DP_CUDA(cudaMemset(status, 0, sizeof(int)));
   if (h == STATUS_TIMEOUT) return DP_ERR_TIMEOUT;
   if (h == STATUS_BAD_ID) return DP_ERR_BAD_ID;
+  return DP_OK;
+}
+
+int dp_last_timeout_info(int info[5]) {
+  int* status = status_ptr();
+  if (!status || !info) return DP_ERR_ARG;
+  DP_CUDA(cudaMemcpy(info, status + 1, 5 * sizeof(int), cudaMemcpyDeviceToHost));
   return DP_OK;
 }
 

@@ -62,8 +62,11 @@ constexpr int kStatusTimeout = 1;
 // of the CTA has already given up (abort flag); the caller then leaves its loop.
 // SLEEP_NS > 0 backs off between polls (for waiters that are not on the critical path: polling warps cost
 // issue slots and power that the tensor pipe could use).
+// `tag` and `aux` identify the wait in the diagnostic record that the first waiter to give up leaves behind
+// (status[1..5] = tag, block, aux, parity, thread), read on the host by dp_last_timeout_info.
 template <int SLEEP_NS = 0>
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status) {
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status,
+                                          int tag = 0, int aux = 0) {
   if (mbar_try_wait(bar, parity)) return true;
   const unsigned long long t0 = globaltimer_ns();
   for (uint32_t spin = 1;; ++spin) {
@@ -72,7 +75,13 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
     if ((spin & 63u) == 0u) {
       if (*abort_flag) return false;
       if (globaltimer_ns() - t0 > kWaitLimitNs) {
-        atomicCAS(status, 0, kStatusTimeout);
+        if (atomicCAS(status, 0, kStatusTimeout) == 0) {
+          status[1] = tag;
+          status[2] = (int)blockIdx.x;
+          status[3] = aux;
+          status[4] = (int)parity;
+          status[5] = (int)threadIdx.x;
+        }
         *abort_flag = 1;
         return false;
       }

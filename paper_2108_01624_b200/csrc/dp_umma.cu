@@ -3,7 +3,10 @@
 //   k_gram_sqnorm  per-example squared norm by the token-Gram identity
 //                  |A_i^T G_i|_F^2 + |1^T G_i|^2 = < A_i A_i^T + [bias] 1 1^T , G_i G_i^T >.
 //                  Both 128x128 fp32 Grams of a token-block pair live in TMEM (2 x 128 columns,
-//                  double-buffered); operands are K-major 128x64 tiles fetched by TMA.
+//                  double-buffered); operands are K-major 128x64 tiles fetched by TMA.  For a token
+//                  embedding the input is one-hot, so A_i A_i^T is the token-id equality mask: only
+//                  G_i G_i^T is formed on the tensor cores and the epilogue multiplies it by
+//                  [id_t == id_s] (integer compares).
 //   k_tile<ACCUM>  acc_w^T tile (128 of d_out x 256 of d_in) += sum over tokens of G^T diag(c) A: one
 //                  128x256x16 UMMA per 16 tokens, both operands MN-major straight from the row-major
 //                  activations.  The per-example factor c is applied to the 128-wide G tile in shared
@@ -30,11 +33,12 @@ struct alignas(64) UmmaLayer {
   CUtensorMap mapA;   // [B, T, d_in]  bf16
   float* acc_w;
   float* acc_b;
-  int d_out, d_in;
+  const int32_t* ids;     // embedding layers (Gram kernel): token ids [B, T]; the id-equality mask replaces A A^T
+  int d_out, d_in;        // embedding: d_in = 0 (there is no A operand to stream)
   int tiles_m, tiles_n;   // tile kernels: 128-wide tiles over d_out, 256-wide tiles over d_in
   int item_start;         // first work item of this layer within the launch
   int partial_base;       // first per-example partial slot of this layer
-  int has_bias, pad;
+  int has_bias, is_emb;
 };
 
 struct UmmaParams {
@@ -199,15 +203,34 @@ __global__ void __launch_bounds__(G_THREADS, 1) k_gram_sqnorm(const __grid_const
       tc_fence_after();
       const float bias1 = L.has_bias ? 1.0f : 0.0f;
       float sum = 0.0f;
+      if (L.is_emb) {
+        // first factor = [id_t == id_s]; rows and columns beyond T meet zero entries of G G^T
+        const int32_t* idrow = L.ids + (size_t)i * P.T;
+        const int trow = r * 128 + (int)q * 32 + lane;
+        const int32_t my_id = trow < P.T ? __ldg(idrow + trow) : -1;
 #pragma unroll 1
-      for (int ch = 0; ch < 4; ++ch) {
-        uint32_t pv[32], qv[32];
-        const uint32_t ta = tmem_base + ((q * 32u) << 16) + buf * 256u + (uint32_t)ch * 32u;
-        tmem_ld_32x32(ta, pv);
-        tmem_ld_32x32(ta + 128u, qv);
-        tmem_ld_wait();
+        for (int ch = 0; ch < 4; ++ch) {
+          uint32_t qv[32];
+          tmem_ld_32x32(tmem_base + ((q * 32u) << 16) + buf * 256u + 128u + (uint32_t)ch * 32u, qv);
+          tmem_ld_wait();
+          const int s0 = c * 128 + ch * 32;
 #pragma unroll
-        for (int j = 0; j < 32; ++j) sum = fmaf(__uint_as_float(pv[j]) + bias1, __uint_as_float(qv[j]), sum);
+          for (int j = 0; j < 32; ++j) {
+            const int32_t other = (s0 + j < P.T) ? __ldg(idrow + s0 + j) : -2;
+            sum += (other == my_id) ? __uint_as_float(qv[j]) : 0.0f;
+          }
+        }
+      } else {
+#pragma unroll 1
+        for (int ch = 0; ch < 4; ++ch) {
+          uint32_t pv[32], qv[32];
+          const uint32_t ta = tmem_base + ((q * 32u) << 16) + buf * 256u + (uint32_t)ch * 32u;
+          tmem_ld_32x32(ta, pv);
+          tmem_ld_32x32(ta + 128u, qv);
+          tmem_ld_wait();
+#pragma unroll
+          for (int j = 0; j < 32; ++j) sum = fmaf(__uint_as_float(pv[j]) + bias1, __uint_as_float(qv[j]), sum);
+        }
       }
       tc_fence_before();
       __syncwarp();
@@ -585,7 +608,7 @@ __global__ void __launch_bounds__(A_THREADS, 1) k_accum(const __grid_constant__ 
         for (int e = t.e0; e < t.e1 && alive; ++e) {
           for (int tb = 0; tb < n_tb; ++tb) {
             const uint32_t slot = it % A_STAGES, ph = (it / A_STAGES) & 1u;
-            if (!mbar_wait(&S->empty[slot], ph ^ 1u, abort_flag, P.status)) { alive = false; break; }
+            if (!mbar_wait(&S->empty[slot], ph ^ 1u, abort_flag, P.status, 1, (int)it)) { alive = false; break; }
             uint8_t* st = tiles + slot * A_STAGE_BYTES;
             mbar_arrive_expect_tx(&S->full[slot], 8u * box_bytes);
 #pragma unroll
@@ -610,14 +633,14 @@ __global__ void __launch_bounds__(A_THREADS, 1) k_accum(const __grid_constant__ 
       bool alive = true;
       for (int item = blockIdx.x; item < P.total_items && alive; item += gridDim.x, ++tile_it) {
         const AccumItem t = accum_decode(P, item);
-        if (!mbar_wait(&S->tmem_empty, (tile_it & 1u) ^ 1u, abort_flag, P.status)) { alive = false; break; }
+        if (!mbar_wait(&S->tmem_empty, (tile_it & 1u) ^ 1u, abort_flag, P.status, 2, (int)tile_it)) { alive = false; break; }
         tc_fence_after();
         uint32_t acc = 0;
         for (int e = t.e0; e < t.e1 && alive; ++e) {
           for (int tb = 0; tb < n_tb; ++tb) {
             const uint32_t slot = it % A_STAGES, ph = (it / A_STAGES) & 1u;
             ++it;
-            if (!mbar_wait(&S->ready[slot], ph, abort_flag, P.status)) { alive = false; break; }
+            if (!mbar_wait(&S->ready[slot], ph, abort_flag, P.status, 3, (int)it)) { alive = false; break; }
             tc_fence_after();
             const uint32_t am = smem_u32(tiles + slot * A_STAGE_BYTES), an = am + A_M_BYTES;
 #pragma unroll
@@ -640,6 +663,9 @@ __global__ void __launch_bounds__(A_THREADS, 1) k_accum(const __grid_constant__ 
       mbar_wait_drain(&S->drain, 0u, P.status);
     }
   } else {   // ---------------- warps 2..9: scale the G tile (and bias column sums), then drain the accumulator
+    // All 256 threads handle every stage and all arrive on `ready`: an mbarrier wait tells phases apart by
+    // parity only, so no waiter may ever be two phases away from its barrier; here the MMA cannot pass a
+    // stage (and the producer cannot refill its slot) before every worker thread has seen it.
     const uint32_t q = (uint32_t)warp & 3u;
     const int h = warp >= 6 ? 1 : 0;                  // which 128-row half of the tile this warp drains
     const int tt = threadIdx.x - 64;                  // 0..255
@@ -663,7 +689,7 @@ __global__ void __launch_bounds__(A_THREADS, 1) k_accum(const __grid_constant__ 
         for (int tb = 0; tb < n_tb; ++tb) {
           const uint32_t slot = it % A_STAGES, ph = (it / A_STAGES) & 1u;
           ++it;
-          if (alive && !mbar_wait(&S->full[slot], ph, abort_flag, P.status)) alive = false;
+          if (alive && !mbar_wait(&S->full[slot], ph, abort_flag, P.status, 4, (int)it)) alive = false;
           if (!alive) continue;
           if (cf != 1.0f || need_bias) {
             uint8_t* base = tiles + slot * A_STAGE_BYTES + ta * A_ATOM_BYTES + kk * 128 + jp * 16;
@@ -704,7 +730,7 @@ __global__ void __launch_bounds__(A_THREADS, 1) k_accum(const __grid_constant__ 
         asm volatile("bar.sync 2, 256;" ::: "memory");
       }
       // ---- drain the accumulator: rows [h*128 + q*32, +32) of the tile
-      if (alive) alive = __all_sync(0xffffffffu, mbar_wait(&S->tmem_full, tile_it & 1u, abort_flag, P.status));
+      if (alive) alive = __all_sync(0xffffffffu, mbar_wait(&S->tmem_full, tile_it & 1u, abort_flag, P.status, 5, (int)tile_it));
       if (!alive) continue;
       tc_fence_after();
       const int m = t.m0 + h * 128 + (int)q * 32 + lane;
@@ -764,6 +790,10 @@ static bool encode_map(CUtensorMap* map, const void* base, int B, int T, int d, 
 }
 
 bool umma_supported(const dp_layer& L) {
+  if (L.kind == DP_EMBEDDING) {   // mask-Gram norm only (the accumulate is a scatter, not a contraction)
+    return L.dtype == DP_BF16 && L.d_out % 64 == 0 && (reinterpret_cast<uintptr_t>(L.G) & 15u) == 0 &&
+           (long long)L.T * L.d_out * 2 < (1ll << 40);
+  }
   if (L.kind != DP_LINEAR || L.dtype != DP_BF16) return false;
   if (L.d_in % 64 != 0 || L.d_out % 64 != 0) return false;
   if ((reinterpret_cast<uintptr_t>(L.A) | reinterpret_cast<uintptr_t>(L.G)) & 15u) return false;
@@ -799,16 +829,19 @@ static bool ensure_smem(K kernel, int bytes) {
 }
 
 static bool fill_layer(UmmaLayer& U, const dp_layer& L, int box_rows) {
+  const bool emb = L.kind == DP_EMBEDDING;
   if (!encode_map(&U.mapG, L.G, L.B, L.T, L.d_out, box_rows)) return false;
-  if (!encode_map(&U.mapA, L.A, L.B, L.T, L.d_in, box_rows)) return false;
+  if (emb) U.mapA = U.mapG;      // never used: an embedding streams no A operand (d_in = 0 below)
+  else if (!encode_map(&U.mapA, L.A, L.B, L.T, L.d_in, box_rows)) return false;
   U.acc_w = L.acc_w;
   U.acc_b = L.acc_b;
+  U.ids = emb ? L.ids : nullptr;
   U.d_out = L.d_out;
-  U.d_in = L.d_in;
+  U.d_in = emb ? 0 : L.d_in;
   U.tiles_m = ceil_div(L.d_out, 128);
   U.tiles_n = ceil_div(L.d_in, 256);
-  U.has_bias = L.has_bias;
-  U.pad = 0;
+  U.has_bias = emb ? 0 : L.has_bias;
+  U.is_emb = emb ? 1 : 0;
   return true;
 }
 

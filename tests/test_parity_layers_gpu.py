@@ -157,6 +157,23 @@ def test_out_of_range_token_id_is_skipped_and_reported():
     assert rel_l2(to_np(accs[0][0]), E) <= 1e-6
 
 
+def test_embedding_mask_gram_equals_grouped_rows():
+    """Token-id equality Gram (tensor cores) against the grouped-row kernel and the checker, heavy duplicates."""
+    spec = [LayerSpec(EMBEDDING, 40, 128, False, "emb")]
+    for B, T in ((5, 128), (3, 200), (4, 33)):
+        data = random_layers(spec, B, T, torch.bfloat16, DEV, seed=T, g_scale=0.05, vocab_dup=9)
+        n_ref = O.per_example_sqnorms(to_oracle_layers(data))
+        got = {}
+        for path in (b.DP_PATH_GRAM, b.DP_PATH_MATERIALIZED):
+            ll, _ = make_layer_list(data, DEV, [path])
+            n, _, _ = gpu_norms_clip(ll, 1.0)
+            got[path] = to_np(n)
+            np.testing.assert_allclose(got[path], n_ref, rtol=2 * CLIP_TOL)
+        np.testing.assert_allclose(got[b.DP_PATH_GRAM], got[b.DP_PATH_MATERIALIZED], rtol=1e-4)
+    assert b.dp_poll_status() == 0
+    assert len(b.dp_last_timeout_info()) == 5
+
+
 def test_workspace_too_small_is_refused():
     data = random_layers(SMALL, 2, 16, torch.bfloat16, DEV, seed=2)
     ll, _ = make_layer_list(data, DEV)
