@@ -120,6 +120,21 @@ DP_API int dp_noise_scale_adamw_step(float* theta, float* m, float* v, float* ac
                               uint64_t step, double lr, double beta1, double beta2, double xi, double weight_decay,
                               int64_t t, void* cuda_stream);
 
+/* dp_noise_scale_adamw_step that also accumulates the two squared norms of the gradient-SNR diagnostic of
+ * Section 5.2.1 (norm of the aggregated clipped gradient over norm of the noise vector) in the same pass:
+ *   sq_sums[0] += sum_e acc_e^2,   sq_sums[1] += sum_e (sigma C z_e)^2      (device double[2], 8-byte aligned).
+ * The caller zeroes sq_sums before the first tensor of a macro-batch; SNR = sqrt(sq_sums[0] / sq_sums[1]).
+ * Block sums are combined with fp64 atomics, so the last bits depend on the launch. */
+DP_API int dp_noise_scale_adamw_step_snr(float* theta, float* m, float* v, float* acc, int zero_acc, int64_t n,
+                                         int64_t elem_offset, double sigma, double C, int64_t batch_size,
+                                         uint64_t seed, uint64_t step, double lr, double beta1, double beta2,
+                                         double xi, double weight_decay, int64_t t, double* sq_sums,
+                                         void* cuda_stream);
+
+/* Clipping statistics of a microbatch (the other diagnostic that accompanies the gradient-SNR curves of
+ * Section 5.2.1): out[0] = fraction of examples with clip_i < 1, out[1] = mean clip_i.  out: device float[2]. */
+DP_API int dp_clip_stats(const float* clip, int B, float* out, void* cuda_stream);
+
 /* Test utility: out[k] = the raw Philox word of element elem_offset + k (lane (e & 3) of block e >> 2). */
 DP_API int dp_philox_u32(uint32_t* out, int64_t n_words, int64_t elem_offset, uint64_t seed, uint64_t step,
                   void* cuda_stream);

@@ -305,3 +305,21 @@ def privatised_gradient(microbatches: Sequence[Sequence[OracleLayer]], C: float,
     g = [[add_noise_and_scale(a, sigma, C, N, seed, step, off)
           for a, off in zip(acc, offs)] for acc, offs in zip(accs, elem_offsets)]
     return g, clips
+
+
+# ---------------------------------------------------------------------------
+# Diagnostics of Section 5.2.1: gradient-SNR and clipping statistics
+# ---------------------------------------------------------------------------
+
+def gradient_snr_sums(acc: np.ndarray, sigma: float, C: float, seed: int, step: int, elem_offset: int = 0):
+    """(sum acc^2, sum (sigma C z)^2) over one tensor; gradient-SNR of a macro-batch is the root of the ratio
+    of the two sums taken over ALL tensors: ||aggregated clipped gradient|| / ||noise vector||."""
+    S = np.asarray(acc, dtype=np.float64).ravel()
+    z = standard_normals(S.size, elem_offset, seed, step)
+    return float(np.sum(S * S)), float(np.sum((float(sigma) * float(C) * z) ** 2))
+
+
+def clip_stats(clip: np.ndarray):
+    """(fraction of examples that were clipped, mean clip factor)."""
+    c = np.asarray(clip, dtype=np.float64)
+    return float(np.mean(c < 1.0)), float(np.mean(c))

@@ -22,7 +22,8 @@ DP_PATH_AUTO, DP_PATH_GRAM, DP_PATH_MATERIALIZED = 0, 1, 2
 _KINDS = {"linear": DP_LINEAR, "layernorm": DP_LAYERNORM, "embedding": DP_EMBEDDING}
 
 EXPORTS = ["dp_workspace_bytes", "dp_per_example_sqnorms", "dp_clip_factors", "dp_clipped_accumulate",
-           "dp_add_noise_and_scale", "dp_adamw_step", "dp_noise_scale_adamw_step", "dp_philox_u32",
+           "dp_add_noise_and_scale", "dp_adamw_step", "dp_noise_scale_adamw_step", "dp_noise_scale_adamw_step_snr",
+           "dp_clip_stats", "dp_philox_u32",
            "dp_token_equality_mask", "dp_layernorm_sqnorms_static", "dp_poll_status", "dp_last_timeout_info", "dp_launch_count",
            "dp_status_string", "dp_version"]
 
@@ -61,6 +62,9 @@ def lib() -> C.CDLL:
         L.dp_adamw_step.argtypes = [vp, vp, vp, vp, i64, f32, f32, f32, f32, f32, i64, vp]
         L.dp_noise_scale_adamw_step.argtypes = [vp, vp, vp, vp, i32, i64, i64, f32, f32, i64, u64, u64,
                                                 f32, f32, f32, f32, f32, i64, vp]
+        L.dp_noise_scale_adamw_step_snr.argtypes = [vp, vp, vp, vp, i32, i64, i64, f32, f32, i64, u64, u64,
+                                                    f32, f32, f32, f32, f32, i64, vp, vp]
+        L.dp_clip_stats.argtypes = [vp, i32, vp, vp]
         L.dp_philox_u32.argtypes = [vp, i64, i64, u64, u64, vp]
         L.dp_token_equality_mask.argtypes = [vp, i32, i32, vp, vp]
         L.dp_layernorm_sqnorms_static.argtypes = [vp, vp, i32, vp]
@@ -212,6 +216,24 @@ def dp_noise_scale_adamw_step(theta, m, v, acc, zero_acc, sigma, C_, batch_size,
                                            theta.numel(), int(elem_offset), float(sigma), float(C_),
                                            int(batch_size), int(seed), int(step), float(lr), float(beta1),
                                            float(beta2), float(xi), float(weight_decay), int(t), _stream(stream)))
+
+
+def dp_noise_scale_adamw_step_snr(theta, m, v, acc, zero_acc, sigma, C_, batch_size, seed, step, lr, beta1, beta2,
+                                  xi, weight_decay, t, sq_sums: torch.Tensor, elem_offset: int = 0, stream=None) -> None:
+    """sq_sums: float64 device tensor [2], accumulated into (sum acc^2, sum (sigma C z)^2)."""
+    if sq_sums.dtype != torch.float64 or sq_sums.numel() != 2:
+        raise ValueError("sq_sums must be a float64 tensor with 2 elements")
+    _check("dp_noise_scale_adamw_step_snr",
+           lib().dp_noise_scale_adamw_step_snr(_ptr(theta), _ptr(m), _ptr(v), _ptr(acc), int(bool(zero_acc)),
+                                               theta.numel(), int(elem_offset), float(sigma), float(C_),
+                                               int(batch_size), int(seed), int(step), float(lr), float(beta1),
+                                               float(beta2), float(xi), float(weight_decay), int(t),
+                                               _ptr(sq_sums), _stream(stream)))
+
+
+def dp_clip_stats(clip: torch.Tensor, out: torch.Tensor, stream=None) -> torch.Tensor:
+    _check("dp_clip_stats", lib().dp_clip_stats(_ptr(clip), clip.numel(), _ptr(out), _stream(stream)))
+    return out
 
 
 def dp_philox_u32(out: torch.Tensor, elem_offset: int, seed: int, step: int, stream=None) -> torch.Tensor:

@@ -295,6 +295,31 @@ int dp_noise_scale_adamw_step(float* theta, float* m, float* v, float* acc, int 
   return DP_OK;
 }
 
+int dp_noise_scale_adamw_step_snr(float* theta, float* m, float* v, float* acc, int zero_acc, int64_t n,
+                                  int64_t elem_offset, double sigma, double C, int64_t batch_size, uint64_t seed,
+                                  uint64_t step, double lr, double beta1, double beta2, double xi,
+                                  double weight_decay, int64_t t, double* sq_sums, void* cuda_stream) {
+  NoiseArgs na;
+  AdamArgs aa;
+  int rc = make_noise_args(n, elem_offset, sigma, C, batch_size, seed, step, &na);
+  if (rc != DP_OK) return rc;
+  if ((rc = make_adam_args(lr, beta1, beta2, xi, weight_decay, t, &aa)) != DP_OK) return rc;
+  if (!sq_sums) return DP_ERR_ARG;
+  if (misaligned(sq_sums, 8)) return DP_ERR_ALIGN;
+  if (n == 0) return DP_OK;
+  if (!theta || !m || !v || !acc) return DP_ERR_ARG;
+  if (misaligned(theta, 4) || misaligned(m, 4) || misaligned(v, 4) || misaligned(acc, 4)) return DP_ERR_ALIGN;
+  DP_CUDA(launch_noise_adamw(theta, m, v, acc, zero_acc, n, na, aa, static_cast<cudaStream_t>(cuda_stream), sq_sums));
+  return DP_OK;
+}
+
+int dp_clip_stats(const float* clip, int B, float* out, void* cuda_stream) {
+  if (!clip || !out || B <= 0) return DP_ERR_ARG;
+  if (misaligned(clip, 4) || misaligned(out, 4)) return DP_ERR_ALIGN;
+  DP_CUDA(launch_clip_stats(clip, B, out, static_cast<cudaStream_t>(cuda_stream)));
+  return DP_OK;
+}
+
 int dp_philox_u32(uint32_t* out, int64_t n_words, int64_t elem_offset, uint64_t seed, uint64_t step,
                   void* cuda_stream) {
   if (n_words < 0 || elem_offset < 0) return DP_ERR_ARG;

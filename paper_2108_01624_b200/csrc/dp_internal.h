@@ -37,8 +37,10 @@ cudaError_t launch_clip_factors(const float* sqnorm, int B, float C, float* clip
 cudaError_t launch_noise_scale(float* acc, long long n, const NoiseArgs& na, cudaStream_t s);
 cudaError_t launch_adamw(float* theta, float* m, float* v, const float* g, long long n, const AdamArgs& aa,
                          cudaStream_t s);
+// sq_sums (optional, device double[2]): adds sum(acc^2) and sum((sigma C z)^2), the gradient-SNR terms.
 cudaError_t launch_noise_adamw(float* theta, float* m, float* v, float* acc, int zero_acc, long long n,
-                               const NoiseArgs& na, const AdamArgs& aa, cudaStream_t s);
+                               const NoiseArgs& na, const AdamArgs& aa, cudaStream_t s, double* sq_sums = nullptr);
+cudaError_t launch_clip_stats(const float* clip, int B, float* out, cudaStream_t s);
 cudaError_t launch_philox_u32(uint32_t* out, long long n, const NoiseArgs& na, cudaStream_t s);
 cudaError_t launch_equality_mask(const int32_t* ids, int B, int T, uint8_t* mask, cudaStream_t s);
 

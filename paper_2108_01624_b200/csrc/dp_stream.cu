@@ -81,8 +81,9 @@ template <int MODE, bool VEC>
 __global__ void __launch_bounds__(256)
 k_stream(float* __restrict__ theta, float* __restrict__ m, float* __restrict__ v, float* __restrict__ acc,
          const float* __restrict__ g_in, int zero_acc, long long n, unsigned long long j0,
-         unsigned long long n_blocks, NoiseArgs na, AdamArgs aa) {
+         unsigned long long n_blocks, NoiseArgs na, AdamArgs aa, double* __restrict__ sq_sums) {
   const unsigned long long stride = (unsigned long long)gridDim.x * blockDim.x;
+  float s_sig = 0.0f, s_noi = 0.0f;      // sum acc^2 and sum (sigma C z)^2 of this thread (gradient-SNR terms)
   for (unsigned long long b = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x; b < n_blocks; b += stride) {
     const unsigned long long j = j0 + b;
     const long long k0 = (long long)(4ull * j) - na.elem_offset;   // local index of lane 0
@@ -91,6 +92,11 @@ k_stream(float* __restrict__ theta, float* __restrict__ m, float* __restrict__ v
       if (MODE != 1) {
         const float4 a4 = *reinterpret_cast<const float4*>(acc + k0);
         const float4 z = normals4(j, na);
+        if (sq_sums) {
+          s_sig += a4.x * a4.x + a4.y * a4.y + a4.z * a4.z + a4.w * a4.w;
+          const float nx = na.sigmaC * z.x, ny = na.sigmaC * z.y, nz = na.sigmaC * z.z, nw = na.sigmaC * z.w;
+          s_noi += nx * nx + ny * ny + nz * nz + nw * nw;
+        }
         gv.x = (a4.x + na.sigmaC * z.x) * na.inv_n;
         gv.y = (a4.y + na.sigmaC * z.y) * na.inv_n;
         gv.z = (a4.z + na.sigmaC * z.z) * na.inv_n;
@@ -124,7 +130,13 @@ k_stream(float* __restrict__ theta, float* __restrict__ m, float* __restrict__ v
         const long long k = k0 + l;
         if (k < 0 || k >= n) continue;
         float gv;
-        if (MODE != 1) gv = (acc[k] + na.sigmaC * z[l]) * na.inv_n; else gv = g_in[k];
+        if (MODE != 1) {
+          const float a1 = acc[k], n1 = na.sigmaC * z[l];
+          if (sq_sums) { s_sig += a1 * a1; s_noi += n1 * n1; }
+          gv = (a1 + n1) * na.inv_n;
+        } else {
+          gv = g_in[k];
+        }
         if (MODE == 0) {
           acc[k] = gv;
         } else {
@@ -134,6 +146,24 @@ k_stream(float* __restrict__ theta, float* __restrict__ m, float* __restrict__ v
           if (MODE == 2 && zero_acc) acc[k] = 0.0f;
         }
       }
+    }
+  }
+  if (MODE != 1 && sq_sums) {      // uniform branch: one double atomic per block and quantity
+    __shared__ double red[2][8];
+    double a = (double)s_sig, b = (double)s_noi;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      a += __shfl_down_sync(0xffffffffu, a, o);
+      b += __shfl_down_sync(0xffffffffu, b, o);
+    }
+    if ((threadIdx.x & 31) == 0) { red[0][threadIdx.x >> 5] = a; red[1][threadIdx.x >> 5] = b; }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      double ta = 0.0, tb = 0.0;
+#pragma unroll
+      for (int w = 0; w < 8; ++w) { ta += red[0][w]; tb += red[1][w]; }
+      atomicAdd(sq_sums, ta);
+      atomicAdd(sq_sums + 1, tb);
     }
   }
 }
@@ -153,7 +183,8 @@ static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 
 
 template <int MODE>
 static cudaError_t launch_stream(float* theta, float* m, float* v, float* acc, const float* g, int zero_acc,
-                                 long long n, const NoiseArgs& na, const AdamArgs& aa, cudaStream_t s) {
+                                 long long n, const NoiseArgs& na, const AdamArgs& aa, cudaStream_t s,
+                                 double* sq_sums = nullptr) {
   if (n <= 0) return cudaSuccess;
   const unsigned long long j0 = (unsigned long long)na.elem_offset >> 2;
   const unsigned long long j1 = ((unsigned long long)na.elem_offset + (unsigned long long)n + 3ull) >> 2;
@@ -163,8 +194,8 @@ static cudaError_t launch_stream(float* theta, float* m, float* v, float* acc, c
   if (MODE == 1) vec = vec && aligned16(g);
   if (MODE != 0) vec = vec && aligned16(theta) && aligned16(m) && aligned16(v);
   const int grid = stream_grid(nb);
-  if (vec) k_stream<MODE, true><<<grid, 256, 0, s>>>(theta, m, v, acc, g, zero_acc, n, j0, nb, na, aa);
-  else     k_stream<MODE, false><<<grid, 256, 0, s>>>(theta, m, v, acc, g, zero_acc, n, j0, nb, na, aa);
+  if (vec) k_stream<MODE, true><<<grid, 256, 0, s>>>(theta, m, v, acc, g, zero_acc, n, j0, nb, na, aa, sq_sums);
+  else     k_stream<MODE, false><<<grid, 256, 0, s>>>(theta, m, v, acc, g, zero_acc, n, j0, nb, na, aa, sq_sums);
   return counted(1);
 }
 
@@ -178,8 +209,36 @@ cudaError_t launch_adamw(float* theta, float* m, float* v, const float* g, long 
   return launch_stream<1>(theta, m, v, nullptr, g, 0, n, na, aa, s);
 }
 cudaError_t launch_noise_adamw(float* theta, float* m, float* v, float* acc, int zero_acc, long long n,
-                               const NoiseArgs& na, const AdamArgs& aa, cudaStream_t s) {
-  return launch_stream<2>(theta, m, v, acc, nullptr, zero_acc, n, na, aa, s);
+                               const NoiseArgs& na, const AdamArgs& aa, cudaStream_t s, double* sq_sums) {
+  return launch_stream<2>(theta, m, v, acc, nullptr, zero_acc, n, na, aa, s, sq_sums);
+}
+
+// out[0] = fraction of examples with clip < 1, out[1] = mean clip factor.  One block, fixed order.
+__global__ void __launch_bounds__(256) k_clip_stats(const float* __restrict__ clip, int B, float* __restrict__ out) {
+  __shared__ float red[2][8];
+  float cnt = 0.0f, sum = 0.0f;
+  for (int i = threadIdx.x; i < B; i += 256) {
+    const float c = clip[i];
+    cnt += (c < 1.0f) ? 1.0f : 0.0f;
+    sum += c;
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    cnt += __shfl_down_sync(0xffffffffu, cnt, o);
+    sum += __shfl_down_sync(0xffffffffu, sum, o);
+  }
+  if ((threadIdx.x & 31) == 0) { red[0][threadIdx.x >> 5] = cnt; red[1][threadIdx.x >> 5] = sum; }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    float a = 0.0f, b = 0.0f;
+    for (int w = 0; w < 8; ++w) { a += red[0][w]; b += red[1][w]; }
+    out[0] = a / (float)B;
+    out[1] = b / (float)B;
+  }
+}
+cudaError_t launch_clip_stats(const float* clip, int B, float* out, cudaStream_t s) {
+  k_clip_stats<<<1, 256, 0, s>>>(clip, B, out);
+  return counted(1);
 }
 
 // ---------------------------------------------------------------------------------------------

@@ -23,7 +23,8 @@ class DPStep:
     """
 
     def __init__(self, specs: Sequence[LayerSpec], device, C: float, sigma: float, lr: float, beta1: float,
-                 beta2: float, xi: float, weight_decay: float, seed: int = 0, theta: Optional[torch.Tensor] = None):
+                 beta2: float, xi: float, weight_decay: float, seed: int = 0, theta: Optional[torch.Tensor] = None,
+                 track_snr: bool = False):
         self.specs = list(specs)
         self.device = torch.device(device)
         self.C, self.sigma, self.lr, self.beta1, self.beta2 = C, sigma, lr, beta1, beta2
@@ -54,6 +55,8 @@ class DPStep:
         self.theta = torch.zeros_like(self.acc) if theta is None else theta
         self.t = 0
         self.examples_seen = 0
+        # gradient-SNR of Section 5.2.1: (sum acc^2, sum noise^2) of the last macro-batch, filled by the fused pass
+        self.sq_sums = torch.zeros(2, dtype=torch.float64, device=self.device) if track_snr else None
         self._ws = None
         self._sqnorm = None
         self._clip = None
@@ -98,7 +101,12 @@ class DPStep:
         """Noise, division by the macro-batch size and the AdamW update; clears the accumulator."""
         N = self.examples_seen if batch_size is None else batch_size
         self.t += 1
-        if fused:
+        if fused and self.sq_sums is not None:
+            self.sq_sums.zero_()
+            b.dp_noise_scale_adamw_step_snr(self.theta, self.m, self.v, self.acc, True, self.sigma, self.C, N,
+                                            self.seed, self.t, self.lr, self.beta1, self.beta2, self.xi,
+                                            self.weight_decay, self.t, self.sq_sums, 0, stream)
+        elif fused:
             b.dp_noise_scale_adamw_step(self.theta, self.m, self.v, self.acc, True, self.sigma, self.C, N, self.seed,
                                         self.t, self.lr, self.beta1, self.beta2, self.xi, self.weight_decay, self.t,
                                         0, stream)
@@ -108,3 +116,10 @@ class DPStep:
                             self.weight_decay, self.t, stream)
             self.acc.zero_()
         self.examples_seen = 0
+
+    def gradient_snr(self) -> float:
+        """||aggregated clipped gradient|| / ||noise vector|| of the last finished macro-batch (host sync)."""
+        if self.sq_sums is None:
+            raise RuntimeError("construct DPStep with track_snr=True")
+        s = self.sq_sums.cpu()
+        return float((s[0] / s[1]).sqrt()) if float(s[1]) > 0 else float("inf")

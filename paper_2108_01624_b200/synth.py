@@ -34,6 +34,7 @@ class LayerSpec:
     d_out: int
     has_bias: bool = False
     name: str = ""
+    ids: str = "zipf"   # EMBEDDING: "zipf" word-pieces, "position" 0..T-1, "segment" two sentence segments
 
     def n_params(self) -> int:
         if self.kind == LINEAR:
@@ -102,6 +103,13 @@ def workload(name: str) -> Workload:
         specs.append(LayerSpec(EMBEDDING, 30522, 1024, False, "tok_emb"))
         mb = 8192 if name == "bert_large_megabatch" else 1
         return Workload(name, 256, 128, torch.bfloat16, specs, microbatches=mb)
+    if name == "bert_large_embeddings":
+        # the input layer of BERT: word-piece, positional and token-type embeddings summed, then LayerNorm
+        specs = [LayerSpec(EMBEDDING, 30522, 1024, False, "tok_emb", "zipf"),
+                 LayerSpec(EMBEDDING, 512, 1024, False, "pos_emb", "position"),
+                 LayerSpec(EMBEDDING, 2, 1024, False, "type_emb", "segment"),
+                 LayerSpec(LAYERNORM, 1024, 1024, False, "emb_ln")]
+        return Workload(name, 256, 128, torch.bfloat16, specs)
     if name == "bert_large_layer_t512":
         return Workload(name, 64, 512, torch.bfloat16, encoder_layer_specs(1024, 4096))
     raise KeyError(name)
@@ -173,8 +181,15 @@ def generate(wl: Workload, seed: int = 0, device="cpu", microbatch: int = 0,
             G = G * s.view(B, 1, 1)
         G = G.to(wl.dtype)
         if sp.kind == EMBEDDING:
-            ids = zipf_ids(B, T, sp.d_in, 1.1, _gen(device, seed, microbatch, li, 2), device)
-            out.append(LayerData(sp, G=G, ids=ids))
+            gi = _gen(device, seed, microbatch, li, 2)
+            if sp.ids == "position":
+                ids = torch.arange(T, dtype=torch.int32, device=device).repeat(B, 1)
+            elif sp.ids == "segment":      # sentence A then sentence B, split point drawn per example
+                cut = torch.randint(1, max(T, 2), (B, 1), generator=gi, device=device)
+                ids = (torch.arange(T, device=device).view(1, T) >= cut).to(torch.int32)
+            else:
+                ids = zipf_ids(B, T, sp.d_in, 1.1, gi, device)
+            out.append(LayerData(sp, G=G, ids=ids.contiguous()))
         else:
             gA = _gen(device, seed, microbatch, li, 0)
             A = torch.randn(B, T, sp.d_in, generator=gA, device=device, dtype=torch.float32).to(wl.dtype)

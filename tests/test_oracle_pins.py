@@ -343,3 +343,30 @@ def test_privatised_gradient_composes(rng):
             z = O.standard_normals(x.size, pos, 1, 1).reshape(x.shape)
             np.testing.assert_allclose(y - x, 2.0 * 1.5 * z / 6.0, rtol=1e-9, atol=1e-12)
             pos += x.size
+
+
+# ---------------------------------------------------------------- gradient-SNR and clip statistics (Section 5.2.1)
+
+def test_gradient_snr_sums_closed_forms(rng):
+    n = 1_000_000
+    S = rng.standard_normal(n) * 3.0
+    sig2, noi2 = O.gradient_snr_sums(S, 1.3, 0.5, seed=8, step=2)
+    assert sig2 == pytest.approx(float(S @ S), rel=1e-13)
+    # ||sigma C z||^2 / (sigma^2 C^2 n) -> 1 (chi-square with n degrees of freedom)
+    assert noi2 / ((1.3 * 0.5) ** 2 * n) == pytest.approx(1.0, abs=5 * math.sqrt(2.0 / n))
+    # scaling the gradient by k scales the SNR by k; sigma scales it by 1/sigma
+    s2, n2 = O.gradient_snr_sums(2 * S, 2.6, 0.5, seed=8, step=2)
+    assert math.sqrt(s2 / n2) == pytest.approx(math.sqrt(sig2 / noi2), rel=1e-12)
+    # additive over a partition when the offsets follow the flat layout
+    a = O.gradient_snr_sums(S[:1234], 1.3, 0.5, 8, 2, 0)
+    b = O.gradient_snr_sums(S[1234:], 1.3, 0.5, 8, 2, 1234)
+    assert a[0] + b[0] == pytest.approx(sig2, rel=1e-12) and a[1] + b[1] == pytest.approx(noi2, rel=1e-12)
+    # the noise term is the residual of add_noise_and_scale
+    g = O.add_noise_and_scale(S[:5000], 1.3, 0.5, 7, 8, 2, 0)
+    resid = g * 7 - S[:5000]
+    assert float(resid @ resid) == pytest.approx(O.gradient_snr_sums(S[:5000], 1.3, 0.5, 8, 2, 0)[1], rel=1e-9)
+
+
+def test_clip_stats_values():
+    assert O.clip_stats(np.array([1.0, 1.0, 0.5, 0.25])) == (0.5, 0.6875)
+    assert O.clip_stats(np.ones(7)) == (0.0, 1.0)

@@ -1,0 +1,82 @@
+"""GPU parity of whole macro-steps through DPStep: varying batch size per step (the increasing schedule of
+Section 5.2.2 in miniature), gradient-SNR tracking, and the BERT input layer with its three embeddings."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2108_01624_b200 import DPStep, synth
+
+from .helpers import (EMBEDDING, LAYERNORM, LINEAR, LayerSpec, O, b, gpu_norms_clip, make_layer_list, random_layers,
+                      rel_l2, to_np, to_oracle_layers)
+
+pytestmark = pytest.mark.gpu
+
+if not torch.cuda.is_available():
+    pytest.skip("needs a CUDA device", allow_module_level=True)
+
+DEV = "cuda:0"
+SPECS = [LayerSpec(LINEAR, 128, 256, True, "fc1"), LayerSpec(LAYERNORM, 128, 128, False, "ln"),
+         LayerSpec(EMBEDDING, 30, 64, False, "emb")]
+
+
+def test_macro_steps_with_a_growing_batch_and_snr():
+    B, T = 8, 64
+    hp = dict(C=0.05, sigma=0.8, lr=1e-2, beta1=0.9, beta2=0.999, xi=1e-11, weight_decay=0.5)
+    step = DPStep(SPECS, DEV, seed=9, track_snr=True, **hp)
+    th = synth.initial_weights(step.n_flat, 1, DEV)
+    step.theta.copy_(th)
+    r_th, r_m, r_v = to_np(th), np.zeros(step.n_flat), np.zeros(step.n_flat)
+    seed_ctr = 0
+    for t, n_mb in enumerate((2, 3), start=1):              # the batch grows from 16 to 24 examples
+        mbs = []
+        for _ in range(n_mb):
+            data = random_layers(SPECS, B, T, torch.bfloat16, DEV, seed=100 + seed_ctr, g_scale=0.02, vocab_dup=6)
+            seed_ctr += 1
+            step.accumulate_microbatch(step.layer_list(data))
+            mbs.append(to_oracle_layers(data))
+        assert step.examples_seen == n_mb * B
+        acc = to_np(step.acc)
+        step.finish_macro_batch()
+        # checker: clipped sums -> flat layout -> noise / N -> AdamW
+        accs = O.zero_accumulators(mbs[0])
+        for ol in mbs:
+            O.clipped_accumulate(ol, O.clip_factors(O.per_example_sqnorms(ol), hp["C"]), accs)
+        flat = np.zeros(step.n_flat)
+        for li in range(len(SPECS)):
+            for k, a in enumerate(accs[li]):
+                off = step.offsets[li][k]
+                flat[off:off + a.size] = a.ravel()
+        assert rel_l2(acc, flat) <= 2e-2
+        g = O.add_noise_and_scale(acc, hp["sigma"], hp["C"], n_mb * B, seed=9, step=t, elem_offset=0)
+        new = O.adamw_step(r_th, r_m, r_v, g, hp["lr"], hp["beta1"], hp["beta2"], hp["xi"], hp["weight_decay"], t)
+        d, rd = to_np(step.theta) - r_th, new[0] - r_th
+        assert np.max(np.abs(d - rd)) <= 1e-4 * np.max(np.abs(rd)) + 1e-7 * np.max(np.abs(r_th))
+        r_th, r_m, r_v = to_np(step.theta), to_np(step.m), to_np(step.v)
+        s2, n2 = O.gradient_snr_sums(acc, hp["sigma"], hp["C"], 9, t, 0)
+        assert step.gradient_snr() == pytest.approx(np.sqrt(s2 / n2), rel=1e-4)
+    assert step.t == 2 and step.examples_seen == 0
+
+
+def test_bert_input_layer_three_embeddings():
+    """Word-piece (Zipf), positional (all ids distinct) and token-type (two ids) embeddings plus their LayerNorm."""
+    wl = synth.workload("bert_large_embeddings")
+    data = synth.generate(wl, seed=3, device=DEV, B=8)
+    ol = to_oracle_layers(data)
+    n_ref = O.per_example_sqnorms(ol)
+    c_ref = O.clip_factors(n_ref, 1e-3)
+    for path in (b.DP_PATH_AUTO, b.DP_PATH_MATERIALIZED):
+        ll, accs = make_layer_list(data, DEV, [path] * len(data))
+        n, c, ws = gpu_norms_clip(ll, 1e-3)
+        np.testing.assert_allclose(to_np(n), n_ref, rtol=2e-3)
+        np.testing.assert_allclose(to_np(c), c_ref, rtol=1e-3)
+        b.dp_clipped_accumulate(ll, c, ws)
+        ref = O.clipped_accumulate(ol, c_ref, O.zero_accumulators(ol))
+        for ld, acc, racc in zip(data, accs, ref):
+            for x, y in zip(acc, racc):
+                assert rel_l2(to_np(x), y) <= 2e-2, ld.spec.name
+    # closed forms: positions are all distinct -> |G|_F^2; a single segment id per half -> two row sums
+    G = to_np(data[1].G)
+    ll1, _ = make_layer_list([data[1]], DEV)
+    n1, _, _ = gpu_norms_clip(ll1, 1.0)
+    np.testing.assert_allclose(to_np(n1), (G ** 2).sum((1, 2)), rtol=2e-3)
+    assert b.dp_poll_status() == 0

@@ -172,3 +172,38 @@ def test_clip_factors_special_values():
     b.dp_clip_factors(n, C, c)
     ref = O.clip_factors(to_np(n), C)
     np.testing.assert_allclose(to_np(c), ref, rtol=1e-6)
+
+
+@pytest.mark.parametrize("n,off", [(1 << 20, 0), (50_003, 5)])
+def test_gradient_snr_sums_in_the_fused_pass(n, off):
+    """Same update as the plain fused call, plus sum acc^2 and sum (sigma C z)^2 against the checker."""
+    th, m, v, _ = _adam_case(n, 3)
+    S = (np.random.default_rng(4).standard_normal(n) * 20).astype(np.float32)
+    hp = dict(lr=6.0902e-4, b1=0.9, b2=0.999, xi=1e-11, wd=0.5, t=2)
+    sigma, C, N, seed, step = 1.1, 0.9, 1024, 5, 2
+    a = [torch.from_numpy(x.copy()).to(DEV) for x in (th, m, v, S)]
+    b_ = [torch.from_numpy(x.copy()).to(DEV) for x in (th, m, v, S)]
+    sums = torch.zeros(2, dtype=torch.float64, device=DEV)
+    b.dp_noise_scale_adamw_step_snr(a[0], a[1], a[2], a[3], True, sigma, C, N, seed, step, hp["lr"], hp["b1"],
+                                    hp["b2"], hp["xi"], hp["wd"], hp["t"], sums, elem_offset=off)
+    b.dp_noise_scale_adamw_step(b_[0], b_[1], b_[2], b_[3], True, sigma, C, N, seed, step, hp["lr"], hp["b1"],
+                                hp["b2"], hp["xi"], hp["wd"], hp["t"], elem_offset=off)
+    for x, y in zip(a, b_):
+        assert torch.equal(x, y)
+    ref = O.gradient_snr_sums(S.astype(np.float64), sigma, C, seed, step, off)
+    got = sums.cpu().numpy()
+    assert got[0] == pytest.approx(ref[0], rel=1e-5) and got[1] == pytest.approx(ref[1], rel=1e-4)
+    # accumulates across calls (tensors of one macro-batch)
+    c = [torch.from_numpy(x.copy()).to(DEV) for x in (th, m, v, S)]
+    b.dp_noise_scale_adamw_step_snr(c[0], c[1], c[2], c[3], False, sigma, C, N, seed, step, hp["lr"], hp["b1"],
+                                    hp["b2"], hp["xi"], hp["wd"], hp["t"], sums, elem_offset=off)
+    np.testing.assert_allclose(sums.cpu().numpy(), 2 * got, rtol=1e-9)
+
+
+def test_clip_stats_matches_checker():
+    g = torch.Generator().manual_seed(1)
+    for B in (1, 33, 256, 1000):
+        clip = torch.where(torch.rand(B, generator=g) < 0.4, torch.ones(B), torch.rand(B, generator=g)).to(DEV)
+        out = torch.empty(2, dtype=torch.float32, device=DEV)
+        b.dp_clip_stats(clip, out)
+        np.testing.assert_allclose(to_np(out), O.clip_stats(to_np(clip)), rtol=1e-5)
