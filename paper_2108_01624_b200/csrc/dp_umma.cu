@@ -28,6 +28,14 @@ using namespace ptx;
 
 constexpr int kMaxLayers = 96;
 
+// Tunables (overridable with -D for experiments; the defaults are what was measured best).
+#ifndef DP_ACCUM_WORKER_SLEEP_NS
+#define DP_ACCUM_WORKER_SLEEP_NS 0     // back-off between polls of the accumulate kernel's worker and producer waits
+#endif
+#ifndef DP_TMA_L2_PROMOTION
+#define DP_TMA_L2_PROMOTION 2          // 0 none, 1 128 B, 2 256 B
+#endif
+
 struct alignas(64) UmmaLayer {
   CUtensorMap mapG;   // [B, T, d_out] bf16
   CUtensorMap mapA;   // [B, T, d_in]  bf16
@@ -39,6 +47,7 @@ struct alignas(64) UmmaLayer {
   int item_start;         // first work item of this layer within the launch
   int partial_base;       // first per-example partial slot of this layer
   int has_bias, is_emb;
+  int scaled_g, pad;      // accumulate with pre-scaled operands: 1 if G is the operand that carries the clip factor
 };
 
 struct UmmaParams {
@@ -564,6 +573,11 @@ __device__ __forceinline__ void accum_store_chunk(const UmmaLayer& L, int m, int
   }
 }
 
+// PRE = false: the clip factor is applied to the G tile in shared memory by the worker warps (needs no scratch).
+// PRE = true : one operand of every layer was multiplied by the clip factors beforehand (k_prescale, a copy in
+//              the caller's workspace), so the tiles go from TMA straight to the UMMAs; the worker warps only
+//              read the G tile of the tiles that own a bias slice (column sums), and otherwise just drain.
+template <bool PRE>
 __global__ void __launch_bounds__(A_THREADS, 1) k_accum(const __grid_constant__ UmmaParams P) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* tiles = align1024(smem_raw);
@@ -608,7 +622,7 @@ __global__ void __launch_bounds__(A_THREADS, 1) k_accum(const __grid_constant__ 
         for (int e = t.e0; e < t.e1 && alive; ++e) {
           for (int tb = 0; tb < n_tb; ++tb) {
             const uint32_t slot = it % A_STAGES, ph = (it / A_STAGES) & 1u;
-            if (!mbar_wait(&S->empty[slot], ph ^ 1u, abort_flag, P.status, 1, (int)it)) { alive = false; break; }
+            if (!mbar_wait<DP_ACCUM_WORKER_SLEEP_NS>(&S->empty[slot], ph ^ 1u, abort_flag, P.status, 1, (int)it)) { alive = false; break; }
             uint8_t* st = tiles + slot * A_STAGE_BYTES;
             mbar_arrive_expect_tx(&S->full[slot], 8u * box_bytes);
 #pragma unroll
@@ -629,10 +643,11 @@ __global__ void __launch_bounds__(A_THREADS, 1) k_accum(const __grid_constant__ 
     }
   } else if (warp == 1) {
     if (lane == 0) {   // ---------------- MMA issuer ----------------
-      uint32_t it = 0, tile_it = 0;
+      uint32_t it = 0, rit = 0, tile_it = 0;     // rit counts the stages that go through the `ready` barriers
       bool alive = true;
       for (int item = blockIdx.x; item < P.total_items && alive; item += gridDim.x, ++tile_it) {
         const AccumItem t = accum_decode(P, item);
+        const bool use_ready = !PRE || (P.L[t.l].has_bias && t.nt == 0);
         if (!mbar_wait(&S->tmem_empty, (tile_it & 1u) ^ 1u, abort_flag, P.status, 2, (int)tile_it)) { alive = false; break; }
         tc_fence_after();
         uint32_t acc = 0;
@@ -640,7 +655,13 @@ __global__ void __launch_bounds__(A_THREADS, 1) k_accum(const __grid_constant__ 
           for (int tb = 0; tb < n_tb; ++tb) {
             const uint32_t slot = it % A_STAGES, ph = (it / A_STAGES) & 1u;
             ++it;
-            if (!mbar_wait(&S->ready[slot], ph, abort_flag, P.status, 3, (int)it)) { alive = false; break; }
+            if (use_ready) {
+              const uint32_t rs = rit % A_STAGES, rp = (rit / A_STAGES) & 1u;
+              ++rit;
+              if (!mbar_wait(&S->ready[rs], rp, abort_flag, P.status, 3, (int)it)) { alive = false; break; }
+            } else {
+              if (!mbar_wait(&S->full[slot], ph, abort_flag, P.status, 6, (int)it)) { alive = false; break; }
+            }
             tc_fence_after();
             const uint32_t am = smem_u32(tiles + slot * A_STAGE_BYTES), an = am + A_M_BYTES;
 #pragma unroll
@@ -670,7 +691,7 @@ __global__ void __launch_bounds__(A_THREADS, 1) k_accum(const __grid_constant__ 
     const int h = warp >= 6 ? 1 : 0;                  // which 128-row half of the tile this warp drains
     const int tt = threadIdx.x - 64;                  // 0..255
     const int ta = tt >> 6, kk = (tt & 63) >> 3, jp = tt & 7;   // atom, row & 7, physical 16-byte chunk
-    uint32_t it = 0, tile_it = 0;
+    uint32_t it = 0, rit = 0, tile_it = 0;
     bool alive = true;
     for (int item = blockIdx.x; item < P.total_items; item += gridDim.x, ++tile_it) {
       const AccumItem t = accum_decode(P, item);
@@ -679,8 +700,9 @@ __global__ void __launch_bounds__(A_THREADS, 1) k_accum(const __grid_constant__ 
       float col[8];
 #pragma unroll
       for (int u = 0; u < 8; ++u) col[u] = 0.0f;
-      for (int e = t.e0; e < t.e1; ++e) {
-        const float cf = alive ? __ldg(P.clip + e) : 1.0f;
+      if (PRE && !need_bias) it += (uint32_t)((t.e1 - t.e0) * n_tb);     // nothing to do until the tile is done
+      for (int e = t.e0; e < t.e1 && (!PRE || need_bias); ++e) {
+        const float cf = !alive ? 1.0f : (PRE && L.scaled_g) ? 1.0f : __ldg(P.clip + e);
         // c = c_hi + c_lo in bf16: x*c_hi + x*c_lo keeps the factor to ~2^-17 with two packed instructions
         const __nv_bfloat16 chi = __float2bfloat16_rn(cf);
         const __nv_bfloat162 chi2 = __halves2bfloat162(chi, chi);
@@ -689,9 +711,9 @@ __global__ void __launch_bounds__(A_THREADS, 1) k_accum(const __grid_constant__ 
         for (int tb = 0; tb < n_tb; ++tb) {
           const uint32_t slot = it % A_STAGES, ph = (it / A_STAGES) & 1u;
           ++it;
-          if (alive && !mbar_wait(&S->full[slot], ph, abort_flag, P.status, 4, (int)it)) alive = false;
+          if (alive && !mbar_wait<DP_ACCUM_WORKER_SLEEP_NS>(&S->full[slot], ph, abort_flag, P.status, 4, (int)it)) alive = false;
           if (!alive) continue;
-          if (cf != 1.0f || need_bias) {
+          if (PRE || cf != 1.0f || need_bias) {
             uint8_t* base = tiles + slot * A_STAGE_BYTES + ta * A_ATOM_BYTES + kk * 128 + jp * 16;
 #pragma unroll
             for (int i4 = 0; i4 < 4; ++i4) {          // rows kk, kk+8, kk+16, kk+24 of atom ta
@@ -704,15 +726,18 @@ __global__ void __launch_bounds__(A_THREADS, 1) k_accum(const __grid_constant__ 
                   col[2 * u] = fmaf(__uint_as_float(x[u] << 16), cf, col[2 * u]);
                   col[2 * u + 1] = fmaf(__uint_as_float(x[u] & 0xffff0000u), cf, col[2 * u + 1]);
                 }
-                const __nv_bfloat162 xv = *reinterpret_cast<const __nv_bfloat162*>(&x[u]);
-                const __nv_bfloat162 yv = __hfma2(xv, clo2, __hmul2(xv, chi2));
-                x[u] = *reinterpret_cast<const uint32_t*>(&yv);
+                if (!PRE) {
+                  const __nv_bfloat162 xv = *reinterpret_cast<const __nv_bfloat162*>(&x[u]);
+                  const __nv_bfloat162 yv = __hfma2(xv, clo2, __hmul2(xv, chi2));
+                  x[u] = *reinterpret_cast<const uint32_t*>(&yv);
+                }
               }
-              if (cf != 1.0f) *p = make_uint4(x[0], x[1], x[2], x[3]);
+              if (!PRE && cf != 1.0f) *p = make_uint4(x[0], x[1], x[2], x[3]);
             }
-            fence_proxy_async_smem();
+            if (!PRE) fence_proxy_async_smem();
           }
-          mbar_arrive(&S->ready[slot]);
+          mbar_arrive(&S->ready[rit % A_STAGES]);
+          ++rit;
         }
       }
       if (need_bias) {      // uniform over the 256 threads of warps 2..9; executed even after an abort
@@ -785,7 +810,9 @@ static bool encode_map(CUtensorMap* map, const void* base, int B, int T, int d, 
   const cuuint32_t box[3] = {64u, (cuuint32_t)box_rows, 1u};
   const cuuint32_t estr[3] = {1u, 1u, 1u};
   return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+            DP_TMA_L2_PROMOTION == 0 ? CU_TENSOR_MAP_L2_PROMOTION_NONE
+            : DP_TMA_L2_PROMOTION == 1 ? CU_TENSOR_MAP_L2_PROMOTION_L2_128B : CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
@@ -842,6 +869,8 @@ static bool fill_layer(UmmaLayer& U, const dp_layer& L, int box_rows) {
   U.tiles_n = ceil_div(L.d_in, 256);
   U.has_bias = emb ? 0 : L.has_bias;
   U.is_emb = emb ? 1 : 0;
+  U.scaled_g = 0;
+  U.pad = 0;
   return true;
 }
 
@@ -897,12 +926,51 @@ int launch_umma_sqnorms(const dp_layer* layers, const int* idx, int n, const int
   return DP_OK;
 }
 
+// ---- pre-scaling of one operand per layer: dst[r, :] = bf16(clip[r / T] * src[r, :]) --------------------------
+struct PreTask { const uint4* src; uint4* dst; int vec_per_row, pad; };
+struct PreBatch { PreTask t[kMaxLayers]; int n, rows, T, pad; const float* clip; };
+
+__global__ void __launch_bounds__(256) k_prescale(const __grid_constant__ PreBatch P) {
+  const PreTask& t = P.t[blockIdx.y];
+  const long long total = (long long)P.rows * t.vec_per_row;
+  for (long long v = (long long)blockIdx.x * 256 + threadIdx.x; v < total; v += (long long)gridDim.x * 256) {
+    const int row = (int)(v / t.vec_per_row);
+    const float c = __ldg(P.clip + row / P.T);
+    uint4 w = __ldg(t.src + v);
+    uint32_t x[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const __nv_bfloat162 pk = __floats2bfloat162_rn(__uint_as_float(x[u] << 16) * c,
+                                                      __uint_as_float(x[u] & 0xffff0000u) * c);
+      x[u] = *reinterpret_cast<const uint32_t*>(&pk);
+    }
+    t.dst[v] = make_uint4(x[0], x[1], x[2], x[3]);
+  }
+}
+
+// The operand that carries the clip factor is the narrower one (ties: G, whose scaled tile then also gives the
+// bias column sums without a further multiply).
+static bool prescale_uses_g(const dp_layer& L) { return L.d_out <= L.d_in; }
+
+size_t umma_prescale_bytes(const dp_layer* layers, const int* idx, int n) {
+  size_t b = 0;
+  for (int k = 0; k < n; ++k) {
+    const dp_layer& L = layers[idx[k]];
+    if (L.kind != DP_LINEAR) continue;
+    const size_t cols = prescale_uses_g(L) ? L.d_out : L.d_in;
+    b += align_up((size_t)L.B * L.T * cols * 2, 256);
+  }
+  return b;
+}
+
 int launch_umma_accumulate(const dp_layer* layers, const int* idx, int n, const float* clip, int* status,
-                           cudaStream_t s) {
+                           cudaStream_t s, void* prescale_buf) {
   if (n <= 0) return DP_OK;
   const int B = layers[idx[0]].B, T = layers[idx[0]].T;
-  static bool attr_ok = ensure_smem(k_accum, A_SMEM);
+  static bool attr_ok = ensure_smem(k_accum<false>, A_SMEM) && ensure_smem(k_accum<true>, A_SMEM);
   if (!attr_ok) return DP_ERR_CUDA;
+  const bool pre = prescale_buf != nullptr;
+  size_t pre_off = 0;
   const int sms = sm_count();
   for (int k0 = 0; k0 < n; k0 += kMaxLayers) {
     const int nl = (n - k0) < kMaxLayers ? (n - k0) : kMaxLayers;
@@ -921,11 +989,30 @@ int launch_umma_accumulate(const dp_layer* layers, const int* idx, int n, const 
       }
     }
     UmmaParams P;
+    PreBatch Q;
+    Q.n = nl;
+    Q.rows = B * T;
+    Q.T = T;
+    Q.pad = 0;
+    Q.clip = clip;
     long long items = 0;
     for (int k = 0; k < nl; ++k) {
-      const dp_layer& L = layers[idx[k0 + k]];
+      dp_layer L = layers[idx[k0 + k]];
       UmmaLayer& U = P.L[k];
+      int scaled_g = 0;
+      if (pre) {      // point the scaled operand at its copy in the workspace
+        scaled_g = prescale_uses_g(L) ? 1 : 0;
+        const int cols = scaled_g ? L.d_out : L.d_in;
+        void* dst = static_cast<char*>(prescale_buf) + pre_off;
+        pre_off += align_up((size_t)B * T * cols * 2, 256);
+        Q.t[k].src = static_cast<const uint4*>(scaled_g ? L.G : L.A);
+        Q.t[k].dst = static_cast<uint4*>(dst);
+        Q.t[k].vec_per_row = cols / 8;
+        Q.t[k].pad = 0;
+        if (scaled_g) L.G = dst; else L.A = dst;
+      }
       if (!fill_layer(U, L, T < A_BK ? T : A_BK)) return DP_ERR_CUDA;
+      U.scaled_g = scaled_g;
       U.tiles_m = ceil_div(L.d_out, 256);
       U.item_start = (int)items;
       U.partial_base = 0;
@@ -943,7 +1030,13 @@ int launch_umma_accumulate(const dp_layer* layers, const int* idx, int n, const 
     P.partial = nullptr;
     P.status = status;
     const int grid = P.total_items < sms ? P.total_items : sms;
-    k_accum<<<grid, A_THREADS, A_SMEM, s>>>(P);
+    if (pre) {
+      k_prescale<<<dim3(2 * sms, nl), 256, 0, s>>>(Q);
+      if (counted(1) != cudaSuccess) return DP_ERR_CUDA;
+      k_accum<true><<<grid, A_THREADS, A_SMEM, s>>>(P);
+    } else {
+      k_accum<false><<<grid, A_THREADS, A_SMEM, s>>>(P);
+    }
     if (counted(1) != cudaSuccess) return DP_ERR_CUDA;
   }
   return DP_OK;
