@@ -31,7 +31,7 @@ if ROOT not in sys.path:
 
 # DRAM bytes (read + write) of one k_accum launch over the 24-block stack, from the ncu capture summarised in
 # profiles/k_accum_2blocks_full.md (2-block case x 12).  Set to None whenever that kernel changes.
-ACCUM_TRAFFIC_BYTES = 40.7e9
+ACCUM_TRAFFIC_BYTES = None
 
 METRIC = "dp_sgd_examples_per_s_bert_large"
 UNIT = "examples/s"

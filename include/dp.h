@@ -79,14 +79,10 @@ typedef struct dp_layer {
   float* acc_b;      /* LINEAR with bias: [d_out].  LAYERNORM: bias [d].  Otherwise NULL */
 } dp_layer;
 
-/* Bytes of scratch for dp_per_example_sqnorms / dp_clipped_accumulate over these layers.
- *   dp_workspace_bytes      the recommended size: it includes room for clip-scaled bf16 copies of one operand per
- *                           tensor-core linear layer (B*T*min(d_in,d_out)*2 bytes each), which lets the accumulate
- *                           GEMM stream its operands without touching them in shared memory;
- *   dp_workspace_bytes_min  the least the calls accept; with less than the recommended size the GEMM scales its
- *                           tiles in shared memory instead (same results up to bf16 rounding, slower). */
+/* Bytes of scratch that dp_per_example_sqnorms / dp_clipped_accumulate need over these layers (per-example
+ * column sums of the LayerNorm / bias terms and the partial sums of the tensor-core norm kernels); 0 on invalid
+ * layers.  The two calls plan the same layout, so one buffer serves both. */
 DP_API size_t dp_workspace_bytes(const dp_layer* layers /*HOST*/, int n_layers);
-DP_API size_t dp_workspace_bytes_min(const dp_layer* layers /*HOST*/, int n_layers);
 
 /* Squared L2 norm of every example's whole gradient over the given layers (Algorithm 1 clips
  * grad L(theta; x_j) as one vector; Section 4.3 gives the per-layer form).

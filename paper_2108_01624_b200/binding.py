@@ -22,7 +22,7 @@ DP_F32, DP_BF16 = 0, 1
 DP_PATH_AUTO, DP_PATH_GRAM, DP_PATH_MATERIALIZED = 0, 1, 2
 _KINDS = {"linear": DP_LINEAR, "layernorm": DP_LAYERNORM, "embedding": DP_EMBEDDING}
 
-EXPORTS = ["dp_workspace_bytes", "dp_workspace_bytes_min", "dp_per_example_sqnorms", "dp_clip_factors", "dp_clipped_accumulate",
+EXPORTS = ["dp_workspace_bytes", "dp_per_example_sqnorms", "dp_clip_factors", "dp_clipped_accumulate",
            "dp_add_noise_and_scale", "dp_adamw_step", "dp_noise_scale_adamw_step", "dp_noise_scale_adamw_step_snr",
            "dp_clip_stats", "dp_philox_u32",
            "dp_token_equality_mask", "dp_layernorm_sqnorms_static", "dp_poll_status", "dp_last_timeout_info", "dp_launch_count",
@@ -56,8 +56,6 @@ def lib() -> C.CDLL:
         vp, i32, i64, u64, f32, sz = C.c_void_p, C.c_int, C.c_int64, C.c_uint64, C.c_double, C.c_size_t
         L.dp_workspace_bytes.restype = sz
         L.dp_workspace_bytes.argtypes = [vp, i32]
-        L.dp_workspace_bytes_min.restype = sz
-        L.dp_workspace_bytes_min.argtypes = [vp, i32]
         L.dp_per_example_sqnorms.argtypes = [vp, i32, vp, i32, vp, sz, vp]
         L.dp_clip_factors.argtypes = [vp, i32, f32, vp, vp]
         L.dp_clipped_accumulate.argtypes = [vp, i32, vp, vp, sz, vp]
@@ -170,13 +168,9 @@ def dp_workspace_bytes(layers: LayerList) -> int:
     return int(lib().dp_workspace_bytes(layers.ptr, len(layers)))
 
 
-def dp_workspace_bytes_min(layers: LayerList) -> int:
-    return int(lib().dp_workspace_bytes_min(layers.ptr, len(layers)))
-
-
-def alloc_workspace(layers: LayerList, minimal: bool = False) -> Optional[torch.Tensor]:
+def alloc_workspace(layers: LayerList) -> Optional[torch.Tensor]:
     """Caller-owned scratch for the two layer-list calls (torch's allocator aligns to 512 bytes)."""
-    n = dp_workspace_bytes_min(layers) if minimal else dp_workspace_bytes(layers)
+    n = dp_workspace_bytes(layers)
     dev = layers.layers[0].G.device
     return torch.empty(max(n, 256), dtype=torch.uint8, device=dev)
 

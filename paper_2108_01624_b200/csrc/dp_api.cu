@@ -77,9 +77,7 @@ struct WsPlan {
   std::vector<int> umma_gram;  // 1: Gram path, 0: materialised tiles
   std::vector<size_t> col_off; // per layer: byte offset of its column-sum block (or SIZE_MAX if it has none)
   std::vector<int> lin_idx;    // tensor-core layers that are linear (the accumulate GEMM takes only these)
-  size_t prescale_bytes = 0;   // optional third block: clip-scaled copies of one operand per linear layer
-  size_t min_total() const { return align_up(colsum_bytes, 256) + align_up(partial_bytes, 256); }
-  size_t total() const { return min_total() + align_up(prescale_bytes, 256); }
+  size_t total() const { return align_up(colsum_bytes, 256) + align_up(partial_bytes, 256); }
 };
 
 static WsPlan plan_workspace(const dp_layer* layers, int n_layers) {
@@ -110,14 +108,12 @@ static WsPlan plan_workspace(const dp_layer* layers, int n_layers) {
   }
   for (int l : p.umma_idx)
     if (layers[l].kind == DP_LINEAR) p.lin_idx.push_back(l);
-  if (!p.lin_idx.empty()) p.prescale_bytes = umma_prescale_bytes(layers, p.lin_idx.data(), (int)p.lin_idx.size());
   return p;
 }
 
-// The first two blocks are required; the third (pre-scaled operands) is used when the workspace has room for it.
 static int check_ws(const WsPlan& p, void* ws, size_t bytes) {
-  if (p.min_total() == 0) return DP_OK;
-  if (!ws || misaligned(ws, 256) || bytes < p.min_total()) return DP_ERR_WORKSPACE;
+  if (p.total() == 0) return DP_OK;
+  if (!ws || misaligned(ws, 256) || bytes < p.total()) return DP_ERR_WORKSPACE;
   return DP_OK;
 }
 
@@ -134,10 +130,6 @@ size_t dp_workspace_bytes(const dp_layer* layers, int n_layers) {
   return plan_workspace(layers, n_layers).total();
 }
 
-size_t dp_workspace_bytes_min(const dp_layer* layers, int n_layers) {
-  if (validate_layers(layers, n_layers, false) != DP_OK) return 0;
-  return plan_workspace(layers, n_layers).min_total();
-}
 
 int dp_per_example_sqnorms(const dp_layer* layers, int n_layers, float* sqnorm, int accumulate_into,
                            void* workspace, size_t workspace_bytes, void* cuda_stream) {
@@ -210,13 +202,7 @@ int dp_clipped_accumulate(const dp_layer* layers, int n_layers, const float* cli
   int* status = status_ptr();
   if (!status) return DP_ERR_CUDA;
   if (!plan.lin_idx.empty()) {
-    // With room for them, one operand per layer is multiplied by the clip factors into the workspace first and
-    // the GEMM streams the copies (faster: nothing passes through shared memory twice); otherwise the GEMM
-    // scales its G tiles in shared memory.
-    void* pre = nullptr;
-    if (plan.prescale_bytes > 0 && workspace && workspace_bytes >= plan.total())
-      pre = static_cast<char*>(workspace) + plan.min_total();
-    rc = launch_umma_accumulate(layers, plan.lin_idx.data(), (int)plan.lin_idx.size(), clip, status, s, pre);
+    rc = launch_umma_accumulate(layers, plan.lin_idx.data(), (int)plan.lin_idx.size(), clip, status, s);
     if (rc != DP_OK) return rc;
   }
   std::vector<ColTaskHost> tasks;

@@ -73,10 +73,8 @@ bool umma_accumulates_bias();
 size_t umma_sqnorm_partials_per_example(const dp_layer* layers, const int* idx, int n, const int* use_gram);
 int launch_umma_sqnorms(const dp_layer* layers, const int* idx, int n, const int* use_gram, float* partial,
                         int partial_stride, int partial_base, int* status, cudaStream_t s);
-// prescale_buf (optional, umma_prescale_bytes bytes): when given, the narrower operand of every layer is first
-// multiplied by the clip factors into it and the GEMM streams the copies; otherwise the scaling happens in-kernel.
-size_t umma_prescale_bytes(const dp_layer* layers, const int* idx, int n);
+// acc_w (and acc_b) += sum_i clip[i] * A_i^T G_i; the clip factor is applied to the G tile inside the kernel.
 int launch_umma_accumulate(const dp_layer* layers, const int* idx, int n, const float* clip, int* status,
-                           cudaStream_t s, void* prescale_buf);
+                           cudaStream_t s);
 
 }  // namespace dpk

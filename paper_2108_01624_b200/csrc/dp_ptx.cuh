@@ -55,7 +55,9 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
   return ok != 0;
 }
 
-constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s: far beyond any legitimate wait here
+// Wait limit in SM clock cycles (clock64 is cheap to read; %globaltimer is not and would sit on the critical
+// path of every wait that does not succeed at once): 4e9 cycles = 2 to 3 s at 1.3 to 2 GHz.
+constexpr long long kWaitLimitCycles = 4000000000ll;
 constexpr int kStatusTimeout = 1;
 
 // Waits for the phase with the given parity.  Returns false if the limit ran out or another thread
@@ -68,13 +70,13 @@ template <int SLEEP_NS = 0>
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status,
                                           int tag = 0, int aux = 0) {
   if (mbar_try_wait(bar, parity)) return true;
-  const unsigned long long t0 = globaltimer_ns();
+  const long long t0 = clock64();
   for (uint32_t spin = 1;; ++spin) {
     if (SLEEP_NS > 0) __nanosleep(SLEEP_NS);
     if (mbar_try_wait(bar, parity)) return true;
     if ((spin & 63u) == 0u) {
       if (*abort_flag) return false;
-      if (globaltimer_ns() - t0 > kWaitLimitNs) {
+      if (clock64() - t0 > kWaitLimitCycles) {
         if (atomicCAS(status, 0, kStatusTimeout) == 0) {
           status[1] = tag;
           status[2] = (int)blockIdx.x;
@@ -92,10 +94,10 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
 // Same, but for the final drain of a role's own in-flight work: ignores the abort flag, keeps the limit.
 __device__ __forceinline__ bool mbar_wait_drain(uint64_t* bar, uint32_t parity, int* status) {
   if (mbar_try_wait(bar, parity)) return true;
-  const unsigned long long t0 = globaltimer_ns();
+  const long long t0 = clock64();
   for (uint32_t spin = 1;; ++spin) {
     if (mbar_try_wait(bar, parity)) return true;
-    if ((spin & 63u) == 0u && globaltimer_ns() - t0 > kWaitLimitNs) {
+    if ((spin & 63u) == 0u && clock64() - t0 > kWaitLimitCycles) {
       atomicCAS(status, 0, kStatusTimeout);
       return false;
     }
@@ -113,6 +115,16 @@ __device__ __forceinline__ void tma_load_3d(void* smem_dst, const CUtensorMap* m
   asm volatile(
       "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
       ::"r"(smem_u32(smem_dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(smem_u32(bar)), "r"(x), "r"(y), "r"(z)
+      : "memory");
+}
+
+// 4-D variant.  The kernels view a [B, T, d] tensor as (x = 64 features, y = token, a = 64-feature group, z = example)
+// so that ONE copy brings several 64-feature groups of a token block: the cost of a tensor copy on the SM is per
+// instruction (about 130 cycles for a 3-D box, about 300 for a 4-D one, whatever its size), not per byte.
+__device__ __forceinline__ void tma_load_4d(void* smem_dst, const CUtensorMap* map, uint64_t* bar, int x, int y, int a, int z) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+      ::"r"(smem_u32(smem_dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(smem_u32(bar)), "r"(x), "r"(y), "r"(a), "r"(z)
       : "memory");
 }
 

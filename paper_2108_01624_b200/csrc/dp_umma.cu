@@ -47,7 +47,7 @@ struct alignas(64) UmmaLayer {
   int item_start;         // first work item of this layer within the launch
   int partial_base;       // first per-example partial slot of this layer
   int has_bias, is_emb;
-  int scaled_g, pad;      // accumulate with pre-scaled operands: 1 if G is the operand that carries the clip factor
+  int pad[2];
 };
 
 struct UmmaParams {
@@ -55,7 +55,8 @@ struct UmmaParams {
   int n_layers, total_items, B, T;
   int box_rows;           // token rows per TMA box (min(tile rows, T))
   int splits;             // accumulate: number of example ranges a tile is split into
-  int partial_stride, pad;
+  int partial_stride;
+  int wide_boxes;         // tile kernels: 1 = 4-D maps, one copy per operand and stage; 0 = 3-D maps, one copy per 64 features
   const float* clip;
   float* partial;
   int* status;
@@ -348,11 +349,14 @@ __global__ void __launch_bounds__(ACCUM ? 320 : 192, 1) k_tile(const __grid_cons
             if (!mbar_wait(&S->empty[slot], ph ^ 1u, abort_flag, P.status)) { alive = false; break; }
             uint8_t* st = tiles + slot * T_STAGE_BYTES;
             mbar_arrive_expect_tx(&S->full[slot], 6u * box_bytes);
-#pragma unroll
-            for (int a = 0; a < 2; ++a) tma_load_3d(st + a * T_ATOM_BYTES, &L.mapG, &S->full[slot], t.m0 + a * 64, tb * 64, e);
-#pragma unroll
-            for (int a = 0; a < 4; ++a)
-              tma_load_3d(st + T_M_BYTES + a * T_ATOM_BYTES, &L.mapA, &S->full[slot], t.n0 + a * 64, tb * 64, e);
+            if (P.wide_boxes) {
+              tma_load_4d(st, &L.mapG, &S->full[slot], 0, tb * 64, t.m0 / 64, e);               // 2 groups of 64 features
+              tma_load_4d(st + T_M_BYTES, &L.mapA, &S->full[slot], 0, tb * 64, t.n0 / 64, e);    // 4 groups
+            } else {
+              for (int a = 0; a < 2; ++a) tma_load_3d(st + a * T_ATOM_BYTES, &L.mapG, &S->full[slot], t.m0 + a * 64, tb * 64, e);
+              for (int a = 0; a < 4; ++a)
+                tma_load_3d(st + T_M_BYTES + a * T_ATOM_BYTES, &L.mapA, &S->full[slot], t.n0 + a * 64, tb * 64, e);
+            }
             ++it;
           }
         }
@@ -513,20 +517,25 @@ __global__ void __launch_bounds__(ACCUM ? 320 : 192, 1) k_tile(const __grid_cons
 }
 
 // =================================================================================================
-// Clipped-accumulate kernel: 256 (d_out) x 256 (d_in) output tiles, K = tokens, 32 tokens per stage.
+// Clipped-accumulate kernel: 256 (d_out) x 256 (d_in) output tiles, K = tokens, 64 tokens per stage.
 // Two 128x256x16 UMMAs (the two 128-row halves of the G tile) share each 256-wide A tile, so a stage of
-// 32 KB feeds 512 tensor-pipe cycles and a 6-stage ring covers the L2/HBM latency.  The whole 512-column
+// 64 KB feeds 1024 tensor-pipe cycles and a 3-stage ring covers the L2/HBM latency.  The whole 512-column
 // TMEM holds the one fp32 accumulator; at the end of a tile all eight non-producer warps drain it.
-// What bounds the kernel is the shared-memory data pipe (one 128-byte wavefront per cycle, shared by TMA
-// writes, UMMA operand reads and ld/st.shared): per stage 384 operand + 256 TMA wavefronts, plus up to 256
-// for scaling the G tile in place (skipped for examples whose clip factor is 1).
+// A TMA copy costs the SM a fixed issue time per instruction, whatever its size, and the copies of one lane
+// are serial: a stage therefore arrives as two 4-D boxes (64 features x 64 tokens x four 64-feature groups,
+// one for G and one for A) instead of eight 3-D ones, which is what keeps the producer ahead of the UMMAs.
+// The clip factor is applied to the G tile in shared memory by the eight worker warps, hidden behind the
+// UMMAs of the previous stage (skipped for examples whose factor is 1).
 // =================================================================================================
-constexpr int A_STAGES = 6;
-constexpr int A_BK = 32;
-constexpr int A_ATOM_BYTES = A_BK * 128;                // 32 tokens x 64 bf16 features
+#ifndef DP_ACCUM_BK
+#define DP_ACCUM_BK 64
+#endif
+constexpr int A_BK = DP_ACCUM_BK;                       // tokens per stage (32 or 64)
+constexpr int A_STAGES = 192 / A_BK;                    // 192 KB of operand ring: 3 stages of 64 KB (or 6 of 32 KB)
+constexpr int A_ATOM_BYTES = A_BK * 128;                // A_BK tokens x 64 bf16 features
 constexpr int A_M_BYTES = 4 * A_ATOM_BYTES;             // G tile: 256 features of d_out
 constexpr int A_N_BYTES = 4 * A_ATOM_BYTES;             // A tile: 256 features of d_in
-constexpr int A_STAGE_BYTES = A_M_BYTES + A_N_BYTES;    // 32 KB
+constexpr int A_STAGE_BYTES = A_M_BYTES + A_N_BYTES;
 constexpr int A_THREADS = 320;
 
 struct AccumCtl {
@@ -573,11 +582,6 @@ __device__ __forceinline__ void accum_store_chunk(const UmmaLayer& L, int m, int
   }
 }
 
-// PRE = false: the clip factor is applied to the G tile in shared memory by the worker warps (needs no scratch).
-// PRE = true : one operand of every layer was multiplied by the clip factors beforehand (k_prescale, a copy in
-//              the caller's workspace), so the tiles go from TMA straight to the UMMAs; the worker warps only
-//              read the G tile of the tiles that own a bias slice (column sums), and otherwise just drain.
-template <bool PRE>
 __global__ void __launch_bounds__(A_THREADS, 1) k_accum(const __grid_constant__ UmmaParams P) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* tiles = align1024(smem_raw);
@@ -625,12 +629,15 @@ __global__ void __launch_bounds__(A_THREADS, 1) k_accum(const __grid_constant__ 
             if (!mbar_wait<DP_ACCUM_WORKER_SLEEP_NS>(&S->empty[slot], ph ^ 1u, abort_flag, P.status, 1, (int)it)) { alive = false; break; }
             uint8_t* st = tiles + slot * A_STAGE_BYTES;
             mbar_arrive_expect_tx(&S->full[slot], 8u * box_bytes);
-#pragma unroll
-            for (int a = 0; a < 4; ++a)
-              tma_load_3d(st + a * A_ATOM_BYTES, &L.mapG, &S->full[slot], t.m0 + a * 64, tb * A_BK, e);
-#pragma unroll
-            for (int a = 0; a < 4; ++a)
-              tma_load_3d(st + A_M_BYTES + a * A_ATOM_BYTES, &L.mapA, &S->full[slot], t.n0 + a * 64, tb * A_BK, e);
+            if (P.wide_boxes) {
+              tma_load_4d(st, &L.mapG, &S->full[slot], 0, tb * A_BK, t.m0 / 64, e);              // 4 groups of 64 features
+              tma_load_4d(st + A_M_BYTES, &L.mapA, &S->full[slot], 0, tb * A_BK, t.n0 / 64, e);
+            } else {
+              for (int a = 0; a < 4; ++a)
+                tma_load_3d(st + a * A_ATOM_BYTES, &L.mapG, &S->full[slot], t.m0 + a * 64, tb * A_BK, e);
+              for (int a = 0; a < 4; ++a)
+                tma_load_3d(st + A_M_BYTES + a * A_ATOM_BYTES, &L.mapA, &S->full[slot], t.n0 + a * 64, tb * A_BK, e);
+            }
             ++it;
           }
         }
@@ -643,11 +650,10 @@ __global__ void __launch_bounds__(A_THREADS, 1) k_accum(const __grid_constant__ 
     }
   } else if (warp == 1) {
     if (lane == 0) {   // ---------------- MMA issuer ----------------
-      uint32_t it = 0, rit = 0, tile_it = 0;     // rit counts the stages that go through the `ready` barriers
+      uint32_t it = 0, tile_it = 0;
       bool alive = true;
       for (int item = blockIdx.x; item < P.total_items && alive; item += gridDim.x, ++tile_it) {
         const AccumItem t = accum_decode(P, item);
-        const bool use_ready = !PRE || (P.L[t.l].has_bias && t.nt == 0);
         if (!mbar_wait(&S->tmem_empty, (tile_it & 1u) ^ 1u, abort_flag, P.status, 2, (int)tile_it)) { alive = false; break; }
         tc_fence_after();
         uint32_t acc = 0;
@@ -655,17 +661,11 @@ __global__ void __launch_bounds__(A_THREADS, 1) k_accum(const __grid_constant__ 
           for (int tb = 0; tb < n_tb; ++tb) {
             const uint32_t slot = it % A_STAGES, ph = (it / A_STAGES) & 1u;
             ++it;
-            if (use_ready) {
-              const uint32_t rs = rit % A_STAGES, rp = (rit / A_STAGES) & 1u;
-              ++rit;
-              if (!mbar_wait(&S->ready[rs], rp, abort_flag, P.status, 3, (int)it)) { alive = false; break; }
-            } else {
-              if (!mbar_wait(&S->full[slot], ph, abort_flag, P.status, 6, (int)it)) { alive = false; break; }
-            }
+            if (!mbar_wait(&S->ready[slot], ph, abort_flag, P.status, 3, (int)it)) { alive = false; break; }
             tc_fence_after();
             const uint32_t am = smem_u32(tiles + slot * A_STAGE_BYTES), an = am + A_M_BYTES;
 #pragma unroll
-            for (int k2 = 0; k2 < 2; ++k2) {
+            for (int k2 = 0; k2 < A_BK / 16; ++k2) {
               const uint64_t bdesc = smem_desc_sw128(an + k2 * 2048, A_ATOM_BYTES, 1024);
 #pragma unroll
               for (int h = 0; h < 2; ++h) {
@@ -691,7 +691,7 @@ __global__ void __launch_bounds__(A_THREADS, 1) k_accum(const __grid_constant__ 
     const int h = warp >= 6 ? 1 : 0;                  // which 128-row half of the tile this warp drains
     const int tt = threadIdx.x - 64;                  // 0..255
     const int ta = tt >> 6, kk = (tt & 63) >> 3, jp = tt & 7;   // atom, row & 7, physical 16-byte chunk
-    uint32_t it = 0, rit = 0, tile_it = 0;
+    uint32_t it = 0, tile_it = 0;
     bool alive = true;
     for (int item = blockIdx.x; item < P.total_items; item += gridDim.x, ++tile_it) {
       const AccumItem t = accum_decode(P, item);
@@ -700,9 +700,8 @@ __global__ void __launch_bounds__(A_THREADS, 1) k_accum(const __grid_constant__ 
       float col[8];
 #pragma unroll
       for (int u = 0; u < 8; ++u) col[u] = 0.0f;
-      if (PRE && !need_bias) it += (uint32_t)((t.e1 - t.e0) * n_tb);     // nothing to do until the tile is done
-      for (int e = t.e0; e < t.e1 && (!PRE || need_bias); ++e) {
-        const float cf = !alive ? 1.0f : (PRE && L.scaled_g) ? 1.0f : __ldg(P.clip + e);
+      for (int e = t.e0; e < t.e1; ++e) {
+        const float cf = alive ? __ldg(P.clip + e) : 1.0f;
         // c = c_hi + c_lo in bf16: x*c_hi + x*c_lo keeps the factor to ~2^-17 with two packed instructions
         const __nv_bfloat16 chi = __float2bfloat16_rn(cf);
         const __nv_bfloat162 chi2 = __halves2bfloat162(chi, chi);
@@ -713,10 +712,10 @@ __global__ void __launch_bounds__(A_THREADS, 1) k_accum(const __grid_constant__ 
           ++it;
           if (alive && !mbar_wait<DP_ACCUM_WORKER_SLEEP_NS>(&S->full[slot], ph, abort_flag, P.status, 4, (int)it)) alive = false;
           if (!alive) continue;
-          if (PRE || cf != 1.0f || need_bias) {
+          if (cf != 1.0f || need_bias) {
             uint8_t* base = tiles + slot * A_STAGE_BYTES + ta * A_ATOM_BYTES + kk * 128 + jp * 16;
 #pragma unroll
-            for (int i4 = 0; i4 < 4; ++i4) {          // rows kk, kk+8, kk+16, kk+24 of atom ta
+            for (int i4 = 0; i4 < A_BK / 8; ++i4) {   // rows kk, kk+8, ... of atom ta
               uint4* p = reinterpret_cast<uint4*>(base + i4 * 1024);
               uint4 w = *p;
               uint32_t x[4] = {w.x, w.y, w.z, w.w};
@@ -726,18 +725,15 @@ __global__ void __launch_bounds__(A_THREADS, 1) k_accum(const __grid_constant__ 
                   col[2 * u] = fmaf(__uint_as_float(x[u] << 16), cf, col[2 * u]);
                   col[2 * u + 1] = fmaf(__uint_as_float(x[u] & 0xffff0000u), cf, col[2 * u + 1]);
                 }
-                if (!PRE) {
-                  const __nv_bfloat162 xv = *reinterpret_cast<const __nv_bfloat162*>(&x[u]);
-                  const __nv_bfloat162 yv = __hfma2(xv, clo2, __hmul2(xv, chi2));
-                  x[u] = *reinterpret_cast<const uint32_t*>(&yv);
-                }
+                const __nv_bfloat162 xv = *reinterpret_cast<const __nv_bfloat162*>(&x[u]);
+                const __nv_bfloat162 yv = __hfma2(xv, clo2, __hmul2(xv, chi2));
+                x[u] = *reinterpret_cast<const uint32_t*>(&yv);
               }
-              if (!PRE && cf != 1.0f) *p = make_uint4(x[0], x[1], x[2], x[3]);
+              if (cf != 1.0f) *p = make_uint4(x[0], x[1], x[2], x[3]);
             }
-            if (!PRE) fence_proxy_async_smem();
+            fence_proxy_async_smem();
           }
-          mbar_arrive(&S->ready[rit % A_STAGES]);
-          ++rit;
+          mbar_arrive(&S->ready[slot]);
         }
       }
       if (need_bias) {      // uniform over the 256 threads of warps 2..9; executed even after an abort
@@ -816,6 +812,21 @@ static bool encode_map(CUtensorMap* map, const void* base, int B, int T, int d, 
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// The same tensor as (x = 64 features, y = token, a = 64-feature group, z = example); box = 64 x box_rows x groups x 1.
+static bool encode_map4(CUtensorMap* map, const void* base, int B, int T, int d, int box_rows, int groups) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[4] = {64u, (cuuint64_t)T, (cuuint64_t)(d / 64), (cuuint64_t)B};
+  const cuuint64_t strides[3] = {(cuuint64_t)d * 2, 128u, (cuuint64_t)T * d * 2};
+  const cuuint32_t box[4] = {64u, (cuuint32_t)box_rows, (cuuint32_t)groups, 1u};
+  const cuuint32_t estr[4] = {1u, 1u, 1u, 1u};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+            DP_TMA_L2_PROMOTION == 0 ? CU_TENSOR_MAP_L2_PROMOTION_NONE
+            : DP_TMA_L2_PROMOTION == 1 ? CU_TENSOR_MAP_L2_PROMOTION_L2_128B : CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 bool umma_supported(const dp_layer& L) {
   if (L.kind == DP_EMBEDDING) {   // mask-Gram norm only (the accumulate is a scatter, not a contraction)
     return L.dtype == DP_BF16 && L.d_out % 64 == 0 && (reinterpret_cast<uintptr_t>(L.G) & 15u) == 0 &&
@@ -855,11 +866,17 @@ static bool ensure_smem(K kernel, int bytes) {
   return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) == cudaSuccess;
 }
 
-static bool fill_layer(UmmaLayer& U, const dp_layer& L, int box_rows) {
+// groups_g / groups_a > 0: 4-D maps whose box spans that many 64-feature groups (tile kernels); 0: 3-D maps (Gram).
+static bool fill_layer(UmmaLayer& U, const dp_layer& L, int box_rows, int groups_g = 0, int groups_a = 0) {
   const bool emb = L.kind == DP_EMBEDDING;
-  if (!encode_map(&U.mapG, L.G, L.B, L.T, L.d_out, box_rows)) return false;
-  if (emb) U.mapA = U.mapG;      // never used: an embedding streams no A operand (d_in = 0 below)
-  else if (!encode_map(&U.mapA, L.A, L.B, L.T, L.d_in, box_rows)) return false;
+  if (groups_g > 0) {
+    if (!encode_map4(&U.mapG, L.G, L.B, L.T, L.d_out, box_rows, groups_g)) return false;
+    if (!encode_map4(&U.mapA, L.A, L.B, L.T, L.d_in, box_rows, groups_a)) return false;
+  } else {
+    if (!encode_map(&U.mapG, L.G, L.B, L.T, L.d_out, box_rows)) return false;
+    if (emb) U.mapA = U.mapG;      // never used: an embedding streams no A operand (d_in = 0 below)
+    else if (!encode_map(&U.mapA, L.A, L.B, L.T, L.d_in, box_rows)) return false;
+  }
   U.acc_w = L.acc_w;
   U.acc_b = L.acc_b;
   U.ids = emb ? L.ids : nullptr;
@@ -869,8 +886,7 @@ static bool fill_layer(UmmaLayer& U, const dp_layer& L, int box_rows) {
   U.tiles_n = ceil_div(L.d_in, 256);
   U.has_bias = emb ? 0 : L.has_bias;
   U.is_emb = emb ? 1 : 0;
-  U.scaled_g = 0;
-  U.pad = 0;
+  U.pad[0] = U.pad[1] = 0;
   return true;
 }
 
@@ -900,7 +916,8 @@ int launch_umma_sqnorms(const dp_layer* layers, const int* idx, int n, const int
         const long long add = (long long)B * (gram ? gram_pairs(T) : tile_count(L));
         if (items + add > 0x7fffffffll) break;
         UmmaLayer& U = P.L[P.n_layers];
-        if (!fill_layer(U, L, gram ? (T < 128 ? T : 128) : (T < 64 ? T : 64))) return DP_ERR_CUDA;
+        if (!(gram ? fill_layer(U, L, T < 128 ? T : 128)
+                   : (T >= 64 ? fill_layer(U, L, 64, 2, 4) : fill_layer(U, L, T)))) return DP_ERR_CUDA;
         U.item_start = (int)items;
         U.partial_base = base[k];
         items += add;
@@ -912,9 +929,9 @@ int launch_umma_sqnorms(const dp_layer* layers, const int* idx, int n, const int
       P.T = T;
       P.box_rows = gram ? (T < 128 ? T : 128) : (T < 64 ? T : 64);
       P.splits = 1;
+      P.wide_boxes = (!gram && T >= 64) ? 1 : 0;
       P.partial_stride = partial_stride;
-      P.pad = 0;
-      P.clip = nullptr;
+        P.clip = nullptr;
       P.partial = partial;
       P.status = status;
       const int grid = P.total_items < sm_count() ? P.total_items : sm_count();
@@ -926,51 +943,13 @@ int launch_umma_sqnorms(const dp_layer* layers, const int* idx, int n, const int
   return DP_OK;
 }
 
-// ---- pre-scaling of one operand per layer: dst[r, :] = bf16(clip[r / T] * src[r, :]) --------------------------
-struct PreTask { const uint4* src; uint4* dst; int vec_per_row, pad; };
-struct PreBatch { PreTask t[kMaxLayers]; int n, rows, T, pad; const float* clip; };
-
-__global__ void __launch_bounds__(256) k_prescale(const __grid_constant__ PreBatch P) {
-  const PreTask& t = P.t[blockIdx.y];
-  const long long total = (long long)P.rows * t.vec_per_row;
-  for (long long v = (long long)blockIdx.x * 256 + threadIdx.x; v < total; v += (long long)gridDim.x * 256) {
-    const int row = (int)(v / t.vec_per_row);
-    const float c = __ldg(P.clip + row / P.T);
-    uint4 w = __ldg(t.src + v);
-    uint32_t x[4] = {w.x, w.y, w.z, w.w};
-#pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      const __nv_bfloat162 pk = __floats2bfloat162_rn(__uint_as_float(x[u] << 16) * c,
-                                                      __uint_as_float(x[u] & 0xffff0000u) * c);
-      x[u] = *reinterpret_cast<const uint32_t*>(&pk);
-    }
-    t.dst[v] = make_uint4(x[0], x[1], x[2], x[3]);
-  }
-}
-
-// The operand that carries the clip factor is the narrower one (ties: G, whose scaled tile then also gives the
-// bias column sums without a further multiply).
-static bool prescale_uses_g(const dp_layer& L) { return L.d_out <= L.d_in; }
-
-size_t umma_prescale_bytes(const dp_layer* layers, const int* idx, int n) {
-  size_t b = 0;
-  for (int k = 0; k < n; ++k) {
-    const dp_layer& L = layers[idx[k]];
-    if (L.kind != DP_LINEAR) continue;
-    const size_t cols = prescale_uses_g(L) ? L.d_out : L.d_in;
-    b += align_up((size_t)L.B * L.T * cols * 2, 256);
-  }
-  return b;
-}
-
 int launch_umma_accumulate(const dp_layer* layers, const int* idx, int n, const float* clip, int* status,
-                           cudaStream_t s, void* prescale_buf) {
+                           cudaStream_t s) {
   if (n <= 0) return DP_OK;
   const int B = layers[idx[0]].B, T = layers[idx[0]].T;
-  static bool attr_ok = ensure_smem(k_accum<false>, A_SMEM) && ensure_smem(k_accum<true>, A_SMEM);
+  static bool attr_ok = ensure_smem(k_accum, A_SMEM);
   if (!attr_ok) return DP_ERR_CUDA;
-  const bool pre = prescale_buf != nullptr;
-  size_t pre_off = 0;
+  const int bk = A_BK;
   const int sms = sm_count();
   for (int k0 = 0; k0 < n; k0 += kMaxLayers) {
     const int nl = (n - k0) < kMaxLayers ? (n - k0) : kMaxLayers;
@@ -989,30 +968,11 @@ int launch_umma_accumulate(const dp_layer* layers, const int* idx, int n, const 
       }
     }
     UmmaParams P;
-    PreBatch Q;
-    Q.n = nl;
-    Q.rows = B * T;
-    Q.T = T;
-    Q.pad = 0;
-    Q.clip = clip;
     long long items = 0;
     for (int k = 0; k < nl; ++k) {
-      dp_layer L = layers[idx[k0 + k]];
+      const dp_layer& L = layers[idx[k0 + k]];
       UmmaLayer& U = P.L[k];
-      int scaled_g = 0;
-      if (pre) {      // point the scaled operand at its copy in the workspace
-        scaled_g = prescale_uses_g(L) ? 1 : 0;
-        const int cols = scaled_g ? L.d_out : L.d_in;
-        void* dst = static_cast<char*>(prescale_buf) + pre_off;
-        pre_off += align_up((size_t)B * T * cols * 2, 256);
-        Q.t[k].src = static_cast<const uint4*>(scaled_g ? L.G : L.A);
-        Q.t[k].dst = static_cast<uint4*>(dst);
-        Q.t[k].vec_per_row = cols / 8;
-        Q.t[k].pad = 0;
-        if (scaled_g) L.G = dst; else L.A = dst;
-      }
-      if (!fill_layer(U, L, T < A_BK ? T : A_BK)) return DP_ERR_CUDA;
-      U.scaled_g = scaled_g;
+      if (!(T >= bk ? fill_layer(U, L, bk, 4, 4) : fill_layer(U, L, T))) return DP_ERR_CUDA;
       U.tiles_m = ceil_div(L.d_out, 256);
       U.item_start = (int)items;
       U.partial_base = 0;
@@ -1022,21 +982,15 @@ int launch_umma_accumulate(const dp_layer* layers, const int* idx, int n, const 
     P.total_items = (int)items;
     P.B = B;
     P.T = T;
-    P.box_rows = T < A_BK ? T : A_BK;
+    P.box_rows = T < bk ? T : bk;
     P.splits = splits;
+    P.wide_boxes = T >= bk ? 1 : 0;
     P.partial_stride = 0;
-    P.pad = 0;
     P.clip = clip;
     P.partial = nullptr;
     P.status = status;
     const int grid = P.total_items < sms ? P.total_items : sms;
-    if (pre) {
-      k_prescale<<<dim3(2 * sms, nl), 256, 0, s>>>(Q);
-      if (counted(1) != cudaSuccess) return DP_ERR_CUDA;
-      k_accum<true><<<grid, A_THREADS, A_SMEM, s>>>(P);
-    } else {
-      k_accum<false><<<grid, A_THREADS, A_SMEM, s>>>(P);
-    }
+    k_accum<<<grid, A_THREADS, A_SMEM, s>>>(P);
     if (counted(1) != cudaSuccess) return DP_ERR_CUDA;
   }
   return DP_OK;

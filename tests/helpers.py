@@ -33,9 +33,9 @@ def make_layer_list(data, device, paths=None, accs=None):
     return b.LayerList(layers), accs
 
 
-def gpu_norms_clip(ll, C, minimal_ws=False):
+def gpu_norms_clip(ll, C):
     dev = ll.layers[0].G.device
-    ws = b.alloc_workspace(ll, minimal=minimal_ws)
+    ws = b.alloc_workspace(ll)
     n = torch.full((ll.B,), float("nan"), dtype=torch.float32, device=dev)
     c = torch.empty(ll.B, dtype=torch.float32, device=dev)
     b.dp_per_example_sqnorms(ll, n, False, ws)
