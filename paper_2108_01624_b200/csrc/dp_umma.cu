@@ -7,15 +7,15 @@
 //                  embedding the input is one-hot, so A_i A_i^T is the token-id equality mask: only
 //                  G_i G_i^T is formed on the tensor cores and the epilogue multiplies it by
 //                  [id_t == id_s] (integer compares).
-//   k_tile<ACCUM>  acc_w^T tile (128 of d_out x 256 of d_in) += sum over tokens of G^T diag(c) A: one
-//                  128x256x16 UMMA per 16 tokens, both operands MN-major straight from the row-major
-//                  activations.  The per-example factor c is applied to the 128-wide G tile in shared
-//                  memory by four transform warps (fp32 multiply, one bf16 rounding), which also form
-//                  the bias column sums, so A and G are read from HBM exactly once.
-//   k_tile<SQNORM> the materialised-tile norm: the same tiles for ONE example, squared and summed.
+//   k_tile_sqnorm  the materialised-tile norm: 128 (d_out) x 256 (d_in) tiles of ONE example's A_i^T G_i
+//                  (one 128x256x16 UMMA per 16 tokens, both operands MN-major straight from the
+//                  row-major activations), squared and summed in the epilogue; the tile never leaves TMEM.
+//   k_accum_pair   the clipped sum acc_w += sum_i c_i A_i^T G_i on CTA pairs (cta_group::2): 256 x 512
+//                  tiles, the per-example factor applied to the G rows in shared memory by the worker
+//                  warps, which also form the bias column sums, so A and G are read from HBM once.
 //
 // All three are persistent kernels (grid = number of SMs) over a work list decoded on the device from
-// per-layer tile counts; roles are warp-specialised (TMA producer / MMA issuer / epilogue / transform).
+// per-layer tile counts; roles are warp-specialised (TMA producer / MMA issuer / epilogue or worker warps).
 #include <cuda.h>
 
 #include <vector>
@@ -29,13 +29,9 @@ using namespace ptx;
 constexpr int kMaxLayers = 96;
 
 // Tunables (overridable with -D for experiments; the defaults are what was measured best).
-#ifndef DP_ACCUM_WORKER_SLEEP_NS
-#define DP_ACCUM_WORKER_SLEEP_NS 0     // back-off between polls of the accumulate kernel's worker and producer waits
-#endif
 #ifndef DP_TMA_L2_PROMOTION
 #define DP_TMA_L2_PROMOTION 2          // 0 none, 1 128 B, 2 256 B
 #endif
-
 struct alignas(64) UmmaLayer {
   CUtensorMap mapG;   // [B, T, d_out] bf16
   CUtensorMap mapA;   // [B, T, d_in]  bf16
@@ -43,12 +39,14 @@ struct alignas(64) UmmaLayer {
   float* acc_b;
   const int32_t* ids;     // embedding layers (Gram kernel): token ids [B, T]; the id-equality mask replaces A A^T
   int d_out, d_in;        // embedding: d_in = 0 (there is no A operand to stream)
-  int tiles_m, tiles_n;   // tile kernels: 128-wide tiles over d_out, 256-wide tiles over d_in
   int item_start;         // first work item of this layer within the launch
   int partial_base;       // first per-example partial slot of this layer
-  int has_bias, is_emb;
-  int pad[2];
+  uint16_t tiles_m, tiles_n;   // tile kernels: tiles over d_out and over d_in
+  uint8_t has_bias, is_emb;
+  uint16_t pad;
+  int pad2[4];
 };
+static_assert(sizeof(UmmaLayer) == 320, "UmmaLayer grew: 96 of them must fit the kernel parameter block");
 
 struct UmmaParams {
   UmmaLayer L[kMaxLayers];
@@ -271,52 +269,40 @@ constexpr int T_STAGE_BYTES = T_M_BYTES + T_N_BYTES;   // 48 KB
 constexpr uint32_t T_IDESC = idesc_bf16_f32(128, 256, true, true);
 
 struct TileCtl {
-  uint64_t full[T_STAGES], empty[T_STAGES], ready[T_STAGES], tmem_full[2], tmem_empty[2], drain;
+  uint64_t full[T_STAGES], empty[T_STAGES], tmem_full[2], tmem_empty[2], drain;
   uint32_t tmem_base;
   int abort;
-  float colsum[8][128];
 };
 constexpr int T_SMEM = 1024 + T_STAGES * T_STAGE_BYTES + (int)sizeof(TileCtl);
 
-struct TileItem { int l, m0, n0, e0, e1, nt, slot; };
+struct TileItem { int l, m0, n0, e, slot; };
 
-template <bool ACCUM>
 __device__ __forceinline__ TileItem tile_decode(const UmmaParams& P, int item) {
   TileItem t;
   t.l = find_layer(P, item);
   const UmmaLayer& L = P.L[t.l];
   const int rem = item - L.item_start, tiles = L.tiles_m * L.tiles_n;
-  const int outer = rem / tiles, tile = rem - outer * tiles;
+  t.e = rem / tiles;
+  const int tile = rem - t.e * tiles;
   const int mt = tile / L.tiles_n;
-  t.nt = tile - mt * L.tiles_n;
   t.m0 = mt * 128;
-  t.n0 = t.nt * 256;
-  if (ACCUM) {            // outer = split index over example ranges
-    t.e0 = (int)((long long)outer * P.B / P.splits);
-    t.e1 = (int)((long long)(outer + 1) * P.B / P.splits);
-    t.slot = 0;
-  } else {                // outer = example
-    t.e0 = outer;
-    t.e1 = outer + 1;
-    t.slot = L.partial_base + tile * 4;
-  }
+  t.n0 = (tile - mt * L.tiles_n) * 256;
+  t.slot = L.partial_base + tile * 4;
   return t;
 }
 
-template <bool ACCUM>
-__global__ void __launch_bounds__(ACCUM ? 320 : 192, 1) k_tile(const __grid_constant__ UmmaParams P) {
+__global__ void __launch_bounds__(192, 1) k_tile_sqnorm(const __grid_constant__ UmmaParams P) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* tiles = align1024(smem_raw);
   TileCtl* S = reinterpret_cast<TileCtl*>(tiles + T_STAGES * T_STAGE_BYTES);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   volatile int* abort_flag = &S->abort;
-  constexpr int NT = ACCUM ? 320 : 192;
+  constexpr int NT = 192;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < T_STAGES; ++s) {
       mbar_init(&S->full[s], 1);
       mbar_init(&S->empty[s], 1);
-      mbar_init(&S->ready[s], 128);
     }
     for (int b = 0; b < 2; ++b) { mbar_init(&S->tmem_full[b], 1); mbar_init(&S->tmem_empty[b], 4); }
     mbar_init(&S->drain, 1);
@@ -341,24 +327,23 @@ __global__ void __launch_bounds__(ACCUM ? 320 : 192, 1) k_tile(const __grid_cons
       uint32_t it = 0;
       bool alive = true;
       for (int item = blockIdx.x; item < P.total_items && alive; item += gridDim.x) {
-        const TileItem t = tile_decode<ACCUM>(P, item);
+        const TileItem t = tile_decode(P, item);
         const UmmaLayer& L = P.L[t.l];
-        for (int e = t.e0; e < t.e1 && alive; ++e) {
-          for (int tb = 0; tb < n_tb; ++tb) {
-            const uint32_t slot = it % T_STAGES, ph = (it / T_STAGES) & 1u;
-            if (!mbar_wait(&S->empty[slot], ph ^ 1u, abort_flag, P.status)) { alive = false; break; }
-            uint8_t* st = tiles + slot * T_STAGE_BYTES;
-            mbar_arrive_expect_tx(&S->full[slot], 6u * box_bytes);
-            if (P.wide_boxes) {
-              tma_load_4d(st, &L.mapG, &S->full[slot], 0, tb * 64, t.m0 / 64, e);               // 2 groups of 64 features
-              tma_load_4d(st + T_M_BYTES, &L.mapA, &S->full[slot], 0, tb * 64, t.n0 / 64, e);    // 4 groups
-            } else {
-              for (int a = 0; a < 2; ++a) tma_load_3d(st + a * T_ATOM_BYTES, &L.mapG, &S->full[slot], t.m0 + a * 64, tb * 64, e);
-              for (int a = 0; a < 4; ++a)
-                tma_load_3d(st + T_M_BYTES + a * T_ATOM_BYTES, &L.mapA, &S->full[slot], t.n0 + a * 64, tb * 64, e);
-            }
-            ++it;
+        const int e = t.e;
+        for (int tb = 0; tb < n_tb; ++tb) {
+          const uint32_t slot = it % T_STAGES, ph = (it / T_STAGES) & 1u;
+          if (!mbar_wait(&S->empty[slot], ph ^ 1u, abort_flag, P.status)) { alive = false; break; }
+          uint8_t* st = tiles + slot * T_STAGE_BYTES;
+          mbar_arrive_expect_tx(&S->full[slot], 6u * box_bytes);
+          if (P.wide_boxes) {
+            tma_load_4d(st, &L.mapG, &S->full[slot], 0, tb * 64, t.m0 / 64, e);               // 2 groups of 64 features
+            tma_load_4d(st + T_M_BYTES, &L.mapA, &S->full[slot], 0, tb * 64, t.n0 / 64, e);    // 4 groups
+          } else {
+            for (int a = 0; a < 2; ++a) tma_load_3d(st + a * T_ATOM_BYTES, &L.mapG, &S->full[slot], t.m0 + a * 64, tb * 64, e);
+            for (int a = 0; a < 4; ++a)
+              tma_load_3d(st + T_M_BYTES + a * T_ATOM_BYTES, &L.mapA, &S->full[slot], t.n0 + a * 64, tb * 64, e);
           }
+          ++it;
         }
       }
       const uint32_t pending = it < (uint32_t)T_STAGES ? it : (uint32_t)T_STAGES;
@@ -372,27 +357,25 @@ __global__ void __launch_bounds__(ACCUM ? 320 : 192, 1) k_tile(const __grid_cons
       uint32_t it = 0, tile_it = 0;
       bool alive = true;
       for (int item = blockIdx.x; item < P.total_items && alive; item += gridDim.x, ++tile_it) {
-        const TileItem t = tile_decode<ACCUM>(P, item);
+        const TileItem t = tile_decode(P, item);
         const uint32_t buf = tile_it & 1u, tph = (tile_it >> 1) & 1u;
         if (!mbar_wait(&S->tmem_empty[buf], tph ^ 1u, abort_flag, P.status)) { alive = false; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + buf * 256u;
         uint32_t first = 0;
-        for (int e = t.e0; e < t.e1 && alive; ++e) {
-          for (int tb = 0; tb < n_tb; ++tb) {
-            const uint32_t slot = it % T_STAGES, ph = (it / T_STAGES) & 1u;
-            ++it;
-            if (!mbar_wait(ACCUM ? &S->ready[slot] : &S->full[slot], ph, abort_flag, P.status)) { alive = false; break; }
-            tc_fence_after();
-            const uint32_t am = smem_u32(tiles + slot * T_STAGE_BYTES), an = am + T_M_BYTES;
+        for (int tb = 0; tb < n_tb; ++tb) {
+          const uint32_t slot = it % T_STAGES, ph = (it / T_STAGES) & 1u;
+          ++it;
+          if (!mbar_wait(&S->full[slot], ph, abort_flag, P.status)) { alive = false; break; }
+          tc_fence_after();
+          const uint32_t am = smem_u32(tiles + slot * T_STAGE_BYTES), an = am + T_M_BYTES;
 #pragma unroll
-            for (int k4 = 0; k4 < 4; ++k4) {
-              umma_bf16(d_tmem, smem_desc_sw128(am + k4 * 2048, T_ATOM_BYTES, 1024),
-                        smem_desc_sw128(an + k4 * 2048, T_ATOM_BYTES, 1024), T_IDESC, first | (uint32_t)k4);
-            }
-            first = 1;
-            umma_commit(&S->empty[slot]);
+          for (int k4 = 0; k4 < 4; ++k4) {
+            umma_bf16(d_tmem, smem_desc_sw128(am + k4 * 2048, T_ATOM_BYTES, 1024),
+                      smem_desc_sw128(an + k4 * 2048, T_ATOM_BYTES, 1024), T_IDESC, first | (uint32_t)k4);
           }
+          first = 1;
+          umma_commit(&S->empty[slot]);
         }
         if (alive) umma_commit(&S->tmem_full[buf]);
       }
@@ -404,107 +387,26 @@ __global__ void __launch_bounds__(ACCUM ? 320 : 192, 1) k_tile(const __grid_cons
     uint32_t tile_it = 0;
     bool alive = true;
     for (int item = blockIdx.x; item < P.total_items; item += gridDim.x, ++tile_it) {
-      const TileItem t = tile_decode<ACCUM>(P, item);
-      const UmmaLayer& L = P.L[t.l];
+      const TileItem t = tile_decode(P, item);
       const uint32_t buf = tile_it & 1u, tph = (tile_it >> 1) & 1u;
       if (alive) alive = __all_sync(0xffffffffu, mbar_wait(&S->tmem_full[buf], tph, abort_flag, P.status));
       if (!alive) continue;
       tc_fence_after();
-      const int m = t.m0 + (int)q * 32 + lane;
       float sum = 0.0f;
 #pragma unroll 1
       for (int ch = 0; ch < 8; ++ch) {
         uint32_t v[32];
         tmem_ld_32x32(tmem_base + ((q * 32u) << 16) + buf * 256u + (uint32_t)ch * 32u, v);
         tmem_ld_wait();
-        if (ACCUM) {
-          const int nb = t.n0 + ch * 32;
-          if (m < L.d_out && nb < L.d_in) {
-            float* p = L.acc_w + (size_t)nb * L.d_out + m;
-            const int nv = (L.d_in - nb) < 32 ? (L.d_in - nb) : 32;
-            if (P.splits > 1) {
-#pragma unroll
-              for (int j = 0; j < 32; ++j)
-                if (j < nv) atomicAdd(p + (size_t)j * L.d_out, __uint_as_float(v[j]));
-            } else {
-              float old[32];
-#pragma unroll
-              for (int j = 0; j < 32; ++j) old[j] = (j < nv) ? p[(size_t)j * L.d_out] : 0.0f;
-#pragma unroll
-              for (int j = 0; j < 32; ++j)
-                if (j < nv) p[(size_t)j * L.d_out] = old[j] + __uint_as_float(v[j]);
-            }
-          }
-        } else {
 #pragma unroll
           for (int j = 0; j < 32; ++j) sum = fmaf(__uint_as_float(v[j]), __uint_as_float(v[j]), sum);
-        }
       }
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(&S->tmem_empty[buf]);
-      if (!ACCUM) {
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) sum += __shfl_down_sync(0xffffffffu, sum, o);
-        if (lane == 0) P.partial[(size_t)t.e0 * P.partial_stride + t.slot + (int)q] = sum;
-      }
-    }
-  } else if (ACCUM) {   // ---------------- transform warps 6..9: scale the G tile, bias column sums ----------------
-    const int tt = threadIdx.x - 192;                 // 0..127
-    const int a = tt >> 6, kk = (tt & 63) >> 3, jp = tt & 7;
-    uint32_t it = 0;
-    bool alive = true;
-    for (int item = blockIdx.x; item < P.total_items; item += gridDim.x) {
-      const TileItem t = tile_decode<true>(P, item);
-      const UmmaLayer& L = P.L[t.l];
-      const bool need_bias = L.has_bias && t.nt == 0;
-      float col[8];
-#pragma unroll
-      for (int u = 0; u < 8; ++u) col[u] = 0.0f;
-      for (int e = t.e0; e < t.e1; ++e) {
-        const float cf = alive ? __ldg(P.clip + e) : 1.0f;
-        for (int tb = 0; tb < n_tb; ++tb) {
-          const uint32_t slot = it % T_STAGES, ph = (it / T_STAGES) & 1u;
-          ++it;
-          if (alive && !mbar_wait(&S->full[slot], ph, abort_flag, P.status)) alive = false;
-          if (!alive) continue;
-          if (cf != 1.0f || need_bias) {
-            uint8_t* base = tiles + slot * T_STAGE_BYTES + a * T_ATOM_BYTES + kk * 128 + jp * 16;
-#pragma unroll
-            for (int i8 = 0; i8 < 8; ++i8) {
-              uint4* p = reinterpret_cast<uint4*>(base + i8 * 1024);
-              uint4 w = *p;
-              uint32_t x[4] = {w.x, w.y, w.z, w.w};
-#pragma unroll
-              for (int u = 0; u < 4; ++u) {
-                const float lo = __uint_as_float(x[u] << 16) * cf;
-                const float hi = __uint_as_float(x[u] & 0xffff0000u) * cf;
-                col[2 * u] += lo;
-                col[2 * u + 1] += hi;
-                const __nv_bfloat162 pk = __floats2bfloat162_rn(lo, hi);
-                x[u] = *reinterpret_cast<const uint32_t*>(&pk);
-              }
-              if (cf != 1.0f) *p = make_uint4(x[0], x[1], x[2], x[3]);
-            }
-            fence_proxy_async_smem();
-          }
-          mbar_arrive(&S->ready[slot]);
-        }
-      }
-      if (need_bias) {      // uniform over the 128 transform threads; executed even after an abort
-        const int j = jp ^ kk;                        // logical 16-byte chunk under the 128-byte swizzle
-#pragma unroll
-        for (int u = 0; u < 8; ++u) S->colsum[kk][a * 64 + j * 8 + u] = col[u];
-        asm volatile("bar.sync 2, 128;" ::: "memory");
-        const int mcol = t.m0 + tt;
-        if (alive && mcol < L.d_out) {
-          float s = 0.0f;
-#pragma unroll
-          for (int r8 = 0; r8 < 8; ++r8) s += S->colsum[r8][tt];
-          if (P.splits > 1) atomicAdd(L.acc_b + mcol, s); else L.acc_b[mcol] += s;
-        }
-        asm volatile("bar.sync 2, 128;" ::: "memory");
-      }
+      for (int o = 16; o > 0; o >>= 1) sum += __shfl_down_sync(0xffffffffu, sum, o);
+      if (lane == 0) P.partial[(size_t)t.e * P.partial_stride + t.slot + (int)q] = sum;
     }
   }
   tc_fence_before();
@@ -516,39 +418,53 @@ __global__ void __launch_bounds__(ACCUM ? 320 : 192, 1) k_tile(const __grid_cons
   }
 }
 
-// =================================================================================================
-// Clipped-accumulate kernel: 256 (d_out) x 256 (d_in) output tiles, K = tokens, 64 tokens per stage.
-// Two 128x256x16 UMMAs (the two 128-row halves of the G tile) share each 256-wide A tile, so a stage of
-// 64 KB feeds 1024 tensor-pipe cycles and a 3-stage ring covers the L2/HBM latency.  The whole 512-column
-// TMEM holds the one fp32 accumulator; at the end of a tile all eight non-producer warps drain it.
-// A TMA copy costs the SM a fixed issue time per instruction, whatever its size, and the copies of one lane
-// are serial: a stage therefore arrives as two 4-D boxes (64 features x 64 tokens x four 64-feature groups,
-// one for G and one for A) instead of eight 3-D ones, which is what keeps the producer ahead of the UMMAs.
-// The clip factor is applied to the G tile in shared memory by the eight worker warps, hidden behind the
-// UMMAs of the previous stage (skipped for examples whose factor is 1).
-// =================================================================================================
-#ifndef DP_ACCUM_BK
-#define DP_ACCUM_BK 64
-#endif
-constexpr int A_BK = DP_ACCUM_BK;                       // tokens per stage (32 or 64)
-constexpr int A_STAGES = 192 / A_BK;                    // 192 KB of operand ring: 3 stages of 64 KB (or 6 of 32 KB)
-constexpr int A_ATOM_BYTES = A_BK * 128;                // A_BK tokens x 64 bf16 features
-constexpr int A_M_BYTES = 4 * A_ATOM_BYTES;             // G tile: 256 features of d_out
-constexpr int A_N_BYTES = 4 * A_ATOM_BYTES;             // A tile: 256 features of d_in
-constexpr int A_STAGE_BYTES = A_M_BYTES + A_N_BYTES;
-constexpr int A_THREADS = 320;
-
-struct AccumCtl {
-  uint64_t full[A_STAGES], empty[A_STAGES], ready[A_STAGES], tmem_full, tmem_empty, drain;
-  uint32_t tmem_base;
-  int abort;
-  float colsum[8][256];
-};
-constexpr int A_SMEM = 1024 + A_STAGES * A_STAGE_BYTES + (int)sizeof(AccumCtl);
-
 struct AccumItem { int l, m0, n0, e0, e1, nt; };
 
-__device__ __forceinline__ AccumItem accum_decode(const UmmaParams& P, int item) {
+// acc_w[(nb + j) * d_out + m] += v[j]: one lane owns row m (a d_out index), 32 columns per chunk.  The adds are
+// reductions performed at the L2 (no read-back into the SM); an element has one owner per launch unless the
+// example range is split, so the result does not depend on their order in the unsplit case.
+__device__ __forceinline__ void accum_store_chunk(const UmmaLayer& L, int m, int nb, const uint32_t (&v)[32]) {
+  if (m >= L.d_out || nb >= L.d_in) return;
+  float* p = L.acc_w + (size_t)nb * L.d_out + m;
+  const int nv = (L.d_in - nb) < 32 ? (L.d_in - nb) : 32;
+#pragma unroll
+  for (int j = 0; j < 32; ++j)
+    if (j < nv) atomicAdd(p + (size_t)j * L.d_out, __uint_as_float(v[j]));
+}
+
+// =================================================================================================
+// Clipped-accumulate kernel on CTA pairs (tcgen05 cta_group::2): a cluster of two CTAs owns one
+// 256 (d_out) x 512 (d_in) output tile.  CTA r of the pair streams
+//   G features [m0 + 128 r, +128)  -- the M rows whose accumulator lives in its own TMEM, and
+//   A features [n0 + 256 r, +256)  -- its half of the N operand of both 256 x 256 x 16 UMMAs of a k-step
+//                                     (the first 128 go to N-half 0, the second 128 to N-half 1),
+// so an SM receives 48 KB per 64 tokens instead of the 64 KB a lone CTA needs for the same number of UMMA
+// cycles: the L2 -> SM traffic, which is what bounds the single-CTA form, drops by a quarter.
+// One thread of the even CTA issues the UMMAs for both; every CTA scales its own G rows by the clip factor
+// in shared memory, sums its own bias columns and drains its own 128 x 512 accumulator.
+//   in every CTA   : full[s] (own TMA), empty[s] and tmem_full (multicast commits of the issuer)
+//   in the even CTA: ready[s] (16 worker warps of the pair have scaled stage s), tmem_empty (16 warps drained)
+// Every waiter waits for every phase of its barrier in order and whoever re-arms a barrier is gated on all
+// of its waiters (an mbarrier wait tells phases apart by parity only).  No TMA multicast is used.
+// Column c of N-half j of a CTA's accumulator is A feature n0 + 256 (c / 128) + 128 j + c % 128.
+// =================================================================================================
+constexpr int P_BK = 64;                                // tokens per stage
+constexpr int P_STAGES = 4;
+constexpr int P_ATOM_BYTES = P_BK * 128;                // 64 tokens x 64 bf16 features
+constexpr int P_M_BYTES = 2 * P_ATOM_BYTES;             // this CTA's 128 features of d_out (G)
+constexpr int P_N_BYTES = 4 * P_ATOM_BYTES;             // this CTA's 256 features of d_in (A)
+constexpr int P_STAGE_BYTES = P_M_BYTES + P_N_BYTES;    // 48 KB
+constexpr int P_THREADS = 320;                          // warp 0 TMA, warp 1 UMMA issue, warps 2..9 workers
+
+struct PairCtl {
+  uint64_t full[P_STAGES], empty[P_STAGES], ready[P_STAGES], tmem_full, tmem_empty, drain;
+  uint32_t tmem_base;
+  int abort;
+  float colsum[16][128];
+};
+constexpr int P_SMEM = 1024 + P_STAGES * P_STAGE_BYTES + (int)sizeof(PairCtl);
+
+__device__ __forceinline__ AccumItem pair_decode(const UmmaParams& P, int item) {
   AccumItem t;
   t.l = find_layer(P, item);
   const UmmaLayer& L = P.L[t.l];
@@ -557,144 +473,125 @@ __device__ __forceinline__ AccumItem accum_decode(const UmmaParams& P, int item)
   const int mt = tile / L.tiles_n;
   t.nt = tile - mt * L.tiles_n;
   t.m0 = mt * 256;
-  t.n0 = t.nt * 256;
+  t.n0 = t.nt * 512;
   t.e0 = (int)((long long)split * P.B / P.splits);
   t.e1 = (int)((long long)(split + 1) * P.B / P.splits);
   return t;
 }
 
-// acc_w[(n0 + j) * d_out + m] += tile value; one lane owns row m (a d_out index), 32 columns per chunk.
-__device__ __forceinline__ void accum_store_chunk(const UmmaLayer& L, int m, int nb, const uint32_t (&v)[32], bool atomic) {
-  if (m >= L.d_out || nb >= L.d_in) return;
-  float* p = L.acc_w + (size_t)nb * L.d_out + m;
-  const int nv = (L.d_in - nb) < 32 ? (L.d_in - nb) : 32;
-  if (atomic) {
-#pragma unroll
-    for (int j = 0; j < 32; ++j)
-      if (j < nv) atomicAdd(p + (size_t)j * L.d_out, __uint_as_float(v[j]));
-  } else {
-    float old[32];
-#pragma unroll
-    for (int j = 0; j < 32; ++j) old[j] = (j < nv) ? p[(size_t)j * L.d_out] : 0.0f;
-#pragma unroll
-    for (int j = 0; j < 32; ++j)
-      if (j < nv) p[(size_t)j * L.d_out] = old[j] + __uint_as_float(v[j]);
-  }
-}
-
-__global__ void __launch_bounds__(A_THREADS, 1) k_accum(const __grid_constant__ UmmaParams P) {
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(P_THREADS, 1)
+k_accum_pair(const __grid_constant__ UmmaParams P) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* tiles = align1024(smem_raw);
-  AccumCtl* S = reinterpret_cast<AccumCtl*>(tiles + A_STAGES * A_STAGE_BYTES);
+  PairCtl* S = reinterpret_cast<PairCtl*>(tiles + P_STAGES * P_STAGE_BYTES);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   volatile int* abort_flag = &S->abort;
-  constexpr uint32_t IDESC = idesc_bf16_f32(128, 256, true, true);
+  const uint32_t rank = cluster_ctarank();
+  const int first_item = (int)cluster_id_x(), item_stride = (int)cluster_count_x();
+  constexpr uint32_t IDESC = idesc_bf16_f32(256, 256, true, true);
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < A_STAGES; ++s) {
+    for (int s = 0; s < P_STAGES; ++s) {
       mbar_init(&S->full[s], 1);
       mbar_init(&S->empty[s], 1);
-      mbar_init(&S->ready[s], 256);
+      mbar_init(&S->ready[s], 16);
     }
     mbar_init(&S->tmem_full, 1);
-    mbar_init(&S->tmem_empty, 8);
+    mbar_init(&S->tmem_empty, 16);
     mbar_init(&S->drain, 1);
     S->abort = 0;
     fence_mbar_init();
   }
-  if (P.box_rows < A_BK) {
-    for (int k = threadIdx.x; k < A_STAGES * A_STAGE_BYTES / 16; k += A_THREADS)
+  if (P.box_rows < P_BK) {
+    for (int k = threadIdx.x; k < P_STAGES * P_STAGE_BYTES / 16; k += P_THREADS)
       reinterpret_cast<uint4*>(tiles)[k] = make_uint4(0, 0, 0, 0);
     fence_proxy_async_smem();
   }
-  if (warp == 1) { tmem_alloc(&S->tmem_base, 512); tmem_relinquish(); }
+  if (warp == 1) { tmem_alloc_pair(&S->tmem_base, 512); tmem_relinquish_pair(); }
   tc_fence_before();
   __syncthreads();
+  cluster_sync_all();           // the peer's barriers are initialised before anyone signals them
   tc_fence_after();
   const uint32_t tmem_base = S->tmem_base;
-  const int n_tb = (P.T + A_BK - 1) / A_BK;
+  const int n_tb = (P.T + P_BK - 1) / P_BK;
   const uint32_t box_bytes = (uint32_t)P.box_rows * 128u;
-  const bool atomic = P.splits > 1;
 
   if (warp == 0) {
-    if (lane == 0) {   // ---------------- TMA producer ----------------
+    if (lane == 0) {   // ---------------- TMA producer (each CTA, its own slices) ----------------
       uint32_t it = 0;
       bool alive = true;
-      for (int item = blockIdx.x; item < P.total_items && alive; item += gridDim.x) {
-        const AccumItem t = accum_decode(P, item);
+      for (int item = first_item; item < P.total_items && alive; item += item_stride) {
+        const AccumItem t = pair_decode(P, item);
         const UmmaLayer& L = P.L[t.l];
+        const int mh = t.m0 + 128 * (int)rank, nh = t.n0 + 256 * (int)rank;
         for (int e = t.e0; e < t.e1 && alive; ++e) {
           for (int tb = 0; tb < n_tb; ++tb) {
-            const uint32_t slot = it % A_STAGES, ph = (it / A_STAGES) & 1u;
-            if (!mbar_wait<DP_ACCUM_WORKER_SLEEP_NS>(&S->empty[slot], ph ^ 1u, abort_flag, P.status, 1, (int)it)) { alive = false; break; }
-            uint8_t* st = tiles + slot * A_STAGE_BYTES;
-            mbar_arrive_expect_tx(&S->full[slot], 8u * box_bytes);
+            const uint32_t slot = it % P_STAGES, ph = (it / P_STAGES) & 1u;
+            if (!mbar_wait(&S->empty[slot], ph ^ 1u, abort_flag, P.status, 11, (int)it)) { alive = false; break; }
+            uint8_t* st = tiles + slot * P_STAGE_BYTES;
+            mbar_arrive_expect_tx(&S->full[slot], 6u * box_bytes);
             if (P.wide_boxes) {
-              tma_load_4d(st, &L.mapG, &S->full[slot], 0, tb * A_BK, t.m0 / 64, e);              // 4 groups of 64 features
-              tma_load_4d(st + A_M_BYTES, &L.mapA, &S->full[slot], 0, tb * A_BK, t.n0 / 64, e);
+              tma_load_4d(st, &L.mapG, &S->full[slot], 0, tb * P_BK, mh / 64, e);                // 2 groups of 64 features
+              tma_load_4d(st + P_M_BYTES, &L.mapA, &S->full[slot], 0, tb * P_BK, nh / 64, e);    // 4 groups
             } else {
+              for (int a = 0; a < 2; ++a) tma_load_3d(st + a * P_ATOM_BYTES, &L.mapG, &S->full[slot], mh + a * 64, tb * P_BK, e);
               for (int a = 0; a < 4; ++a)
-                tma_load_3d(st + a * A_ATOM_BYTES, &L.mapG, &S->full[slot], t.m0 + a * 64, tb * A_BK, e);
-              for (int a = 0; a < 4; ++a)
-                tma_load_3d(st + A_M_BYTES + a * A_ATOM_BYTES, &L.mapA, &S->full[slot], t.n0 + a * 64, tb * A_BK, e);
+                tma_load_3d(st + P_M_BYTES + a * P_ATOM_BYTES, &L.mapA, &S->full[slot], nh + a * 64, tb * P_BK, e);
             }
             ++it;
           }
         }
       }
-      const uint32_t pending = it < (uint32_t)A_STAGES ? it : (uint32_t)A_STAGES;
+      const uint32_t pending = it < (uint32_t)P_STAGES ? it : (uint32_t)P_STAGES;
       for (uint32_t k = 0; k < pending; ++k) {
         const uint32_t j = it - 1 - k;
-        mbar_wait_drain(&S->full[j % A_STAGES], (j / A_STAGES) & 1u, P.status);
+        mbar_wait_drain(&S->full[j % P_STAGES], (j / P_STAGES) & 1u, P.status);
       }
     }
   } else if (warp == 1) {
-    if (lane == 0) {   // ---------------- MMA issuer ----------------
+    if (lane == 0 && rank == 0) {   // ---------------- UMMA issuer (even CTA only) ----------------
       uint32_t it = 0, tile_it = 0;
       bool alive = true;
-      for (int item = blockIdx.x; item < P.total_items && alive; item += gridDim.x, ++tile_it) {
-        const AccumItem t = accum_decode(P, item);
-        if (!mbar_wait(&S->tmem_empty, (tile_it & 1u) ^ 1u, abort_flag, P.status, 2, (int)tile_it)) { alive = false; break; }
+      for (int item = first_item; item < P.total_items && alive; item += item_stride, ++tile_it) {
+        const AccumItem t = pair_decode(P, item);
+        if (!mbar_wait(&S->tmem_empty, (tile_it & 1u) ^ 1u, abort_flag, P.status, 12, (int)tile_it)) { alive = false; break; }
         tc_fence_after();
         uint32_t acc = 0;
         for (int e = t.e0; e < t.e1 && alive; ++e) {
           for (int tb = 0; tb < n_tb; ++tb) {
-            const uint32_t slot = it % A_STAGES, ph = (it / A_STAGES) & 1u;
+            const uint32_t slot = it % P_STAGES, ph = (it / P_STAGES) & 1u;
             ++it;
-            if (!mbar_wait(&S->ready[slot], ph, abort_flag, P.status, 3, (int)it)) { alive = false; break; }
+            if (!mbar_wait(&S->ready[slot], ph, abort_flag, P.status, 13, (int)it)) { alive = false; break; }
             tc_fence_after();
-            const uint32_t am = smem_u32(tiles + slot * A_STAGE_BYTES), an = am + A_M_BYTES;
+            const uint32_t am = smem_u32(tiles + slot * P_STAGE_BYTES), an = am + P_M_BYTES;
 #pragma unroll
-            for (int k2 = 0; k2 < A_BK / 16; ++k2) {
-              const uint64_t bdesc = smem_desc_sw128(an + k2 * 2048, A_ATOM_BYTES, 1024);
+            for (int k4 = 0; k4 < P_BK / 16; ++k4) {
+              const uint64_t adesc = smem_desc_sw128(am + k4 * 2048, P_ATOM_BYTES, 1024);
 #pragma unroll
-              for (int h = 0; h < 2; ++h) {
-                umma_bf16(tmem_base + (uint32_t)h * 256u,
-                          smem_desc_sw128(am + h * 2 * A_ATOM_BYTES + k2 * 2048, A_ATOM_BYTES, 1024), bdesc, IDESC,
-                          acc | (uint32_t)k2);
-              }
+              for (int j = 0; j < 2; ++j)
+                umma_bf16_pair(tmem_base + (uint32_t)j * 256u, adesc,
+                               smem_desc_sw128(an + j * 2 * P_ATOM_BYTES + k4 * 2048, P_ATOM_BYTES, 1024), IDESC,
+                               acc | (uint32_t)k4);
             }
             acc = 1;
-            umma_commit(&S->empty[slot]);
+            umma_commit_pair(&S->empty[slot], (uint16_t)3);
           }
         }
-        if (alive) umma_commit(&S->tmem_full);
+        if (alive) umma_commit_pair(&S->tmem_full, (uint16_t)3);
       }
-      umma_commit(&S->drain);
+      umma_commit_pair(&S->drain, (uint16_t)1);
       mbar_wait_drain(&S->drain, 0u, P.status);
     }
-  } else {   // ---------------- warps 2..9: scale the G tile (and bias column sums), then drain the accumulator
-    // All 256 threads handle every stage and all arrive on `ready`: an mbarrier wait tells phases apart by
-    // parity only, so no waiter may ever be two phases away from its barrier; here the MMA cannot pass a
-    // stage (and the producer cannot refill its slot) before every worker thread has seen it.
+  } else {   // ---------------- warps 2..9: scale this CTA's G rows (and sum its bias columns), then drain ----------------
     const uint32_t q = (uint32_t)warp & 3u;
-    const int h = warp >= 6 ? 1 : 0;                  // which 128-row half of the tile this warp drains
+    const int h = warp >= 6 ? 1 : 0;                  // which N-half (256 accumulator columns) this warp drains
     const int tt = threadIdx.x - 64;                  // 0..255
-    const int ta = tt >> 6, kk = (tt & 63) >> 3, jp = tt & 7;   // atom, row & 7, physical 16-byte chunk
+    const int ta = tt >> 7, kk = (tt & 127) >> 3, jp = tt & 7;   // atom, token row & 15, physical 16-byte chunk
+    const int jl = jp ^ (kk & 7);                     // logical chunk under the 128-byte swizzle
     uint32_t it = 0, tile_it = 0;
     bool alive = true;
-    for (int item = blockIdx.x; item < P.total_items; item += gridDim.x, ++tile_it) {
-      const AccumItem t = accum_decode(P, item);
+    for (int item = first_item; item < P.total_items; item += item_stride, ++tile_it) {
+      const AccumItem t = pair_decode(P, item);
       const UmmaLayer& L = P.L[t.l];
       const bool need_bias = L.has_bias && t.nt == 0;
       float col[8];
@@ -708,15 +605,15 @@ __global__ void __launch_bounds__(A_THREADS, 1) k_accum(const __grid_constant__ 
         const __nv_bfloat16 clo = __float2bfloat16_rn(cf - __bfloat162float(chi));
         const __nv_bfloat162 clo2 = __halves2bfloat162(clo, clo);
         for (int tb = 0; tb < n_tb; ++tb) {
-          const uint32_t slot = it % A_STAGES, ph = (it / A_STAGES) & 1u;
+          const uint32_t slot = it % P_STAGES, ph = (it / P_STAGES) & 1u;
           ++it;
-          if (alive && !mbar_wait<DP_ACCUM_WORKER_SLEEP_NS>(&S->full[slot], ph, abort_flag, P.status, 4, (int)it)) alive = false;
+          if (alive && !mbar_wait(&S->full[slot], ph, abort_flag, P.status, 14, (int)it)) alive = false;
           if (!alive) continue;
           if (cf != 1.0f || need_bias) {
-            uint8_t* base = tiles + slot * A_STAGE_BYTES + ta * A_ATOM_BYTES + kk * 128 + jp * 16;
+            uint8_t* base = tiles + slot * P_STAGE_BYTES + ta * P_ATOM_BYTES + kk * 128 + jp * 16;
 #pragma unroll
-            for (int i4 = 0; i4 < A_BK / 8; ++i4) {   // rows kk, kk+8, ... of atom ta
-              uint4* p = reinterpret_cast<uint4*>(base + i4 * 1024);
+            for (int i4 = 0; i4 < P_BK / 16; ++i4) {   // rows kk, kk+16, ... of atom ta
+              uint4* p = reinterpret_cast<uint4*>(base + i4 * 2048);
               uint4 w = *p;
               uint32_t x[4] = {w.x, w.y, w.z, w.w};
 #pragma unroll
@@ -733,46 +630,46 @@ __global__ void __launch_bounds__(A_THREADS, 1) k_accum(const __grid_constant__ 
             }
             fence_proxy_async_smem();
           }
-          mbar_arrive(&S->ready[slot]);
+          __syncwarp();
+          if (lane == 0) mbar_arrive_cluster(&S->ready[slot], 0u);
         }
       }
-      if (need_bias) {      // uniform over the 256 threads of warps 2..9; executed even after an abort
-        const int j = jp ^ kk;                        // logical 16-byte chunk under the 128-byte swizzle
+      if (need_bias) {      // uniform over the 256 worker threads; executed even after an abort
 #pragma unroll
-        for (int u = 0; u < 8; ++u) S->colsum[kk][ta * 64 + j * 8 + u] = col[u];
+        for (int u = 0; u < 8; ++u) S->colsum[kk][ta * 64 + jl * 8 + u] = col[u];
         asm volatile("bar.sync 2, 256;" ::: "memory");
-        const int mcol = t.m0 + tt;
-        if (alive && mcol < L.d_out) {
+        const int mcol = t.m0 + 128 * (int)rank + tt;
+        if (alive && tt < 128 && mcol < L.d_out) {
           float sacc = 0.0f;
 #pragma unroll
-          for (int r8 = 0; r8 < 8; ++r8) sacc += S->colsum[r8][tt];
-          if (atomic) atomicAdd(L.acc_b + mcol, sacc); else L.acc_b[mcol] += sacc;
+          for (int r = 0; r < 16; ++r) sacc += S->colsum[r][tt];
+          atomicAdd(L.acc_b + mcol, sacc);
         }
         asm volatile("bar.sync 2, 256;" ::: "memory");
       }
-      // ---- drain the accumulator: rows [h*128 + q*32, +32) of the tile
-      if (alive) alive = __all_sync(0xffffffffu, mbar_wait(&S->tmem_full, tile_it & 1u, abort_flag, P.status, 5, (int)tile_it));
+      // ---- drain this CTA's accumulator: lanes [32 q, +32), columns [256 h, +256)
+      if (alive) alive = __all_sync(0xffffffffu, mbar_wait(&S->tmem_full, tile_it & 1u, abort_flag, P.status, 15, (int)tile_it));
       if (!alive) continue;
       tc_fence_after();
-      const int m = t.m0 + h * 128 + (int)q * 32 + lane;
+      const int m = t.m0 + 128 * (int)rank + (int)q * 32 + lane;
 #pragma unroll 1
       for (int ch = 0; ch < 8; ++ch) {
         uint32_t v[32];
         tmem_ld_32x32(tmem_base + ((q * 32u) << 16) + (uint32_t)h * 256u + (uint32_t)ch * 32u, v);
         tmem_ld_wait();
-        accum_store_chunk(L, m, t.n0 + ch * 32, v, atomic);
+        accum_store_chunk(L, m, t.n0 + 256 * (ch >> 2) + 128 * h + (ch & 3) * 32, v);
       }
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(&S->tmem_empty);
+      if (lane == 0) mbar_arrive_cluster(&S->tmem_empty, 0u);
     }
   }
   tc_fence_before();
   __syncthreads();
+  cluster_sync_all();           // neither CTA leaves while the other may still read its memory or signal it
   if (warp == 1) {
-    __syncwarp();
     tc_fence_after();
-    tmem_dealloc(tmem_base, 512);
+    tmem_dealloc_pair(tmem_base, 512);
   }
 }
 
@@ -842,7 +739,6 @@ bool umma_accumulates_bias() { return true; }
 
 static int gram_pairs(int T) { const int nb = (T + 127) / 128; return nb * (nb + 1) / 2; }
 static int tile_count(const dp_layer& L) { return ceil_div(L.d_out, 128) * ceil_div(L.d_in, 256); }
-static int accum_tile_count(const dp_layer& L) { return ceil_div(L.d_out, 256) * ceil_div(L.d_in, 256); }
 
 size_t umma_sqnorm_partials_per_example(const dp_layer* layers, const int* idx, int n, const int* use_gram) {
   size_t c = 0;
@@ -882,11 +778,12 @@ static bool fill_layer(UmmaLayer& U, const dp_layer& L, int box_rows, int groups
   U.ids = emb ? L.ids : nullptr;
   U.d_out = L.d_out;
   U.d_in = emb ? 0 : L.d_in;
-  U.tiles_m = ceil_div(L.d_out, 128);
-  U.tiles_n = ceil_div(L.d_in, 256);
+  U.tiles_m = (uint16_t)ceil_div(L.d_out, 128);
+  U.tiles_n = (uint16_t)ceil_div(L.d_in, 256);
   U.has_bias = emb ? 0 : L.has_bias;
   U.is_emb = emb ? 1 : 0;
-  U.pad[0] = U.pad[1] = 0;
+  U.pad = 0;
+  U.pad2[0] = U.pad2[1] = U.pad2[2] = U.pad2[3] = 0;
   return true;
 }
 
@@ -894,7 +791,7 @@ int launch_umma_sqnorms(const dp_layer* layers, const int* idx, int n, const int
                         int partial_stride, int partial_base, int* status, cudaStream_t s) {
   if (n <= 0) return DP_OK;
   const int B = layers[idx[0]].B, T = layers[idx[0]].T;
-  static bool attr_ok = ensure_smem(k_gram_sqnorm, G_SMEM) && ensure_smem(k_tile<false>, T_SMEM);
+  static bool attr_ok = ensure_smem(k_gram_sqnorm, G_SMEM) && ensure_smem(k_tile_sqnorm, T_SMEM);
   if (!attr_ok) return DP_ERR_CUDA;
   // Partial slots are assigned in the caller's layer order, whichever kernel fills them.
   std::vector<int> base(n);
@@ -936,7 +833,7 @@ int launch_umma_sqnorms(const dp_layer* layers, const int* idx, int n, const int
       P.status = status;
       const int grid = P.total_items < sm_count() ? P.total_items : sm_count();
       if (gram) k_gram_sqnorm<<<grid, G_THREADS, G_SMEM, s>>>(P);
-      else      k_tile<false><<<grid, 192, T_SMEM, s>>>(P);
+      else      k_tile_sqnorm<<<grid, 192, T_SMEM, s>>>(P);
       if (counted(1) != cudaSuccess) return DP_ERR_CUDA;
     }
   }
@@ -947,22 +844,25 @@ int launch_umma_accumulate(const dp_layer* layers, const int* idx, int n, const 
                            cudaStream_t s) {
   if (n <= 0) return DP_OK;
   const int B = layers[idx[0]].B, T = layers[idx[0]].T;
-  static bool attr_ok = ensure_smem(k_accum, A_SMEM);
+  static bool attr_ok = ensure_smem(k_accum_pair, P_SMEM);
   if (!attr_ok) return DP_ERR_CUDA;
-  const int bk = A_BK;
-  const int sms = sm_count();
+  const int bk = P_BK;
+  const int units = sm_count() / 2;      // CTA pairs that work on tiles side by side
   for (int k0 = 0; k0 < n; k0 += kMaxLayers) {
     const int nl = (n - k0) < kMaxLayers ? (n - k0) : kMaxLayers;
     long long tiles = 0;
-    for (int k = 0; k < nl; ++k) tiles += accum_tile_count(layers[idx[k0 + k]]);
+    for (int k = 0; k < nl; ++k) {
+      const dp_layer& L = layers[idx[k0 + k]];
+      tiles += (long long)ceil_div(L.d_out, 256) * ceil_div(L.d_in, 512);
+    }
     // Split the example range when the tiles alone cannot fill the machine: pick the smallest split count
     // (<= 8, <= B) whose last wave is at least 85% full.  Split tiles combine through fp32 atomics.
     int splits = 1;
-    if (tiles < 4ll * sms) {
+    if (tiles < 4ll * units) {
       double best = 0.0;
       for (int sp = 1; sp <= 8 && sp <= B; ++sp) {
         const long long it = tiles * sp;
-        const double eff = (double)it / (double)((it + sms - 1) / sms * sms);
+        const double eff = (double)it / (double)((it + units - 1) / units * units);
         if (eff > best + 1e-9) { best = eff; splits = sp; }
         if (eff >= 0.85) { splits = sp; break; }
       }
@@ -972,11 +872,12 @@ int launch_umma_accumulate(const dp_layer* layers, const int* idx, int n, const 
     for (int k = 0; k < nl; ++k) {
       const dp_layer& L = layers[idx[k0 + k]];
       UmmaLayer& U = P.L[k];
-      if (!(T >= bk ? fill_layer(U, L, bk, 4, 4) : fill_layer(U, L, T))) return DP_ERR_CUDA;
-      U.tiles_m = ceil_div(L.d_out, 256);
+      if (!(T >= bk ? fill_layer(U, L, bk, 2, 4) : fill_layer(U, L, T))) return DP_ERR_CUDA;
+      U.tiles_m = (uint16_t)ceil_div(L.d_out, 256);
+      U.tiles_n = (uint16_t)ceil_div(L.d_in, 512);
       U.item_start = (int)items;
       U.partial_base = 0;
-      items += (long long)accum_tile_count(L) * splits;
+      items += (long long)U.tiles_m * U.tiles_n * splits;
     }
     P.n_layers = nl;
     P.total_items = (int)items;
@@ -989,8 +890,8 @@ int launch_umma_accumulate(const dp_layer* layers, const int* idx, int n, const 
     P.clip = clip;
     P.partial = nullptr;
     P.status = status;
-    const int grid = P.total_items < sms ? P.total_items : sms;
-    k_accum<<<grid, A_THREADS, A_SMEM, s>>>(P);
+    const int active = P.total_items < units ? P.total_items : units;
+    k_accum_pair<<<2 * active, P_THREADS, P_SMEM, s>>>(P);
     if (counted(1) != cudaSuccess) return DP_ERR_CUDA;
   }
   return DP_OK;
