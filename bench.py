@@ -231,7 +231,11 @@ def main():
     ll_all = step.layer_list(data)
     ll_lin = pkg.LayerList([ll_all.layers[k] for k in lin_idx])
     ll_rest = pkg.LayerList([ll_all.layers[k] for k in rest_idx])
-    ws = torch.empty(max(pkg.dp_workspace_bytes(ll_all), 256), dtype=torch.uint8, device=dev)
+    # The model is passed in two calls (linear layers; LayerNorm + embedding) so that the accumulate GEMM can be
+    # bracketed by events of its own; each list has its workspace, and the second accumulate reuses the
+    # LayerNorm column sums its norm call left there.
+    ws = torch.empty(max(pkg.dp_workspace_bytes(ll_lin), 256), dtype=torch.uint8, device=dev)
+    ws_rest = torch.empty(max(pkg.dp_workspace_bytes(ll_rest), 256), dtype=torch.uint8, device=dev)
     sq = torch.empty(wl.B, dtype=torch.float32, device=dev)
     clip = torch.empty(wl.B, dtype=torch.float32, device=dev)
     sharded = ShardedUpdate(step, dist, world, rank) if world > 1 else None
@@ -240,14 +244,15 @@ def main():
     def one_step(ev=None):
         if ev:
             ev[0].record(stream)
-        pkg.dp_per_example_sqnorms(ll_all, sq, False, ws)
+        pkg.dp_per_example_sqnorms(ll_lin, sq, False, ws)
+        pkg.dp_per_example_sqnorms(ll_rest, sq, True, ws_rest)
         pkg.dp_clip_factors(sq, wl.C, clip)
         if ev:
             ev[1].record(stream)
         pkg.dp_clipped_accumulate(ll_lin, clip, ws)
         if ev:
             ev[2].record(stream)
-        pkg.dp_clipped_accumulate(ll_rest, clip, ws)
+        pkg.dp_clipped_accumulate_after_sqnorms(ll_rest, clip, ws_rest)
         if ev:
             ev[3].record(stream)
         step.examples_seen = wl.B * world

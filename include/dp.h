@@ -100,6 +100,15 @@ DP_API int dp_clip_factors(const float* sqnorm, int B, double C, float* clip, vo
 DP_API int dp_clipped_accumulate(const dp_layer* layers /*HOST*/, int n_layers, const float* clip,
                           void* workspace, size_t workspace_bytes, void* cuda_stream);
 
+/* The same sum, for the usual sequence norms -> clip factors -> accumulate of one microbatch: the per-example
+ * column sums of the LayerNorm terms (sum_t G and sum_t G*xhat, Section 4.3) are taken from `workspace`, where
+ * the latest dp_per_example_sqnorms call left them, instead of being formed again from G and xhat.  The caller
+ * guarantees that that call ran on the same stream over the same layer list (same order, shapes and tensors,
+ * unchanged since) with the same workspace, and that nothing wrote the workspace in between; the library
+ * cannot check this.  Results are bit-identical to dp_clipped_accumulate. */
+DP_API int dp_clipped_accumulate_after_sqnorms(const dp_layer* layers /*HOST*/, int n_layers, const float* clip,
+                                        void* workspace, size_t workspace_bytes, void* cuda_stream);
+
 /* acc <- (acc + sigma * C * z) / batch_size in place, z ~ N(0, I): the g_t line of Algorithm 1.
  * z_e depends only on (seed, step, e) with e = elem_offset + index: Philox4x32-10 block e >> 2 with
  * counter (lo(e>>2), hi(e>>2), lo(step), hi(step)) and key (lo(seed), hi(seed)); Box-Muller on the word

@@ -22,7 +22,7 @@ DP_F32, DP_BF16 = 0, 1
 DP_PATH_AUTO, DP_PATH_GRAM, DP_PATH_MATERIALIZED = 0, 1, 2
 _KINDS = {"linear": DP_LINEAR, "layernorm": DP_LAYERNORM, "embedding": DP_EMBEDDING}
 
-EXPORTS = ["dp_workspace_bytes", "dp_per_example_sqnorms", "dp_clip_factors", "dp_clipped_accumulate",
+EXPORTS = ["dp_workspace_bytes", "dp_per_example_sqnorms", "dp_clip_factors", "dp_clipped_accumulate", "dp_clipped_accumulate_after_sqnorms",
            "dp_add_noise_and_scale", "dp_adamw_step", "dp_noise_scale_adamw_step", "dp_noise_scale_adamw_step_snr",
            "dp_clip_stats", "dp_philox_u32",
            "dp_token_equality_mask", "dp_layernorm_sqnorms_static", "dp_poll_status", "dp_last_timeout_info", "dp_launch_count",
@@ -59,6 +59,7 @@ def lib() -> C.CDLL:
         L.dp_per_example_sqnorms.argtypes = [vp, i32, vp, i32, vp, sz, vp]
         L.dp_clip_factors.argtypes = [vp, i32, f32, vp, vp]
         L.dp_clipped_accumulate.argtypes = [vp, i32, vp, vp, sz, vp]
+        L.dp_clipped_accumulate_after_sqnorms.argtypes = [vp, i32, vp, vp, sz, vp]
         L.dp_add_noise_and_scale.argtypes = [vp, i64, i64, f32, f32, i64, u64, u64, vp]
         L.dp_adamw_step.argtypes = [vp, vp, vp, vp, i64, f32, f32, f32, f32, f32, i64, vp]
         L.dp_noise_scale_adamw_step.argtypes = [vp, vp, vp, vp, i32, i64, i64, f32, f32, i64, u64, u64,
@@ -194,6 +195,15 @@ def dp_clipped_accumulate(layers: LayerList, clip: torch.Tensor, workspace: Opti
     ws_p, ws_n = (_ptr(workspace), workspace.numel() * workspace.element_size()) if workspace is not None else (None, 0)
     _check("dp_clipped_accumulate",
            lib().dp_clipped_accumulate(layers.ptr, len(layers), _ptr(clip), ws_p, ws_n, _stream(stream)))
+
+
+def dp_clipped_accumulate_after_sqnorms(layers: LayerList, clip: torch.Tensor, workspace: Optional[torch.Tensor] = None,
+                                        stream=None) -> None:
+    """dp_clipped_accumulate for the call that directly follows dp_per_example_sqnorms over the same `layers`
+    and `workspace`: the LayerNorm column sums left there are reused instead of being recomputed."""
+    ws_p, ws_n = (_ptr(workspace), workspace.numel() * workspace.element_size()) if workspace is not None else (None, 0)
+    _check("dp_clipped_accumulate_after_sqnorms",
+           lib().dp_clipped_accumulate_after_sqnorms(layers.ptr, len(layers), _ptr(clip), ws_p, ws_n, _stream(stream)))
 
 
 def dp_add_noise_and_scale(acc: torch.Tensor, sigma: float, C_: float, batch_size: int, seed: int, step: int,

@@ -190,8 +190,9 @@ int dp_clip_factors(const float* sqnorm, int B, double C, float* clip, void* cud
   return DP_OK;
 }
 
-int dp_clipped_accumulate(const dp_layer* layers, int n_layers, const float* clip, void* workspace,
-                          size_t workspace_bytes, void* cuda_stream) {
+// reuse_colsums: the LayerNorm column sums are already in the workspace (left by dp_per_example_sqnorms).
+static int clipped_accumulate(const dp_layer* layers, int n_layers, const float* clip, void* workspace,
+                              size_t workspace_bytes, void* cuda_stream, bool reuse_colsums) {
   int rc = validate_layers(layers, n_layers, true);
   if (rc != DP_OK) return rc;
   if (!clip) return DP_ERR_ARG;
@@ -205,7 +206,7 @@ int dp_clipped_accumulate(const dp_layer* layers, int n_layers, const float* cli
     rc = launch_umma_accumulate(layers, plan.lin_idx.data(), (int)plan.lin_idx.size(), clip, status, s);
     if (rc != DP_OK) return rc;
   }
-  std::vector<ColTaskHost> tasks;
+  std::vector<ColTaskHost> tasks, fresh;     // all column-sum tasks / those whose sums must be formed now
   size_t u = 0;
   for (int l = 0; l < n_layers; ++l) {
     const dp_layer& L = layers[l];
@@ -215,18 +216,30 @@ int dp_clipped_accumulate(const dp_layer* layers, int n_layers, const float* cli
     if (on_umma) ++u;
     if (L.kind == DP_LINEAR) {
       if (!on_umma) DP_CUDA(launch_linear_accum_generic(L, clip, s));
-      if (L.has_bias && !(on_umma && umma_accumulates_bias())) tasks.push_back({&L, false, out});
+      if (L.has_bias && !(on_umma && umma_accumulates_bias())) {
+        tasks.push_back({&L, false, out});
+        fresh.push_back({&L, false, out});    // the norm pass does not leave these behind
+      }
     } else if (L.kind == DP_LAYERNORM) {
       tasks.push_back({&L, true, out});
+      if (!reuse_colsums) fresh.push_back({&L, true, out});
     } else {
       DP_CUDA(launch_embedding_accum(L, clip, status, s));
     }
   }
-  if (!tasks.empty()) {
-    DP_CUDA(launch_colsums_batched(tasks.data(), (int)tasks.size(), s));
-    DP_CUDA(launch_weighted_rows_sum_batched(tasks.data(), (int)tasks.size(), clip, s));
-  }
+  if (!fresh.empty()) DP_CUDA(launch_colsums_batched(fresh.data(), (int)fresh.size(), s));
+  if (!tasks.empty()) DP_CUDA(launch_weighted_rows_sum_batched(tasks.data(), (int)tasks.size(), clip, s));
   return DP_OK;
+}
+
+int dp_clipped_accumulate(const dp_layer* layers, int n_layers, const float* clip, void* workspace,
+                          size_t workspace_bytes, void* cuda_stream) {
+  return clipped_accumulate(layers, n_layers, clip, workspace, workspace_bytes, cuda_stream, false);
+}
+
+int dp_clipped_accumulate_after_sqnorms(const dp_layer* layers, int n_layers, const float* clip, void* workspace,
+                                        size_t workspace_bytes, void* cuda_stream) {
+  return clipped_accumulate(layers, n_layers, clip, workspace, workspace_bytes, cuda_stream, true);
 }
 
 static int make_noise_args(int64_t n, int64_t elem_offset, double sigma, double C, int64_t batch_size, uint64_t seed,

@@ -93,7 +93,7 @@ class DPStep:
             self._ws = torch.empty(max(need, 256), dtype=torch.uint8, device=self.device)
         b.dp_per_example_sqnorms(layers, self._sqnorm, False, self._ws, stream)
         b.dp_clip_factors(self._sqnorm, self.C, self._clip, stream)
-        b.dp_clipped_accumulate(layers, self._clip, self._ws, stream)
+        b.dp_clipped_accumulate_after_sqnorms(layers, self._clip, self._ws, stream)
         self.examples_seen += B
         return self._sqnorm, self._clip
 

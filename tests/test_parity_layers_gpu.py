@@ -114,6 +114,28 @@ def test_sqnorm_accumulate_into_splits_the_model():
     np.testing.assert_allclose(to_np(n_split), to_np(n_all), rtol=1e-5)
 
 
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+def test_accumulate_after_sqnorms_reuses_the_layernorm_sums(dtype):
+    """The entry point that takes the LayerNorm column sums from the workspace gives bit-identical accumulators
+    for every layer kind (the GEMM's L2 reductions have one owner per element here: no example split)."""
+    data = random_layers(SMALL, 6, 80, dtype, DEV, seed=13, g_scale=0.02, vocab_dup=7)
+    ol = to_oracle_layers(data)
+    C = float(np.sqrt(np.median(O.per_example_sqnorms(ol))))
+    ll_a, acc_a = make_layer_list(data, DEV)
+    n, c, ws = gpu_norms_clip(ll_a, C)
+    b.dp_clipped_accumulate(ll_a, c, ws)
+    ll_b, acc_b = make_layer_list(data, DEV)
+    n2, c2, ws2 = gpu_norms_clip(ll_b, C)
+    b.dp_clipped_accumulate_after_sqnorms(ll_b, c2, ws2)
+    assert b.dp_poll_status() == 0
+    ref = O.clipped_accumulate(ol, O.clip_factors(O.per_example_sqnorms(ol), C), O.zero_accumulators(ol))
+    for ld, xa, xb, r in zip(data, acc_a, acc_b, ref):
+        for x, y, z in zip(xa, xb, r):
+            if ld.spec.kind == LAYERNORM:
+                assert torch.equal(x, y), ld.spec.name
+            assert rel_l2(to_np(y), z) <= (BF16_TOL if dtype == torch.bfloat16 else 1e-4), ld.spec.name
+
+
 def test_zero_gradient_example_is_left_unscaled():
     data = random_layers(SMALL[:3], 3, 32, torch.bfloat16, DEV, seed=4, g_scale=0.02)
     for ld in data:
