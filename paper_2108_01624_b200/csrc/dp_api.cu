@@ -68,7 +68,7 @@ static bool use_gram(const dp_layer& L) {
 }
 
 // Workspace layout: [per-example column sums of every LayerNorm / bias task | partial sums of the tensor-core
-// norm kernels].  The two layer-list calls plan the same layout, so one workspace serves both.
+// norm kernels | wave-alignment counter of the accumulate GEMM].  The two layer-list calls plan the same layout, so one workspace serves both.
 struct WsPlan {
   size_t colsum_bytes = 0;
   size_t partial_bytes = 0;    // B * partials_per_example floats
@@ -77,7 +77,9 @@ struct WsPlan {
   std::vector<int> umma_gram;  // 1: Gram path, 0: materialised tiles
   std::vector<size_t> col_off; // per layer: byte offset of its column-sum block (or SIZE_MAX if it has none)
   std::vector<int> lin_idx;    // tensor-core layers that are linear (the accumulate GEMM takes only these)
-  size_t total() const { return align_up(colsum_bytes, 256) + align_up(partial_bytes, 256); }
+  size_t sync_bytes = 0;       // accumulate GEMM: wave-alignment counter
+  size_t sync_off() const { return align_up(colsum_bytes, 256) + align_up(partial_bytes, 256); }
+  size_t total() const { return sync_off() + sync_bytes; }
 };
 
 static WsPlan plan_workspace(const dp_layer* layers, int n_layers) {
@@ -108,6 +110,7 @@ static WsPlan plan_workspace(const dp_layer* layers, int n_layers) {
   }
   for (int l : p.umma_idx)
     if (layers[l].kind == DP_LINEAR) p.lin_idx.push_back(l);
+  if (!p.lin_idx.empty()) p.sync_bytes = 256;
   return p;
 }
 
@@ -203,7 +206,8 @@ static int clipped_accumulate(const dp_layer* layers, int n_layers, const float*
   int* status = status_ptr();
   if (!status) return DP_ERR_CUDA;
   if (!plan.lin_idx.empty()) {
-    rc = launch_umma_accumulate(layers, plan.lin_idx.data(), (int)plan.lin_idx.size(), clip, status, s);
+    unsigned int* wave_sync = reinterpret_cast<unsigned int*>(static_cast<char*>(workspace) + plan.sync_off());
+    rc = launch_umma_accumulate(layers, plan.lin_idx.data(), (int)plan.lin_idx.size(), clip, status, wave_sync, s);
     if (rc != DP_OK) return rc;
   }
   std::vector<ColTaskHost> tasks, fresh;     // all column-sum tasks / those whose sums must be formed now

@@ -74,7 +74,8 @@ size_t umma_sqnorm_partials_per_example(const dp_layer* layers, const int* idx, 
 int launch_umma_sqnorms(const dp_layer* layers, const int* idx, int n, const int* use_gram, float* partial,
                         int partial_stride, int partial_base, int* status, cudaStream_t s);
 // acc_w (and acc_b) += sum_i clip[i] * A_i^T G_i; the clip factor is applied to the G tile inside the kernel.
+// wave_sync: one zero-initialisable device word of scratch (the kernel's CTAs align their waves through it).
 int launch_umma_accumulate(const dp_layer* layers, const int* idx, int n, const float* clip, int* status,
-                           cudaStream_t s);
+                           unsigned int* wave_sync, cudaStream_t s);
 
 }  // namespace dpk

@@ -18,6 +18,7 @@
 // per-layer tile counts; roles are warp-specialised (TMA producer / MMA issuer / epilogue or worker warps).
 #include <cuda.h>
 
+#include <algorithm>
 #include <vector>
 
 #include "dp_internal.h"
@@ -29,6 +30,9 @@ using namespace ptx;
 constexpr int kMaxLayers = 96;
 
 // Tunables (overridable with -D for experiments; the defaults are what was measured best).
+#ifndef DP_ACCUM_ALIGN
+#define DP_ACCUM_ALIGN 1                // accumulate kernel: soft per-wave alignment of the CTA pairs
+#endif
 #ifndef DP_TMA_L2_PROMOTION
 #define DP_TMA_L2_PROMOTION 2          // 0 none, 1 128 B, 2 256 B
 #endif
@@ -55,6 +59,7 @@ struct UmmaParams {
   int splits;             // accumulate: number of example ranges a tile is split into
   int partial_stride;
   int wide_boxes;         // tile kernels: 1 = 4-D maps, one copy per operand and stage; 0 = 3-D maps, one copy per 64 features
+  unsigned int* wave_sync;  // accumulate: arrival counter of the soft per-wave alignment (zeroed before the launch)
   const float* clip;
   float* partial;
   int* status;
@@ -418,7 +423,7 @@ __global__ void __launch_bounds__(192, 1) k_tile_sqnorm(const __grid_constant__ 
   }
 }
 
-struct AccumItem { int l, m0, n0, e0, e1, nt; };
+struct AccumItem { int l, m0, n0, e0, e1, nt; bool valid; };
 
 // acc_w[(nb + j) * d_out + m] += v[j]: one lane owns row m (a d_out index), 32 columns per chunk.  The adds are
 // reductions performed at the L2 (no read-back into the SM); an element has one owner per launch unless the
@@ -455,6 +460,7 @@ constexpr int P_M_BYTES = 2 * P_ATOM_BYTES;             // this CTA's 128 featur
 constexpr int P_N_BYTES = 4 * P_ATOM_BYTES;             // this CTA's 256 features of d_in (A)
 constexpr int P_STAGE_BYTES = P_M_BYTES + P_N_BYTES;    // 48 KB
 constexpr int P_THREADS = 320;                          // warp 0 TMA, warp 1 UMMA issue, warps 2..9 workers
+constexpr long long kAlignLimitCycles = 40000000ll;     // longest a CTA waits for the others at a wave boundary (20-30 ms)
 
 struct PairCtl {
   uint64_t full[P_STAGES], empty[P_STAGES], ready[P_STAGES], tmem_full, tmem_empty, drain;
@@ -470,6 +476,7 @@ __device__ __forceinline__ AccumItem pair_decode(const UmmaParams& P, int item) 
   const UmmaLayer& L = P.L[t.l];
   const int rem = item - L.item_start, tiles = L.tiles_m * L.tiles_n;
   const int split = rem / tiles, tile = rem - split * tiles;
+  t.valid = item >= L.item_start && split < P.splits;     // the slots of a wave that no layer fills are idle
   const int mt = tile / L.tiles_n;
   t.nt = tile - mt * L.tiles_n;
   t.m0 = mt * 256;
@@ -520,8 +527,23 @@ k_accum_pair(const __grid_constant__ UmmaParams P) {
     if (lane == 0) {   // ---------------- TMA producer (each CTA, its own slices) ----------------
       uint32_t it = 0;
       bool alive = true;
-      for (int item = first_item; item < P.total_items && alive; item += item_stride) {
+      bool align = P.wave_sync != nullptr;
+      uint32_t wave = 0;
+      for (int item = first_item; item < P.total_items && alive; item += item_stride, ++wave) {
+        // Soft alignment: the tiles of a wave share operand blocks, which reach L2 once only if the pairs stream
+        // them at the same time.  Every CTA announces that it has reached wave w and waits, for a bounded time,
+        // until all have; a CTA that gives up once stops waiting altogether (the result does not depend on it).
+        if (align && wave > 0) {
+          atomicAdd(P.wave_sync, 1u);
+          const unsigned int target = wave * gridDim.x;
+          const long long t0 = clock64();
+          while (*reinterpret_cast<volatile unsigned int*>(P.wave_sync) < target) {
+            __nanosleep(200);
+            if (clock64() - t0 > kAlignLimitCycles) { align = false; break; }
+          }
+        }
         const AccumItem t = pair_decode(P, item);
+        if (!t.valid) continue;
         const UmmaLayer& L = P.L[t.l];
         const int mh = t.m0 + 128 * (int)rank, nh = t.n0 + 256 * (int)rank;
         for (int e = t.e0; e < t.e1 && alive; ++e) {
@@ -552,8 +574,9 @@ k_accum_pair(const __grid_constant__ UmmaParams P) {
     if (lane == 0 && rank == 0) {   // ---------------- UMMA issuer (even CTA only) ----------------
       uint32_t it = 0, tile_it = 0;
       bool alive = true;
-      for (int item = first_item; item < P.total_items && alive; item += item_stride, ++tile_it) {
+      for (int item = first_item; item < P.total_items && alive; item += item_stride) {
         const AccumItem t = pair_decode(P, item);
+        if (!t.valid) continue;
         if (!mbar_wait(&S->tmem_empty, (tile_it & 1u) ^ 1u, abort_flag, P.status, 12, (int)tile_it)) { alive = false; break; }
         tc_fence_after();
         uint32_t acc = 0;
@@ -578,6 +601,7 @@ k_accum_pair(const __grid_constant__ UmmaParams P) {
           }
         }
         if (alive) umma_commit_pair(&S->tmem_full, (uint16_t)3);
+        ++tile_it;
       }
       umma_commit_pair(&S->drain, (uint16_t)1);
       mbar_wait_drain(&S->drain, 0u, P.status);
@@ -590,8 +614,9 @@ k_accum_pair(const __grid_constant__ UmmaParams P) {
     const int jl = jp ^ (kk & 7);                     // logical chunk under the 128-byte swizzle
     uint32_t it = 0, tile_it = 0;
     bool alive = true;
-    for (int item = first_item; item < P.total_items; item += item_stride, ++tile_it) {
+    for (int item = first_item; item < P.total_items; item += item_stride) {
       const AccumItem t = pair_decode(P, item);
+      if (!t.valid) continue;
       const UmmaLayer& L = P.L[t.l];
       const bool need_bias = L.has_bias && t.nt == 0;
       float col[8];
@@ -648,7 +673,9 @@ k_accum_pair(const __grid_constant__ UmmaParams P) {
         asm volatile("bar.sync 2, 256;" ::: "memory");
       }
       // ---- drain this CTA's accumulator: lanes [32 q, +32), columns [256 h, +256)
-      if (alive) alive = __all_sync(0xffffffffu, mbar_wait(&S->tmem_full, tile_it & 1u, abort_flag, P.status, 15, (int)tile_it));
+      const uint32_t tph = tile_it & 1u;
+      ++tile_it;
+      if (alive) alive = __all_sync(0xffffffffu, mbar_wait(&S->tmem_full, tph, abort_flag, P.status, 15, (int)tile_it));
       if (!alive) continue;
       tc_fence_after();
       const int m = t.m0 + 128 * (int)rank + (int)q * 32 + lane;
@@ -828,7 +855,8 @@ int launch_umma_sqnorms(const dp_layer* layers, const int* idx, int n, const int
       P.splits = 1;
       P.wide_boxes = (!gram && T >= 64) ? 1 : 0;
       P.partial_stride = partial_stride;
-        P.clip = nullptr;
+      P.clip = nullptr;
+      P.wave_sync = nullptr;
       P.partial = partial;
       P.status = status;
       const int grid = P.total_items < sm_count() ? P.total_items : sm_count();
@@ -840,8 +868,40 @@ int launch_umma_sqnorms(const dp_layer* layers, const int* idx, int n, const int
   return DP_OK;
 }
 
+// Work items are laid out in waves of `units` slots (one slot per CTA pair and wave; pair p runs slot p of
+// every wave).  The tiles of a layer share operand blocks, so a layer's items are kept inside one wave where they
+// fit (first-fit over the layers in decreasing size); slots that no layer fills stay idle.
+static long long pack_waves(const std::vector<long long>& group, int units, std::vector<long long>& start) {
+  const int n = (int)group.size();
+  std::vector<int> order(n);
+  for (int k = 0; k < n; ++k) order[k] = k;
+  std::stable_sort(order.begin(), order.end(), [&](int a, int b) { return group[a] > group[b]; });
+  std::vector<long long> fill;    // used slots per wave
+  start.assign(n, 0);
+  for (int k : order) {
+    const long long g = group[k];
+    size_t w = 0;
+    if (g >= units) {
+      w = fill.size();            // whole waves of its own; others may share its last one
+    } else {
+      while (w < fill.size() && fill[w] + g > units) ++w;
+    }
+    if (w == fill.size()) fill.push_back(0);
+    start[k] = (long long)w * units + fill[w];
+    long long left = g;
+    while (left > 0) {
+      if (w == fill.size()) fill.push_back(0);
+      const long long take = left < units - fill[w] ? left : units - fill[w];
+      fill[w] += take;
+      left -= take;
+      ++w;
+    }
+  }
+  return (long long)fill.size() * units;
+}
+
 int launch_umma_accumulate(const dp_layer* layers, const int* idx, int n, const float* clip, int* status,
-                           cudaStream_t s) {
+                           unsigned int* wave_sync, cudaStream_t s) {
   if (n <= 0) return DP_OK;
   const int B = layers[idx[0]].B, T = layers[idx[0]].T;
   static bool attr_ok = ensure_smem(k_accum_pair, P_SMEM);
@@ -867,31 +927,40 @@ int launch_umma_accumulate(const dp_layer* layers, const int* idx, int n, const 
         if (eff >= 0.85) { splits = sp; break; }
       }
     }
-    UmmaParams P;
-    long long items = 0;
+    std::vector<long long> group(nl), start;
     for (int k = 0; k < nl; ++k) {
       const dp_layer& L = layers[idx[k0 + k]];
-      UmmaLayer& U = P.L[k];
+      group[k] = (long long)ceil_div(L.d_out, 256) * ceil_div(L.d_in, 512) * splits;
+    }
+    const long long span = pack_waves(group, units, start);
+    if (span > 0x7fffffffll) return DP_ERR_UNSUPPORTED;
+    std::vector<int> by_start(nl);
+    for (int k = 0; k < nl; ++k) by_start[k] = k;
+    std::sort(by_start.begin(), by_start.end(), [&](int a, int b) { return start[a] < start[b]; });
+    UmmaParams P;
+    for (int j = 0; j < nl; ++j) {
+      const dp_layer& L = layers[idx[k0 + by_start[j]]];
+      UmmaLayer& U = P.L[j];
       if (!(T >= bk ? fill_layer(U, L, bk, 2, 4) : fill_layer(U, L, T))) return DP_ERR_CUDA;
       U.tiles_m = (uint16_t)ceil_div(L.d_out, 256);
       U.tiles_n = (uint16_t)ceil_div(L.d_in, 512);
-      U.item_start = (int)items;
+      U.item_start = (int)start[by_start[j]];
       U.partial_base = 0;
-      items += (long long)U.tiles_m * U.tiles_n * splits;
     }
     P.n_layers = nl;
-    P.total_items = (int)items;
+    P.total_items = (int)span;
     P.B = B;
     P.T = T;
     P.box_rows = T < bk ? T : bk;
     P.splits = splits;
     P.wide_boxes = T >= bk ? 1 : 0;
     P.partial_stride = 0;
+    P.wave_sync = (DP_ACCUM_ALIGN && span > units) ? wave_sync : nullptr;     // a single wave needs no alignment
     P.clip = clip;
     P.partial = nullptr;
     P.status = status;
-    const int active = P.total_items < units ? P.total_items : units;
-    k_accum_pair<<<2 * active, P_THREADS, P_SMEM, s>>>(P);
+    if (P.wave_sync && cudaMemsetAsync(P.wave_sync, 0, sizeof(unsigned int), s) != cudaSuccess) return DP_ERR_CUDA;
+    k_accum_pair<<<2 * units, P_THREADS, P_SMEM, s>>>(P);     // the item stride of the kernel is the cluster count
     if (counted(1) != cudaSuccess) return DP_ERR_CUDA;
   }
   return DP_OK;
