@@ -29,9 +29,10 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
-# DRAM bytes (read + write) of one k_accum launch over the 24-block stack, from the ncu capture summarised in
-# profiles/k_accum_2blocks_full.md (2-block case x 12).  Set to None whenever that kernel changes.
-ACCUM_TRAFFIC_BYTES = None
+# DRAM bytes (read + write) of one k_accum_pair launch over the 24-block stack: the two dram__bytes counters are a
+# single-pass ncu capture, taken on the full workload (profiles/k_accum_pair_2blocks_full.md gives the command).
+# Set to None whenever that kernel changes.
+ACCUM_TRAFFIC_BYTES = 29.46e9
 
 METRIC = "dp_sgd_examples_per_s_bert_large"
 UNIT = "examples/s"
