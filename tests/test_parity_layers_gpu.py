@@ -136,6 +136,48 @@ def test_accumulate_after_sqnorms_reuses_the_layernorm_sums(dtype):
             assert rel_l2(to_np(y), z) <= (BF16_TOL if dtype == torch.bfloat16 else 1e-4), ld.spec.name
 
 
+# ------------------------------------------------------------------ tensor-core tile edges (bf16, widths % 64 == 0)
+
+WIDE = [LayerSpec(LINEAR, 576, 320, True, "w576x320"),      # d_in spans two 512-wide tiles, d_out two 256-wide ones
+        LayerSpec(LINEAR, 64, 64, True, "w64x64"),          # one CTA of the pair has no rows at all
+        LayerSpec(LINEAR, 1088, 192, False, "w1088x192"),   # three tiles along d_in, the last one 64 wide
+        LayerSpec(LINEAR, 256, 512, True, "w256x512")]
+
+
+@pytest.mark.parametrize("B,T", [(1, 1), (5, 16), (3, 63), (4, 64), (2, 65), (3, 130), (9, 128)])
+def test_tensor_core_tile_edges(B, T):
+    """Tiles that overhang d_in / d_out, token counts around the 64-token stage, one example, bias on and off."""
+    data = random_layers(WIDE, B, T, torch.bfloat16, DEV, seed=100 * B + T, g_scale=0.02)
+    ol = to_oracle_layers(data)
+    C = float(np.sqrt(np.median(O.per_example_sqnorms(ol))))
+    check_against_checker(data, C)
+    check_against_checker(data, C, [b.DP_PATH_MATERIALIZED] * len(WIDE))
+
+
+def test_more_linear_layers_than_one_launch_holds():
+    """130 small linear layers: the tensor-core launches take at most 96 layers each, and the accumulate GEMM packs
+    every launch's layers into waves of its own."""
+    specs = [LayerSpec(LINEAR, 64 * (1 + k % 3), 64 * (1 + (k // 3) % 2), k % 2 == 0, f"l{k}") for k in range(130)]
+    data = random_layers(specs, 3, 32, torch.bfloat16, DEV, seed=5, g_scale=0.02)
+    ol = to_oracle_layers(data)
+    C = float(np.sqrt(np.median(O.per_example_sqnorms(ol))))
+    check_against_checker(data, C)
+
+
+def test_accumulate_twice_adds_twice():
+    """acc += ...: a second call over the same microbatch doubles every accumulator (the GEMM adds through L2
+    reductions, the other kernels read-modify-write)."""
+    data = random_layers(SMALL + WIDE[:1], 4, 96, torch.bfloat16, DEV, seed=31, g_scale=0.02, vocab_dup=9)
+    ll, accs = make_layer_list(data, DEV)
+    n, c, ws = gpu_norms_clip(ll, 0.5)
+    b.dp_clipped_accumulate(ll, c, ws)
+    once = [[x.clone() for x in acc] for acc in accs]
+    b.dp_clipped_accumulate(ll, c, ws)
+    for a1, a2 in zip(once, accs):
+        for x, y in zip(a1, a2):
+            assert rel_l2(to_np(y), 2 * to_np(x)) <= 1e-6
+
+
 def test_zero_gradient_example_is_left_unscaled():
     data = random_layers(SMALL[:3], 3, 32, torch.bfloat16, DEV, seed=4, g_scale=0.02)
     for ld in data:
