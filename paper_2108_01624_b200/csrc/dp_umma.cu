@@ -60,6 +60,7 @@ struct UmmaParams {
   int partial_stride;
   int wide_boxes;         // tile kernels: 1 = 4-D maps, one copy per operand and stage; 0 = 3-D maps, one copy per 64 features
   unsigned int* wave_sync;  // accumulate: arrival counter of the soft per-wave alignment (zeroed before the launch)
+  long long align_limit;    // accumulate: longest wait at a wave boundary, in SM cycles (a few tile durations)
   const float* clip;
   float* partial;
   int* status;
@@ -460,7 +461,6 @@ constexpr int P_M_BYTES = 2 * P_ATOM_BYTES;             // this CTA's 128 featur
 constexpr int P_N_BYTES = 4 * P_ATOM_BYTES;             // this CTA's 256 features of d_in (A)
 constexpr int P_STAGE_BYTES = P_M_BYTES + P_N_BYTES;    // 48 KB
 constexpr int P_THREADS = 320;                          // warp 0 TMA, warp 1 UMMA issue, warps 2..9 workers
-constexpr long long kAlignLimitCycles = 40000000ll;     // longest a CTA waits for the others at a wave boundary (20-30 ms)
 
 struct PairCtl {
   uint64_t full[P_STAGES], empty[P_STAGES], ready[P_STAGES], tmem_full, tmem_empty, drain;
@@ -539,7 +539,7 @@ k_accum_pair(const __grid_constant__ UmmaParams P) {
           const long long t0 = clock64();
           while (*reinterpret_cast<volatile unsigned int*>(P.wave_sync) < target) {
             __nanosleep(200);
-            if (clock64() - t0 > kAlignLimitCycles) { align = false; break; }
+            if (clock64() - t0 > P.align_limit) { align = false; break; }
           }
         }
         const AccumItem t = pair_decode(P, item);
@@ -857,6 +857,7 @@ int launch_umma_sqnorms(const dp_layer* layers, const int* idx, int n, const int
       P.partial_stride = partial_stride;
       P.clip = nullptr;
       P.wave_sync = nullptr;
+      P.align_limit = 0;
       P.partial = partial;
       P.status = status;
       const int grid = P.total_items < sm_count() ? P.total_items : sm_count();
@@ -956,6 +957,9 @@ int launch_umma_accumulate(const dp_layer* layers, const int* idx, int n, const 
     P.wide_boxes = T >= bk ? 1 : 0;
     P.partial_stride = 0;
     P.wave_sync = (DP_ACCUM_ALIGN && span > units) ? wave_sync : nullptr;     // a single wave needs no alignment
+    // A pair with an idle slot waits one tile duration (about 1100 cycles per 64-token stage); twice that plus a
+    // margin tells a late CTA from one that is not resident at all.
+    P.align_limit = 2ll * (long long)B * ceil_div(T, bk) * 2000ll + 2000000ll;
     P.clip = clip;
     P.partial = nullptr;
     P.status = status;

@@ -164,6 +164,26 @@ def test_more_linear_layers_than_one_launch_holds():
     check_against_checker(data, C)
 
 
+def test_uniform_tiny_clip_factor_reaches_every_stage():
+    """c_i = 1e-3 for every example: a stage of G that reached the tensor cores unscaled would weigh 1000 times
+    its share, so every accumulator ELEMENT (not only the L2 norm) must stay within rounding of the checker."""
+    specs = [LayerSpec(LINEAR, 512, 512, True, "sq"), LayerSpec(LINEAR, 1024, 256, True, "wide")]
+    data = random_layers(specs, 16, 128, torch.bfloat16, DEV, seed=77, g_scale=0.02)
+    ll, accs = make_layer_list(data, DEV)
+    clip = torch.full((16,), 1e-3, dtype=torch.float32, device=DEV)
+    for _ in range(3):
+        for acc in accs:
+            for x in acc:
+                x.zero_()
+        b.dp_clipped_accumulate(ll, clip, b.alloc_workspace(ll))
+        assert b.dp_poll_status() == 0
+        ol = to_oracle_layers(data)
+        ref = O.clipped_accumulate(ol, np.full(16, 1e-3), O.zero_accumulators(ol))
+        for acc, racc in zip(accs, ref):
+            for x, y in zip(acc, racc):
+                assert np.max(np.abs(to_np(x) - y)) <= 0.05 * np.sqrt(np.mean(y ** 2))
+
+
 def test_accumulate_twice_adds_twice():
     """acc += ...: a second call over the same microbatch doubles every accumulator (the GEMM adds through L2
     reductions, the other kernels read-modify-write)."""
