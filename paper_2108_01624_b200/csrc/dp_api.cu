@@ -220,7 +220,7 @@ static int clipped_accumulate(const dp_layer* layers, int n_layers, const float*
     if (on_umma) ++u;
     if (L.kind == DP_LINEAR) {
       if (!on_umma) DP_CUDA(launch_linear_accum_generic(L, clip, s));
-      if (L.has_bias && !(on_umma && umma_accumulates_bias())) {
+      if (L.has_bias && !on_umma) {    // the tensor-core GEMM adds its own bias column sums
         tasks.push_back({&L, false, out});
         fresh.push_back({&L, false, out});    // the norm pass does not leave these behind
       }

@@ -68,12 +68,11 @@ cudaError_t launch_reduce_partials(const float* partial, int B, int count, float
 bool umma_supported(const dp_layer& L);
 // Number of fp32 partial sums the squared-norm kernels write for these layers (per example).
 // The partial buffer is [B][count] and is summed by launch_reduce_partials.
-// Whether launch_umma_accumulate also adds the bias column sums (else the caller runs the column-sum kernels).
-bool umma_accumulates_bias();
 size_t umma_sqnorm_partials_per_example(const dp_layer* layers, const int* idx, int n, const int* use_gram);
 int launch_umma_sqnorms(const dp_layer* layers, const int* idx, int n, const int* use_gram, float* partial,
                         int partial_stride, int partial_base, int* status, cudaStream_t s);
-// acc_w (and acc_b) += sum_i clip[i] * A_i^T G_i; the clip factor is applied to the G tile inside the kernel.
+// acc_w (and acc_b: the bias column sums are formed in the same kernel) += sum_i clip[i] * A_i^T G_i; the clip
+// factor is applied to the G tile inside the kernel.
 // wave_sync: one zero-initialisable device word of scratch (the kernel's CTAs align their waves through it).
 int launch_umma_accumulate(const dp_layer* layers, const int* idx, int n, const float* clip, int* status,
                            unsigned int* wave_sync, cudaStream_t s);

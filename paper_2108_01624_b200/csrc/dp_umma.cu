@@ -762,7 +762,6 @@ bool umma_supported(const dp_layer& L) {
   if ((long long)L.T * (L.d_in > L.d_out ? L.d_in : L.d_out) * 2 >= (1ll << 40)) return false;
   return true;
 }
-bool umma_accumulates_bias() { return true; }
 
 static int gram_pairs(int T) { const int nb = (T + 127) / 128; return nb * (nb + 1) / 2; }
 static int tile_count(const dp_layer& L) { return ceil_div(L.d_out, 128) * ceil_div(L.d_in, 256); }
