@@ -184,6 +184,16 @@ def test_uniform_tiny_clip_factor_reaches_every_stage():
                 assert np.max(np.abs(to_np(x) - y)) <= 0.05 * np.sqrt(np.mean(y ** 2))
 
 
+def test_layer_with_more_tiles_than_one_wave():
+    """A 4096 x 4096 layer has 128 accumulate tiles, more than the CTA pairs of one wave: it takes whole waves of
+    its own and the small layer beside it shares its last one."""
+    specs = [LayerSpec(LINEAR, 4096, 4096, True, "big"), LayerSpec(LINEAR, 512, 256, False, "small")]
+    data = random_layers(specs, 2, 64, torch.bfloat16, DEV, seed=41, g_scale=0.02)
+    ol = to_oracle_layers(data)
+    C = float(np.sqrt(np.median(O.per_example_sqnorms(ol))))
+    check_against_checker(data, C)
+
+
 def test_accumulate_twice_adds_twice():
     """acc += ...: a second call over the same microbatch doubles every accumulator (the GEMM adds through L2
     reductions, the other kernels read-modify-write)."""
