@@ -435,14 +435,13 @@ cudaError_t launch_reduce_partials(const float* partial, int B, int count, float
 // whose ids are equal (the one-hot input makes A_i A_i^T the id-equality mask, so the squared norm
 // sum_{t,s} [id_t == id_s] <G_t, G_s> is the sum over distinct ids of |sum of their rows|^2).
 // One CTA per example.  leader[t] = first token with the same id (integer compares only).
-//   ACCUM = false: sqnorm[i] += sum over leaders of |row sum|^2
-//   ACCUM = true : acc[id] += clip[i] * row sum   (rows of different examples may collide => atomics)
+// Norm kernel: sqnorm[i] += sum over leaders of |row sum|^2 (used when the Gram kernel's mask mode does not apply).
 // Ids outside [0, V) are skipped and reported through the status word.
 // ---------------------------------------------------------------------------------------------
-template <typename T, int VEC, bool ACCUM>
+template <typename T, int VEC>
 __global__ void __launch_bounds__(256)
-k_embedding(const int32_t* __restrict__ ids, const T* __restrict__ G, int Tn, int V, int d,
-            const float* __restrict__ clip, float* __restrict__ out, int* __restrict__ status) {
+k_embedding_sqnorm(const int32_t* __restrict__ ids, const T* __restrict__ G, int Tn, int V, int d,
+                   float* __restrict__ out, int* __restrict__ status) {
   extern __shared__ int sh_i[];          // ids[T], leader[T]
   __shared__ float red[32];
   int* sid = sh_i;
@@ -463,7 +462,6 @@ k_embedding(const int32_t* __restrict__ ids, const T* __restrict__ G, int Tn, in
     leader[t] = l;
   }
   __syncthreads();
-  const float ci = ACCUM ? __ldg(clip + i) : 1.0f;
   float total = 0.0f;
   for (int col = threadIdx.x * VEC; col < d; col += blockDim.x * VEC) {
     for (int l = 0; l < Tn; ++l) {
@@ -478,43 +476,95 @@ k_embedding(const int32_t* __restrict__ ids, const T* __restrict__ G, int Tn, in
 #pragma unroll
         for (int k = 0; k < VEC; ++k) sum[k] += g[k];
       }
-      if (ACCUM) {
-        float* dst = out + (size_t)sid[l] * d + col;
 #pragma unroll
-        for (int k = 0; k < VEC; ++k) atomicAdd(dst + k, ci * sum[k]);
-      } else {
-#pragma unroll
-        for (int k = 0; k < VEC; ++k) total = fmaf(sum[k], sum[k], total);
-      }
+      for (int k = 0; k < VEC; ++k) total = fmaf(sum[k], sum[k], total);
     }
   }
-  if (!ACCUM) {
-    total = block_sum(total, red);
-    if (threadIdx.x == 0) out[i] += total;
+  total = block_sum(total, red);
+  if (threadIdx.x == 0) out[i] += total;
+}
+
+// Accumulate, one warp per token: a warp whose token is the first of its id within the example (the leader) sums
+// the example's rows with that id and adds clip[i] times the sum to acc[id] (fp32 atomics: rows of different
+// examples collide, above all on the frequent ids).  grid = (B, ceil(T / 8)), 8 warps per block.
+template <typename T, int VEC>
+__global__ void __launch_bounds__(256)
+k_embedding_accum(const int32_t* __restrict__ ids, const T* __restrict__ G, int Tn, int V, int d,
+                  const float* __restrict__ clip, float* __restrict__ out, int* __restrict__ status) {
+  extern __shared__ int sid[];           // ids[T] of this example
+  const int i = blockIdx.x, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  for (int t = threadIdx.x; t < Tn; t += blockDim.x) sid[t] = ids[(size_t)i * Tn + t];
+  __syncthreads();
+  const int t = blockIdx.y * 8 + warp;
+  if (t >= Tn) return;
+  const int id = sid[t];
+  if (id < 0 || id >= V) {
+    if (lane == 0) atomicCAS(status, STATUS_OK, STATUS_BAD_ID);
+    return;
+  }
+  bool earlier = false;
+  for (int s = lane; s < t; s += 32) earlier |= sid[s] == id;
+  if (__any_sync(0xffffffffu, earlier)) return;      // not the leader of its id
+  const T* Gi = G + (size_t)i * Tn * d;
+  const float ci = __ldg(clip + i);
+  float* dst = out + (size_t)id * d;
+  for (int col0 = 0; col0 < d; col0 += 32 * VEC) {     // warp-uniform trip count: the ballots below need every lane
+    const int col = col0 + lane * VEC;
+    const bool in = col < d;
+    float sum[VEC];
+#pragma unroll
+    for (int k = 0; k < VEC; ++k) sum[k] = 0.0f;
+    for (int s0 = t & ~31; s0 < Tn; s0 += 32) {
+      const int s = s0 + lane;
+      unsigned m = __ballot_sync(0xffffffffu, s >= t && s < Tn && sid[s] == id);
+      while (m) {
+        const int b = __ffs(m) - 1;
+        m &= m - 1;
+        if (in) {
+          float g[VEC];
+          VecLoad<T, VEC>::ld(Gi + (size_t)(s0 + b) * d + col, g);
+#pragma unroll
+          for (int k = 0; k < VEC; ++k) sum[k] += g[k];
+        }
+      }
+    }
+    if (in) {
+#pragma unroll
+      for (int k = 0; k < VEC; ++k) atomicAdd(dst + col + k, ci * sum[k]);
+    }
   }
 }
 
-template <bool ACCUM>
-static cudaError_t embedding_dispatch(const dp_layer& L, const float* clip, float* out, int* status, cudaStream_t s) {
+cudaError_t launch_embedding_sqnorm(const dp_layer& L, float* sqnorm, int* status, cudaStream_t s) {
   const int d = L.d_out, V = L.d_in;
   const size_t sh = 2 * (size_t)L.T * sizeof(int);
   const bool al = (reinterpret_cast<uintptr_t>(L.G) & 15u) == 0;
   if (L.dtype == DP_F32) {
     const float* G = static_cast<const float*>(L.G);
-    if (al && d % 4 == 0) k_embedding<float, 4, ACCUM><<<L.B, 256, sh, s>>>(L.ids, G, L.T, V, d, clip, out, status);
-    else                  k_embedding<float, 1, ACCUM><<<L.B, 256, sh, s>>>(L.ids, G, L.T, V, d, clip, out, status);
+    if (al && d % 4 == 0) k_embedding_sqnorm<float, 4><<<L.B, 256, sh, s>>>(L.ids, G, L.T, V, d, sqnorm, status);
+    else                  k_embedding_sqnorm<float, 1><<<L.B, 256, sh, s>>>(L.ids, G, L.T, V, d, sqnorm, status);
   } else {
     const __nv_bfloat16* G = static_cast<const __nv_bfloat16*>(L.G);
-    if (al && d % 8 == 0) k_embedding<__nv_bfloat16, 8, ACCUM><<<L.B, 128, sh, s>>>(L.ids, G, L.T, V, d, clip, out, status);
-    else                  k_embedding<__nv_bfloat16, 1, ACCUM><<<L.B, 256, sh, s>>>(L.ids, G, L.T, V, d, clip, out, status);
+    if (al && d % 8 == 0) k_embedding_sqnorm<__nv_bfloat16, 8><<<L.B, 128, sh, s>>>(L.ids, G, L.T, V, d, sqnorm, status);
+    else                  k_embedding_sqnorm<__nv_bfloat16, 1><<<L.B, 256, sh, s>>>(L.ids, G, L.T, V, d, sqnorm, status);
   }
   return counted(1);
 }
-cudaError_t launch_embedding_sqnorm(const dp_layer& L, float* sqnorm, int* status, cudaStream_t s) {
-  return embedding_dispatch<false>(L, nullptr, sqnorm, status, s);
-}
 cudaError_t launch_embedding_accum(const dp_layer& L, const float* clip, int* status, cudaStream_t s) {
-  return embedding_dispatch<true>(L, clip, L.acc_w, status, s);
+  const int d = L.d_out, V = L.d_in;
+  const size_t sh = (size_t)L.T * sizeof(int);
+  const dim3 grid((unsigned)L.B, (unsigned)((L.T + 7) / 8));
+  const bool al = (reinterpret_cast<uintptr_t>(L.G) & 15u) == 0;
+  if (L.dtype == DP_F32) {
+    const float* G = static_cast<const float*>(L.G);
+    if (al && d % 4 == 0) k_embedding_accum<float, 4><<<grid, 256, sh, s>>>(L.ids, G, L.T, V, d, clip, L.acc_w, status);
+    else                  k_embedding_accum<float, 1><<<grid, 256, sh, s>>>(L.ids, G, L.T, V, d, clip, L.acc_w, status);
+  } else {
+    const __nv_bfloat16* G = static_cast<const __nv_bfloat16*>(L.G);
+    if (al && d % 8 == 0) k_embedding_accum<__nv_bfloat16, 8><<<grid, 256, sh, s>>>(L.ids, G, L.T, V, d, clip, L.acc_w, status);
+    else                  k_embedding_accum<__nv_bfloat16, 1><<<grid, 256, sh, s>>>(L.ids, G, L.T, V, d, clip, L.acc_w, status);
+  }
+  return counted(1);
 }
 
 }  // namespace dpk
