@@ -109,6 +109,15 @@ DP_API int dp_clipped_accumulate(const dp_layer* layers /*HOST*/, int n_layers, 
 DP_API int dp_clipped_accumulate_after_sqnorms(const dp_layer* layers /*HOST*/, int n_layers, const float* clip,
                                         void* workspace, size_t workspace_bytes, void* cuda_stream);
 
+/* Host-only, launches nothing: the work schedule that dp_clipped_accumulate uses for those linear layers of the list
+ * that go to the tensor-core GEMM, on a device with `units` CTA pairs (SM count / 2).  A layer of d_in x d_out has
+ * ceil(d_out/256) * ceil(d_in/512) tiles, each split into splits[k] example ranges; pair p runs item p of every
+ * wave of `units` items.  item_start[l] = first item of layer l within its launch (-1: the layer takes another
+ * path), launch[l] = index of that launch, splits[k] and slots[k] (= waves * units) per launch k < max_launches.
+ * Returns the number of launches (>= 0) or a negative status. */
+DP_API int dp_accumulate_schedule(const dp_layer* layers /*HOST*/, int n_layers, int units, int64_t* item_start /*HOST*/,
+                           int32_t* launch /*HOST*/, int32_t* splits /*HOST*/, int64_t* slots /*HOST*/, int max_launches);
+
 /* acc <- (acc + sigma * C * z) / batch_size in place, z ~ N(0, I): the g_t line of Algorithm 1.
  * z_e depends only on (seed, step, e) with e = elem_offset + index: Philox4x32-10 block e >> 2 with
  * counter (lo(e>>2), hi(e>>2), lo(step), hi(step)) and key (lo(seed), hi(seed)); Box-Muller on the word

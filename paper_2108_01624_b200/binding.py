@@ -22,7 +22,7 @@ DP_F32, DP_BF16 = 0, 1
 DP_PATH_AUTO, DP_PATH_GRAM, DP_PATH_MATERIALIZED = 0, 1, 2
 _KINDS = {"linear": DP_LINEAR, "layernorm": DP_LAYERNORM, "embedding": DP_EMBEDDING}
 
-EXPORTS = ["dp_workspace_bytes", "dp_per_example_sqnorms", "dp_clip_factors", "dp_clipped_accumulate", "dp_clipped_accumulate_after_sqnorms",
+EXPORTS = ["dp_workspace_bytes", "dp_per_example_sqnorms", "dp_clip_factors", "dp_clipped_accumulate", "dp_clipped_accumulate_after_sqnorms", "dp_accumulate_schedule",
            "dp_add_noise_and_scale", "dp_adamw_step", "dp_noise_scale_adamw_step", "dp_noise_scale_adamw_step_snr",
            "dp_clip_stats", "dp_philox_u32",
            "dp_token_equality_mask", "dp_layernorm_sqnorms_static", "dp_poll_status", "dp_last_timeout_info", "dp_launch_count",
@@ -60,6 +60,7 @@ def lib() -> C.CDLL:
         L.dp_clip_factors.argtypes = [vp, i32, f32, vp, vp]
         L.dp_clipped_accumulate.argtypes = [vp, i32, vp, vp, sz, vp]
         L.dp_clipped_accumulate_after_sqnorms.argtypes = [vp, i32, vp, vp, sz, vp]
+        L.dp_accumulate_schedule.argtypes = [vp, i32, i32, vp, vp, vp, vp, i32]
         L.dp_add_noise_and_scale.argtypes = [vp, i64, i64, f32, f32, i64, u64, u64, vp]
         L.dp_adamw_step.argtypes = [vp, vp, vp, vp, i64, f32, f32, f32, f32, f32, i64, vp]
         L.dp_noise_scale_adamw_step.argtypes = [vp, vp, vp, vp, i32, i64, i64, f32, f32, i64, u64, u64,

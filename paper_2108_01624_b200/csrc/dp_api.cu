@@ -236,6 +236,30 @@ static int clipped_accumulate(const dp_layer* layers, int n_layers, const float*
   return DP_OK;
 }
 
+int dp_accumulate_schedule(const dp_layer* layers, int n_layers, int units, int64_t* item_start, int32_t* launch,
+                           int32_t* splits, int64_t* slots, int max_launches) {
+  int rc = validate_layers(layers, n_layers, false);
+  if (rc != DP_OK) return rc;
+  if (units <= 0 || !item_start || !launch || !splits || !slots || max_launches <= 0) return DP_ERR_ARG;
+  const WsPlan plan = plan_workspace(layers, n_layers);
+  for (int l = 0; l < n_layers; ++l) { item_start[l] = -1; launch[l] = -1; }
+  const int n = (int)plan.lin_idx.size();
+  int n_launch = 0;
+  for (int k0 = 0; k0 < n; k0 += kUmmaMaxLayers, ++n_launch) {
+    if (n_launch >= max_launches) return DP_ERR_ARG;
+    const int nl = (n - k0) < kUmmaMaxLayers ? (n - k0) : kUmmaMaxLayers;
+    std::vector<long long> start;
+    int sp = 1;
+    slots[n_launch] = umma_accumulate_schedule(layers, plan.lin_idx.data() + k0, nl, units, &sp, start);
+    splits[n_launch] = sp;
+    for (int k = 0; k < nl; ++k) {
+      item_start[plan.lin_idx[k0 + k]] = start[k];
+      launch[plan.lin_idx[k0 + k]] = n_launch;
+    }
+  }
+  return n_launch;
+}
+
 int dp_clipped_accumulate(const dp_layer* layers, int n_layers, const float* clip, void* workspace,
                           size_t workspace_bytes, void* cuda_stream) {
   return clipped_accumulate(layers, n_layers, clip, workspace, workspace_bytes, cuda_stream, false);

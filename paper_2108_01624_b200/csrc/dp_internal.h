@@ -2,6 +2,7 @@
 // Host-side launchers only; the C ABI in include/dp.h is implemented in dp_api.cu.
 #pragma once
 
+#include <vector>
 #include <cuda_runtime.h>
 #include <cuda_bf16.h>
 #include <stddef.h>
@@ -71,6 +72,11 @@ bool umma_supported(const dp_layer& L);
 size_t umma_sqnorm_partials_per_example(const dp_layer* layers, const int* idx, int n, const int* use_gram);
 int launch_umma_sqnorms(const dp_layer* layers, const int* idx, int n, const int* use_gram, float* partial,
                         int partial_stride, int partial_base, int* status, cudaStream_t s);
+// Host-side schedule of one accumulate launch (at most kUmmaMaxLayers layers): splits of the example range, first
+// work item per layer; returns the number of item slots (waves x units).
+constexpr int kUmmaMaxLayers = 96;
+long long umma_accumulate_schedule(const dp_layer* layers, const int* idx, int n, int units, int* splits_out,
+                                   std::vector<long long>& start);
 // acc_w (and acc_b: the bias column sums are formed in the same kernel) += sum_i clip[i] * A_i^T G_i; the clip
 // factor is applied to the G tile inside the kernel.
 // wave_sync: one zero-initialisable device word of scratch (the kernel's CTAs align their waves through it).

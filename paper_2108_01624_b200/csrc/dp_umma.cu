@@ -27,7 +27,7 @@
 namespace dpk {
 using namespace ptx;
 
-constexpr int kMaxLayers = 96;
+constexpr int kMaxLayers = kUmmaMaxLayers;
 
 // Tunables (overridable with -D for experiments; the defaults are what was measured best).
 #ifndef DP_ACCUM_ALIGN
@@ -900,6 +900,37 @@ static long long pack_waves(const std::vector<long long>& group, int units, std:
   return (long long)fill.size() * units;
 }
 
+// The schedule of one accumulate launch over layers idx[0..n): the number of example ranges every tile is split
+// into, the first work item of every layer, and (returned) the number of item slots = waves x units.
+long long umma_accumulate_schedule(const dp_layer* layers, const int* idx, int n, int units, int* splits_out,
+                                   std::vector<long long>& start) {
+  const int B = layers[idx[0]].B;
+  long long tiles = 0;
+  for (int k = 0; k < n; ++k) {
+    const dp_layer& L = layers[idx[k]];
+    tiles += (long long)ceil_div(L.d_out, 256) * ceil_div(L.d_in, 512);
+  }
+  // Split the example range when the tiles alone cannot fill the machine: pick the smallest split count
+  // (<= 8, <= B) whose last wave is at least 85% full.  Split tiles combine through fp32 atomics.
+  int splits = 1;
+  if (tiles < 4ll * units) {
+    double best = 0.0;
+    for (int sp = 1; sp <= 8 && sp <= B; ++sp) {
+      const long long it = tiles * sp;
+      const double eff = (double)it / (double)((it + units - 1) / units * units);
+      if (eff > best + 1e-9) { best = eff; splits = sp; }
+      if (eff >= 0.85) { splits = sp; break; }
+    }
+  }
+  std::vector<long long> group(n);
+  for (int k = 0; k < n; ++k) {
+    const dp_layer& L = layers[idx[k]];
+    group[k] = (long long)ceil_div(L.d_out, 256) * ceil_div(L.d_in, 512) * splits;
+  }
+  *splits_out = splits;
+  return pack_waves(group, units, start);
+}
+
 int launch_umma_accumulate(const dp_layer* layers, const int* idx, int n, const float* clip, int* status,
                            unsigned int* wave_sync, cudaStream_t s) {
   if (n <= 0) return DP_OK;
@@ -910,29 +941,9 @@ int launch_umma_accumulate(const dp_layer* layers, const int* idx, int n, const 
   const int units = sm_count() / 2;      // CTA pairs that work on tiles side by side
   for (int k0 = 0; k0 < n; k0 += kMaxLayers) {
     const int nl = (n - k0) < kMaxLayers ? (n - k0) : kMaxLayers;
-    long long tiles = 0;
-    for (int k = 0; k < nl; ++k) {
-      const dp_layer& L = layers[idx[k0 + k]];
-      tiles += (long long)ceil_div(L.d_out, 256) * ceil_div(L.d_in, 512);
-    }
-    // Split the example range when the tiles alone cannot fill the machine: pick the smallest split count
-    // (<= 8, <= B) whose last wave is at least 85% full.  Split tiles combine through fp32 atomics.
     int splits = 1;
-    if (tiles < 4ll * units) {
-      double best = 0.0;
-      for (int sp = 1; sp <= 8 && sp <= B; ++sp) {
-        const long long it = tiles * sp;
-        const double eff = (double)it / (double)((it + units - 1) / units * units);
-        if (eff > best + 1e-9) { best = eff; splits = sp; }
-        if (eff >= 0.85) { splits = sp; break; }
-      }
-    }
-    std::vector<long long> group(nl), start;
-    for (int k = 0; k < nl; ++k) {
-      const dp_layer& L = layers[idx[k0 + k]];
-      group[k] = (long long)ceil_div(L.d_out, 256) * ceil_div(L.d_in, 512) * splits;
-    }
-    const long long span = pack_waves(group, units, start);
+    std::vector<long long> start;
+    const long long span = umma_accumulate_schedule(layers, idx + k0, nl, units, &splits, start);
     if (span > 0x7fffffffll) return DP_ERR_UNSUPPORTED;
     std::vector<int> by_start(nl);
     for (int k = 0; k < nl; ++k) by_start[k] = k;

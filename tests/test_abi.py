@@ -95,3 +95,62 @@ def test_missing_library_fails_loudly(monkeypatch, tmp_path):
     monkeypatch.setattr(b, "LIB_PATH", str(tmp_path / "nope.so"))
     with pytest.raises(ImportError):
         b.lib()
+
+
+def _fake_bf16_linears(shapes, B, T):
+    """Descriptors with made-up (aligned) device addresses: enough for the host-only planning calls."""
+    L = (b.dp_layer * len(shapes))()
+    for k, (d_in, d_out) in enumerate(shapes):
+        L[k].kind, L[k].dtype, L[k].has_bias, L[k].B, L[k].T, L[k].d_in, L[k].d_out = 0, 1, 1, B, T, d_in, d_out
+        L[k].A, L[k].G = 1 << 20, 1 << 21
+    return L
+
+
+def _schedule(lib, L, units, max_launches=8):
+    n = len(L)
+    start, launch = (C.c_int64 * n)(), (C.c_int32 * n)()
+    splits, slots = (C.c_int32 * max_launches)(), (C.c_int64 * max_launches)()
+    rc = lib.dp_accumulate_schedule(C.cast(L, C.c_void_p), n, units, C.cast(start, C.c_void_p), C.cast(launch, C.c_void_p),
+                                    C.cast(splits, C.c_void_p), C.cast(slots, C.c_void_p), max_launches)
+    return rc, list(start), list(launch), list(splits), list(slots)
+
+
+def _tiles(d_in, d_out):
+    return -(-d_out // 256) * -(-d_in // 512)
+
+
+def test_accumulate_schedule_bert_large_packs_layers_into_waves(lib):
+    """96 linears of BERT-Large on 74 CTA pairs: 2304 tiles in 32 waves, no layer straddling a wave, no overlap."""
+    block = [(1024, 3072), (1024, 1024), (1024, 4096), (4096, 1024)]
+    shapes = block * 24
+    rc, start, launch, splits, slots = _schedule(lib, _fake_bf16_linears(shapes, 256, 128), 74)
+    assert rc == 1 and splits[0] == 1 and slots[0] == 32 * 74
+    taken = set()
+    for (d_in, d_out), s0 in zip(shapes, start):
+        g = _tiles(d_in, d_out)
+        assert s0 >= 0 and s0 // 74 == (s0 + g - 1) // 74          # inside one wave
+        items = set(range(s0, s0 + g))
+        assert not (items & taken)
+        taken |= items
+    assert len(taken) == 2304 and max(taken) < slots[0]
+
+
+def test_accumulate_schedule_splits_large_groups_and_launches(lib):
+    # a layer with more tiles than a wave takes whole waves; the small one shares its last wave
+    rc, start, launch, splits, slots = _schedule(lib, _fake_bf16_linears([(512, 256), (4096, 4096)], 2, 64), 74)
+    assert rc == 1 and splits[0] == 1
+    assert start[1] == 0 and start[0] == 128 and slots[0] == 2 * 74
+    # few tiles: the example range is split (<= B, <= 8) until the wave is at least 85 % full
+    rc, start, launch, splits, slots = _schedule(lib, _fake_bf16_linears([(512, 256)] * 3, 6, 64), 74)
+    assert rc == 1 and splits[0] == 6 and slots[0] == 74 and sorted(start) == [0, 6, 12]
+    # more than 96 tensor-core layers: a second launch with a schedule of its own
+    rc, start, launch, splits, slots = _schedule(lib, _fake_bf16_linears([(64, 64)] * 130, 3, 32), 74)
+    assert rc == 2 and launch[:96] == [0] * 96 and launch[96:] == [1] * 34
+    assert splits[:2] == [2, 2] and slots[:2] == [3 * 74, 74]      # 192 items in 3 waves, 68 items in 1
+    assert sorted(start[:96]) == [2 * k for k in range(96)] and sorted(start[96:]) == [2 * k for k in range(34)]
+    # layers the tensor-core GEMM does not take (fp32, widths not a multiple of 64) are left out
+    L = _fake_bf16_linears([(64, 64), (72, 40)], 3, 32)
+    rc, start, launch, _, _ = _schedule(lib, L, 74)
+    assert rc == 1 and start[1] == -1 and launch[1] == -1
+    # argument checks
+    assert lib.dp_accumulate_schedule(C.cast(L, C.c_void_p), 2, 0, 256, 256, 256, 256, 1) == -1
