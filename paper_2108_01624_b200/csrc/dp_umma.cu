@@ -55,10 +55,8 @@ static_assert(sizeof(UmmaLayer) == 320, "UmmaLayer grew: 96 of them must fit the
 struct UmmaParams {
   UmmaLayer L[kMaxLayers];
   int n_layers, total_items, B, T;
-  int box_rows;           // token rows per TMA box (min(tile rows, T))
   int splits;             // accumulate: number of example ranges a tile is split into
   int partial_stride;
-  int wide_boxes;         // tile kernels: 1 = 4-D maps, one copy per operand and stage; 0 = 3-D maps, one copy per 64 features
   unsigned int* wave_sync;  // accumulate: arrival counter of the soft per-wave alignment (zeroed before the launch)
   long long align_limit;    // accumulate: longest wait at a wave boundary, in SM cycles (a few tile durations)
   const float* clip;
@@ -119,18 +117,14 @@ __global__ void __launch_bounds__(G_THREADS, 1) k_gram_sqnorm(const __grid_const
     S->abort = 0;
     fence_mbar_init();
   }
-  if (P.box_rows < 128) {   // rows the TMA box never writes must read as zero tokens
-    for (int k = threadIdx.x; k < G_SLOTS * G_SLOT_BYTES / 16; k += G_THREADS)
-      reinterpret_cast<uint4*>(tiles)[k] = make_uint4(0, 0, 0, 0);
-    fence_proxy_async_smem();
-  }
   if (warp == 1) { tmem_alloc(&S->tmem_base, 512); tmem_relinquish(); }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = S->tmem_base;
   const int nblk = (P.T + 127) / 128, npairs = nblk * (nblk + 1) / 2;
-  const uint32_t box_bytes = (uint32_t)P.box_rows * 128u;
+  // A box is always 128 tokens high: rows beyond T are outside the tensor and arrive as zeros.
+  constexpr uint32_t box_bytes = 128u * 128u;
 
   if (warp == 0) {
     if (lane == 0) {   // ---------------- TMA producer ----------------
@@ -303,7 +297,6 @@ __global__ void __launch_bounds__(192, 1) k_tile_sqnorm(const __grid_constant__ 
   TileCtl* S = reinterpret_cast<TileCtl*>(tiles + T_STAGES * T_STAGE_BYTES);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   volatile int* abort_flag = &S->abort;
-  constexpr int NT = 192;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < T_STAGES; ++s) {
@@ -315,18 +308,12 @@ __global__ void __launch_bounds__(192, 1) k_tile_sqnorm(const __grid_constant__ 
     S->abort = 0;
     fence_mbar_init();
   }
-  if (P.box_rows < 64) {
-    for (int k = threadIdx.x; k < T_STAGES * T_STAGE_BYTES / 16; k += NT)
-      reinterpret_cast<uint4*>(tiles)[k] = make_uint4(0, 0, 0, 0);
-    fence_proxy_async_smem();
-  }
   if (warp == 1) { tmem_alloc(&S->tmem_base, 512); tmem_relinquish(); }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = S->tmem_base;
   const int n_tb = (P.T + 63) / 64;
-  const uint32_t box_bytes = (uint32_t)P.box_rows * 128u;
 
   if (warp == 0) {
     if (lane == 0) {   // ---------------- TMA producer ----------------
@@ -340,15 +327,10 @@ __global__ void __launch_bounds__(192, 1) k_tile_sqnorm(const __grid_constant__ 
           const uint32_t slot = it % T_STAGES, ph = (it / T_STAGES) & 1u;
           if (!mbar_wait(&S->empty[slot], ph ^ 1u, abort_flag, P.status)) { alive = false; break; }
           uint8_t* st = tiles + slot * T_STAGE_BYTES;
-          mbar_arrive_expect_tx(&S->full[slot], 6u * box_bytes);
-          if (P.wide_boxes) {
-            tma_load_4d(st, &L.mapG, &S->full[slot], 0, tb * 64, t.m0 / 64, e);               // 2 groups of 64 features
-            tma_load_4d(st + T_M_BYTES, &L.mapA, &S->full[slot], 0, tb * 64, t.n0 / 64, e);    // 4 groups
-          } else {
-            for (int a = 0; a < 2; ++a) tma_load_3d(st + a * T_ATOM_BYTES, &L.mapG, &S->full[slot], t.m0 + a * 64, tb * 64, e);
-            for (int a = 0; a < 4; ++a)
-              tma_load_3d(st + T_M_BYTES + a * T_ATOM_BYTES, &L.mapA, &S->full[slot], t.n0 + a * 64, tb * 64, e);
-          }
+          // two boxes of 64 features x 64 tokens x (2 | 4) feature groups; tokens beyond T arrive as zeros
+          mbar_arrive_expect_tx(&S->full[slot], (uint32_t)T_STAGE_BYTES);
+          tma_load_4d(st, &L.mapG, &S->full[slot], 0, tb * 64, t.m0 / 64, e);
+          tma_load_4d(st + T_M_BYTES, &L.mapA, &S->full[slot], 0, tb * 64, t.n0 / 64, e);
           ++it;
         }
       }
@@ -375,10 +357,12 @@ __global__ void __launch_bounds__(192, 1) k_tile_sqnorm(const __grid_constant__ 
           if (!mbar_wait(&S->full[slot], ph, abort_flag, P.status)) { alive = false; break; }
           tc_fence_after();
           const uint32_t am = smem_u32(tiles + slot * T_STAGE_BYTES), an = am + T_M_BYTES;
+          const int left = P.T - tb * 64, nk = left >= 64 ? 4 : (left + 15) >> 4;   // k-steps that hold tokens
 #pragma unroll
           for (int k4 = 0; k4 < 4; ++k4) {
-            umma_bf16(d_tmem, smem_desc_sw128(am + k4 * 2048, T_ATOM_BYTES, 1024),
-                      smem_desc_sw128(an + k4 * 2048, T_ATOM_BYTES, 1024), T_IDESC, first | (uint32_t)k4);
+            if (k4 < nk)
+              umma_bf16(d_tmem, smem_desc_sw128(am + k4 * 2048, T_ATOM_BYTES, 1024),
+                        smem_desc_sw128(an + k4 * 2048, T_ATOM_BYTES, 1024), T_IDESC, first | (uint32_t)k4);
           }
           first = 1;
           umma_commit(&S->empty[slot]);
@@ -509,11 +493,6 @@ k_accum_pair(const __grid_constant__ UmmaParams P) {
     S->abort = 0;
     fence_mbar_init();
   }
-  if (P.box_rows < P_BK) {
-    for (int k = threadIdx.x; k < P_STAGES * P_STAGE_BYTES / 16; k += P_THREADS)
-      reinterpret_cast<uint4*>(tiles)[k] = make_uint4(0, 0, 0, 0);
-    fence_proxy_async_smem();
-  }
   if (warp == 1) { tmem_alloc_pair(&S->tmem_base, 512); tmem_relinquish_pair(); }
   tc_fence_before();
   __syncthreads();
@@ -521,7 +500,6 @@ k_accum_pair(const __grid_constant__ UmmaParams P) {
   tc_fence_after();
   const uint32_t tmem_base = S->tmem_base;
   const int n_tb = (P.T + P_BK - 1) / P_BK;
-  const uint32_t box_bytes = (uint32_t)P.box_rows * 128u;
 
   if (warp == 0) {
     if (lane == 0) {   // ---------------- TMA producer (each CTA, its own slices) ----------------
@@ -551,15 +529,11 @@ k_accum_pair(const __grid_constant__ UmmaParams P) {
             const uint32_t slot = it % P_STAGES, ph = (it / P_STAGES) & 1u;
             if (!mbar_wait(&S->empty[slot], ph ^ 1u, abort_flag, P.status, 11, (int)it)) { alive = false; break; }
             uint8_t* st = tiles + slot * P_STAGE_BYTES;
-            mbar_arrive_expect_tx(&S->full[slot], 6u * box_bytes);
-            if (P.wide_boxes) {
-              tma_load_4d(st, &L.mapG, &S->full[slot], 0, tb * P_BK, mh / 64, e);                // 2 groups of 64 features
-              tma_load_4d(st + P_M_BYTES, &L.mapA, &S->full[slot], 0, tb * P_BK, nh / 64, e);    // 4 groups
-            } else {
-              for (int a = 0; a < 2; ++a) tma_load_3d(st + a * P_ATOM_BYTES, &L.mapG, &S->full[slot], mh + a * 64, tb * P_BK, e);
-              for (int a = 0; a < 4; ++a)
-                tma_load_3d(st + P_M_BYTES + a * P_ATOM_BYTES, &L.mapA, &S->full[slot], nh + a * 64, tb * P_BK, e);
-            }
+            // two boxes of 64 features x 64 tokens x (2 | 4) feature groups; tokens beyond T and feature groups
+            // beyond the layer's width are outside the tensor and arrive as zeros
+            mbar_arrive_expect_tx(&S->full[slot], (uint32_t)P_STAGE_BYTES);
+            tma_load_4d(st, &L.mapG, &S->full[slot], 0, tb * P_BK, mh / 64, e);
+            tma_load_4d(st + P_M_BYTES, &L.mapA, &S->full[slot], 0, tb * P_BK, nh / 64, e);
             ++it;
           }
         }
@@ -587,14 +561,27 @@ k_accum_pair(const __grid_constant__ UmmaParams P) {
             if (!mbar_wait(&S->ready[slot], ph, abort_flag, P.status, 13, (int)it)) { alive = false; break; }
             tc_fence_after();
             const uint32_t am = smem_u32(tiles + slot * P_STAGE_BYTES), an = am + P_M_BYTES;
+            const int left = P.T - tb * P_BK;
+            if (left >= P_BK) {
 #pragma unroll
-            for (int k4 = 0; k4 < P_BK / 16; ++k4) {
-              const uint64_t adesc = smem_desc_sw128(am + k4 * 2048, P_ATOM_BYTES, 1024);
+              for (int k4 = 0; k4 < P_BK / 16; ++k4) {
+                const uint64_t adesc = smem_desc_sw128(am + k4 * 2048, P_ATOM_BYTES, 1024);
 #pragma unroll
-              for (int j = 0; j < 2; ++j)
-                umma_bf16_pair(tmem_base + (uint32_t)j * 256u, adesc,
-                               smem_desc_sw128(an + j * 2 * P_ATOM_BYTES + k4 * 2048, P_ATOM_BYTES, 1024), IDESC,
-                               acc | (uint32_t)k4);
+                for (int j = 0; j < 2; ++j)
+                  umma_bf16_pair(tmem_base + (uint32_t)j * 256u, adesc,
+                                 smem_desc_sw128(an + j * 2 * P_ATOM_BYTES + k4 * 2048, P_ATOM_BYTES, 1024), IDESC,
+                                 acc | (uint32_t)k4);
+              }
+            } else {                                   // ragged last stage: only the k-steps that hold tokens
+              const int nk = (left + 15) >> 4;
+#pragma unroll 1
+              for (int k4 = 0; k4 < nk; ++k4) {
+                const uint64_t adesc = smem_desc_sw128(am + k4 * 2048, P_ATOM_BYTES, 1024);
+                for (int j = 0; j < 2; ++j)
+                  umma_bf16_pair(tmem_base + (uint32_t)j * 256u, adesc,
+                                 smem_desc_sw128(an + j * 2 * P_ATOM_BYTES + k4 * 2048, P_ATOM_BYTES, 1024), IDESC,
+                                 acc | (uint32_t)k4);
+              }
             }
             acc = 1;
             umma_commit_pair(&S->empty[slot], (uint16_t)3);
@@ -789,6 +776,7 @@ static bool ensure_smem(K kernel, int bytes) {
 }
 
 // groups_g / groups_a > 0: 4-D maps whose box spans that many 64-feature groups (tile kernels); 0: 3-D maps (Gram).
+// A box may be taller than T or span more groups than the layer has: what lies outside the tensor is zero-filled.
 static bool fill_layer(UmmaLayer& U, const dp_layer& L, int box_rows, int groups_g = 0, int groups_a = 0) {
   const bool emb = L.kind == DP_EMBEDDING;
   if (groups_g > 0) {
@@ -839,8 +827,7 @@ int launch_umma_sqnorms(const dp_layer* layers, const int* idx, int n, const int
         const long long add = (long long)B * (gram ? gram_pairs(T) : tile_count(L));
         if (items + add > 0x7fffffffll) break;
         UmmaLayer& U = P.L[P.n_layers];
-        if (!(gram ? fill_layer(U, L, T < 128 ? T : 128)
-                   : (T >= 64 ? fill_layer(U, L, 64, 2, 4) : fill_layer(U, L, T)))) return DP_ERR_CUDA;
+        if (!(gram ? fill_layer(U, L, 128) : fill_layer(U, L, 64, 2, 4))) return DP_ERR_CUDA;
         U.item_start = (int)items;
         U.partial_base = base[k];
         items += add;
@@ -850,9 +837,7 @@ int launch_umma_sqnorms(const dp_layer* layers, const int* idx, int n, const int
       P.total_items = (int)items;
       P.B = B;
       P.T = T;
-      P.box_rows = gram ? (T < 128 ? T : 128) : (T < 64 ? T : 64);
       P.splits = 1;
-      P.wide_boxes = (!gram && T >= 64) ? 1 : 0;
       P.partial_stride = partial_stride;
       P.clip = nullptr;
       P.wave_sync = nullptr;
@@ -952,7 +937,7 @@ int launch_umma_accumulate(const dp_layer* layers, const int* idx, int n, const 
     for (int j = 0; j < nl; ++j) {
       const dp_layer& L = layers[idx[k0 + by_start[j]]];
       UmmaLayer& U = P.L[j];
-      if (!(T >= bk ? fill_layer(U, L, bk, 2, 4) : fill_layer(U, L, T))) return DP_ERR_CUDA;
+      if (!fill_layer(U, L, bk, 2, 4)) return DP_ERR_CUDA;
       U.tiles_m = (uint16_t)ceil_div(L.d_out, 256);
       U.tiles_n = (uint16_t)ceil_div(L.d_in, 512);
       U.item_start = (int)start[by_start[j]];
@@ -962,9 +947,7 @@ int launch_umma_accumulate(const dp_layer* layers, const int* idx, int n, const 
     P.total_items = (int)span;
     P.B = B;
     P.T = T;
-    P.box_rows = T < bk ? T : bk;
     P.splits = splits;
-    P.wide_boxes = T >= bk ? 1 : 0;
     P.partial_stride = 0;
     P.wave_sync = (DP_ACCUM_ALIGN && span > units) ? wave_sync : nullptr;     // a single wave needs no alignment
     // A pair with an idle slot waits one tile duration (about 1100 cycles per 64-token stage); twice that plus a

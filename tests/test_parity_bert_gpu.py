@@ -83,8 +83,9 @@ def test_bert_large_stack_subset_and_samples(n_layers):
     b.dp_clipped_accumulate(ll, c, ws)
     torch.cuda.synchronize()
     assert b.dp_poll_status() == 0
-    # (a) checker on examples 0..7, all layers and the embedding
-    rows = slice(0, 8)
+    # (a) checker on eight examples spread over the batch (first, last, and both sides of the half-way and
+    # quarter marks, where an indexing slip would show), all layers and the embedding
+    rows = [0, 1, 63, 64, 127, 128, 254, 255]
     sub = _subset(data, rows)
     ol = to_oracle_layers(sub)
     n_ref = O.per_example_sqnorms(ol)
@@ -93,7 +94,7 @@ def test_bert_large_stack_subset_and_samples(n_layers):
     np.testing.assert_allclose(to_np(c[rows]), c_ref, rtol=CLIP_TOL)
     # (b) full launch size: sampled accumulator entries in fp64
     _sampled_entries_check(data, accs, c, n_samples=6, seed=1)
-    # (c) the 8-example subset through the GPU path, element by element against the checker
+    # (c) the same eight examples as a microbatch of their own through the GPU path, element by element
     ll8, acc8 = make_layer_list(sub, DEV)
     n8, c8, ws8 = gpu_norms_clip(ll8, wl.C)
     b.dp_clipped_accumulate(ll8, c8, ws8)
