@@ -261,11 +261,13 @@ __global__ void __launch_bounds__(G_THREADS, 1) k_gram_sqnorm(const __grid_const
 // =================================================================================================
 // Tile kernel: 128 (d_out) x 256 (d_in) output tiles, K = tokens
 // =================================================================================================
-constexpr int T_STAGES = 4;
-constexpr int T_ATOM_BYTES = 64 * 128;                 // 64 tokens x 64 bf16 features
+constexpr int T_BK = 128;                              // tokens per stage: one box per operand covers 8 k-steps
+constexpr int T_STAGES = 2;
+constexpr int T_THREADS = 320;                          // warp 0 TMA, warp 1 UMMA issue, warps 2..9 epilogue
+constexpr int T_ATOM_BYTES = T_BK * 128;               // 128 tokens x 64 bf16 features
 constexpr int T_M_BYTES = 2 * T_ATOM_BYTES;            // G tile: 128 features of d_out
 constexpr int T_N_BYTES = 4 * T_ATOM_BYTES;            // A tile: 256 features of d_in
-constexpr int T_STAGE_BYTES = T_M_BYTES + T_N_BYTES;   // 48 KB
+constexpr int T_STAGE_BYTES = T_M_BYTES + T_N_BYTES;   // 96 KB
 constexpr uint32_t T_IDESC = idesc_bf16_f32(128, 256, true, true);
 
 struct TileCtl {
@@ -287,11 +289,11 @@ __device__ __forceinline__ TileItem tile_decode(const UmmaParams& P, int item) {
   const int mt = tile / L.tiles_n;
   t.m0 = mt * 128;
   t.n0 = (tile - mt * L.tiles_n) * 256;
-  t.slot = L.partial_base + tile * 4;
+  t.slot = L.partial_base + tile * 8;
   return t;
 }
 
-__global__ void __launch_bounds__(192, 1) k_tile_sqnorm(const __grid_constant__ UmmaParams P) {
+__global__ void __launch_bounds__(T_THREADS, 1) k_tile_sqnorm(const __grid_constant__ UmmaParams P) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* tiles = align1024(smem_raw);
   TileCtl* S = reinterpret_cast<TileCtl*>(tiles + T_STAGES * T_STAGE_BYTES);
@@ -303,7 +305,7 @@ __global__ void __launch_bounds__(192, 1) k_tile_sqnorm(const __grid_constant__ 
       mbar_init(&S->full[s], 1);
       mbar_init(&S->empty[s], 1);
     }
-    for (int b = 0; b < 2; ++b) { mbar_init(&S->tmem_full[b], 1); mbar_init(&S->tmem_empty[b], 4); }
+    for (int b = 0; b < 2; ++b) { mbar_init(&S->tmem_full[b], 1); mbar_init(&S->tmem_empty[b], 8); }
     mbar_init(&S->drain, 1);
     S->abort = 0;
     fence_mbar_init();
@@ -313,7 +315,7 @@ __global__ void __launch_bounds__(192, 1) k_tile_sqnorm(const __grid_constant__ 
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = S->tmem_base;
-  const int n_tb = (P.T + 63) / 64;
+  const int n_tb = (P.T + T_BK - 1) / T_BK;
 
   if (warp == 0) {
     if (lane == 0) {   // ---------------- TMA producer ----------------
@@ -327,10 +329,10 @@ __global__ void __launch_bounds__(192, 1) k_tile_sqnorm(const __grid_constant__ 
           const uint32_t slot = it % T_STAGES, ph = (it / T_STAGES) & 1u;
           if (!mbar_wait(&S->empty[slot], ph ^ 1u, abort_flag, P.status)) { alive = false; break; }
           uint8_t* st = tiles + slot * T_STAGE_BYTES;
-          // two boxes of 64 features x 64 tokens x (2 | 4) feature groups; tokens beyond T arrive as zeros
+          // two boxes of 64 features x 128 tokens x (2 | 4) feature groups; tokens beyond T arrive as zeros
           mbar_arrive_expect_tx(&S->full[slot], (uint32_t)T_STAGE_BYTES);
-          tma_load_4d(st, &L.mapG, &S->full[slot], 0, tb * 64, t.m0 / 64, e);
-          tma_load_4d(st + T_M_BYTES, &L.mapA, &S->full[slot], 0, tb * 64, t.n0 / 64, e);
+          tma_load_4d(st, &L.mapG, &S->full[slot], 0, tb * T_BK, t.m0 / 64, e);
+          tma_load_4d(st + T_M_BYTES, &L.mapA, &S->full[slot], 0, tb * T_BK, t.n0 / 64, e);
           ++it;
         }
       }
@@ -357,12 +359,12 @@ __global__ void __launch_bounds__(192, 1) k_tile_sqnorm(const __grid_constant__ 
           if (!mbar_wait(&S->full[slot], ph, abort_flag, P.status)) { alive = false; break; }
           tc_fence_after();
           const uint32_t am = smem_u32(tiles + slot * T_STAGE_BYTES), an = am + T_M_BYTES;
-          const int left = P.T - tb * 64, nk = left >= 64 ? 4 : (left + 15) >> 4;   // k-steps that hold tokens
+          const int left = P.T - tb * T_BK, nk = left >= T_BK ? T_BK / 16 : (left + 15) >> 4;   // k-steps that hold tokens
 #pragma unroll
-          for (int k4 = 0; k4 < 4; ++k4) {
-            if (k4 < nk)
-              umma_bf16(d_tmem, smem_desc_sw128(am + k4 * 2048, T_ATOM_BYTES, 1024),
-                        smem_desc_sw128(an + k4 * 2048, T_ATOM_BYTES, 1024), T_IDESC, first | (uint32_t)k4);
+          for (int k8 = 0; k8 < T_BK / 16; ++k8) {
+            if (k8 < nk)
+              umma_bf16(d_tmem, smem_desc_sw128(am + k8 * 2048, T_ATOM_BYTES, 1024),
+                        smem_desc_sw128(an + k8 * 2048, T_ATOM_BYTES, 1024), T_IDESC, first | (uint32_t)k8);
           }
           first = 1;
           umma_commit(&S->empty[slot]);
@@ -372,8 +374,8 @@ __global__ void __launch_bounds__(192, 1) k_tile_sqnorm(const __grid_constant__ 
       umma_commit(&S->drain);
       mbar_wait_drain(&S->drain, 0u, P.status);
     }
-  } else if (warp < 6) {   // ---------------- epilogue warps 2..5 ----------------
-    const uint32_t q = (uint32_t)warp & 3u;
+  } else {   // ---------------- epilogue warps 2..9: lanes [32 q, +32), accumulator columns [128 h, +128) ----------------
+    const uint32_t q = (uint32_t)warp & 3u, h = warp >= 6 ? 1u : 0u;
     uint32_t tile_it = 0;
     bool alive = true;
     for (int item = blockIdx.x; item < P.total_items; item += gridDim.x, ++tile_it) {
@@ -384,9 +386,9 @@ __global__ void __launch_bounds__(192, 1) k_tile_sqnorm(const __grid_constant__ 
       tc_fence_after();
       float sum = 0.0f;
 #pragma unroll 1
-      for (int ch = 0; ch < 8; ++ch) {
+      for (int ch = 0; ch < 4; ++ch) {
         uint32_t v[32];
-        tmem_ld_32x32(tmem_base + ((q * 32u) << 16) + buf * 256u + (uint32_t)ch * 32u, v);
+        tmem_ld_32x32(tmem_base + ((q * 32u) << 16) + buf * 256u + h * 128u + (uint32_t)ch * 32u, v);
         tmem_ld_wait();
 #pragma unroll
           for (int j = 0; j < 32; ++j) sum = fmaf(__uint_as_float(v[j]), __uint_as_float(v[j]), sum);
@@ -396,7 +398,7 @@ __global__ void __launch_bounds__(192, 1) k_tile_sqnorm(const __grid_constant__ 
       if (lane == 0) mbar_arrive(&S->tmem_empty[buf]);
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) sum += __shfl_down_sync(0xffffffffu, sum, o);
-      if (lane == 0) P.partial[(size_t)t.e * P.partial_stride + t.slot + (int)q] = sum;
+      if (lane == 0) P.partial[(size_t)t.e * P.partial_stride + t.slot + (int)(h * 4u + q)] = sum;
     }
   }
   tc_fence_before();
@@ -755,7 +757,8 @@ static int tile_count(const dp_layer& L) { return ceil_div(L.d_out, 128) * ceil_
 
 size_t umma_sqnorm_partials_per_example(const dp_layer* layers, const int* idx, int n, const int* use_gram) {
   size_t c = 0;
-  for (int k = 0; k < n; ++k) c += 4 * (size_t)(use_gram[k] ? gram_pairs(layers[idx[k]].T) : tile_count(layers[idx[k]]));
+  for (int k = 0; k < n; ++k)
+    c += use_gram[k] ? 4 * (size_t)gram_pairs(layers[idx[k]].T) : 8 * (size_t)tile_count(layers[idx[k]]);
   return c;
 }
 
@@ -812,7 +815,7 @@ int launch_umma_sqnorms(const dp_layer* layers, const int* idx, int n, const int
   int pos = partial_base;
   for (int k = 0; k < n; ++k) {
     base[k] = pos;
-    pos += 4 * (use_gram[k] ? gram_pairs(T) : tile_count(layers[idx[k]]));
+    pos += use_gram[k] ? 4 * gram_pairs(T) : 8 * tile_count(layers[idx[k]]);
   }
   for (int pass = 0; pass < 2; ++pass) {             // pass 0: Gram layers, pass 1: materialised tiles
     const bool gram = pass == 0;
@@ -827,7 +830,7 @@ int launch_umma_sqnorms(const dp_layer* layers, const int* idx, int n, const int
         const long long add = (long long)B * (gram ? gram_pairs(T) : tile_count(L));
         if (items + add > 0x7fffffffll) break;
         UmmaLayer& U = P.L[P.n_layers];
-        if (!(gram ? fill_layer(U, L, 128) : fill_layer(U, L, 64, 2, 4))) return DP_ERR_CUDA;
+        if (!(gram ? fill_layer(U, L, 128) : fill_layer(U, L, T_BK, 2, 4))) return DP_ERR_CUDA;
         U.item_start = (int)items;
         U.partial_base = base[k];
         items += add;
@@ -846,7 +849,7 @@ int launch_umma_sqnorms(const dp_layer* layers, const int* idx, int n, const int
       P.status = status;
       const int grid = P.total_items < sm_count() ? P.total_items : sm_count();
       if (gram) k_gram_sqnorm<<<grid, G_THREADS, G_SMEM, s>>>(P);
-      else      k_tile_sqnorm<<<grid, 192, T_SMEM, s>>>(P);
+      else      k_tile_sqnorm<<<grid, T_THREADS, T_SMEM, s>>>(P);
       if (counted(1) != cudaSuccess) return DP_ERR_CUDA;
     }
   }
