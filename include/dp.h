@@ -151,6 +151,26 @@ DP_API int dp_noise_scale_adamw_step_snr(float* theta, float* m, float* v, float
                                          double xi, double weight_decay, int64_t t, double* sq_sums,
                                          void* cuda_stream);
 
+/* Data-parallel end of a macro-batch in one pass (the gradient reduction that Section 5.3's large batches
+ * amortise, fused with the g_t ... theta_t lines of Algorithm 1).  Every rank holds a full fp32 accumulator and a
+ * full replica of theta; rank k owns the shard [elem_offset, elem_offset + n) of the flat vector and calls this
+ * with pointers to the START OF THAT SHARD:
+ *   theta, m, v        this rank's own shard (read and written);
+ *   acc_of_rank[r]     the shard inside rank r's accumulator, r < n_ranks <= 16 (HOST array of device pointers
+ *                      that this GPU can load from and store to: its own memory or peer-mapped memory);
+ *   theta_of_rank[r]   the shard inside rank r's replica, or NULL entries / a NULL array to skip the write.
+ * Computes g = (sum_r acc_r + sigma C z) / batch_size with the sum taken in rank order and z keyed by the global
+ * element index (so the result is that of the single-GPU fused call on the summed accumulator), applies AdamW,
+ * stores the new theta into every replica given and, if zero_acc, zeroes the shard of every accumulator.
+ * The kernel waits for nobody: the caller orders it after all ranks' accumulate calls and orders any reader of
+ * theta or writer of the accumulators on any rank after it (a barrier between the ranks on both sides).
+ * elem_offset must be a multiple of 4 and every pointer 16-byte aligned (DP_ERR_ALIGN otherwise). */
+DP_API int dp_reduce_noise_adamw_step(float* theta, float* m, float* v, float* const* acc_of_rank /*HOST*/,
+                                      float* const* theta_of_rank /*HOST or NULL*/, int n_ranks, int zero_acc,
+                                      int64_t n, int64_t elem_offset, double sigma, double C, int64_t batch_size,
+                                      uint64_t seed, uint64_t step, double lr, double beta1, double beta2, double xi,
+                                      double weight_decay, int64_t t, void* cuda_stream);
+
 /* Clipping statistics of a microbatch (the other diagnostic that accompanies the gradient-SNR curves of
  * Section 5.2.1): out[0] = fraction of examples with clip_i < 1, out[1] = mean clip_i.  out: device float[2]. */
 DP_API int dp_clip_stats(const float* clip, int B, float* out, void* cuda_stream);

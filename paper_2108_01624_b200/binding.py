@@ -22,7 +22,7 @@ DP_F32, DP_BF16 = 0, 1
 DP_PATH_AUTO, DP_PATH_GRAM, DP_PATH_MATERIALIZED = 0, 1, 2
 _KINDS = {"linear": DP_LINEAR, "layernorm": DP_LAYERNORM, "embedding": DP_EMBEDDING}
 
-EXPORTS = ["dp_workspace_bytes", "dp_per_example_sqnorms", "dp_clip_factors", "dp_clipped_accumulate", "dp_clipped_accumulate_after_sqnorms", "dp_accumulate_schedule",
+EXPORTS = ["dp_workspace_bytes", "dp_per_example_sqnorms", "dp_clip_factors", "dp_clipped_accumulate", "dp_clipped_accumulate_after_sqnorms", "dp_accumulate_schedule", "dp_reduce_noise_adamw_step",
            "dp_add_noise_and_scale", "dp_adamw_step", "dp_noise_scale_adamw_step", "dp_noise_scale_adamw_step_snr",
            "dp_clip_stats", "dp_philox_u32",
            "dp_token_equality_mask", "dp_layernorm_sqnorms_static", "dp_poll_status", "dp_last_timeout_info", "dp_launch_count",
@@ -65,6 +65,8 @@ def lib() -> C.CDLL:
         L.dp_adamw_step.argtypes = [vp, vp, vp, vp, i64, f32, f32, f32, f32, f32, i64, vp]
         L.dp_noise_scale_adamw_step.argtypes = [vp, vp, vp, vp, i32, i64, i64, f32, f32, i64, u64, u64,
                                                 f32, f32, f32, f32, f32, i64, vp]
+        L.dp_reduce_noise_adamw_step.argtypes = [vp, vp, vp, vp, vp, i32, i32, i64, i64, f32, f32, i64, u64, u64,
+                                                 f32, f32, f32, f32, f32, i64, vp]
         L.dp_noise_scale_adamw_step_snr.argtypes = [vp, vp, vp, vp, i32, i64, i64, f32, f32, i64, u64, u64,
                                                     f32, f32, f32, f32, f32, i64, vp, vp]
         L.dp_clip_stats.argtypes = [vp, i32, vp, vp]
@@ -241,6 +243,24 @@ def dp_noise_scale_adamw_step_snr(theta, m, v, acc, zero_acc, sigma, C_, batch_s
                                                int(batch_size), int(seed), int(step), float(lr), float(beta1),
                                                float(beta2), float(xi), float(weight_decay), int(t),
                                                _ptr(sq_sums), _stream(stream)))
+
+
+def dp_reduce_noise_adamw_step(theta, m, v, acc_shards, theta_shards, zero_acc, sigma, C_, batch_size, seed, step, lr,
+                               beta1, beta2, xi, weight_decay, t, elem_offset: int = 0, stream=None) -> None:
+    """Fused cross-rank sum + noise + AdamW on one shard.  acc_shards: one entry per rank, the shard inside that
+    rank's accumulator (a tensor, or a raw device address for peer-mapped memory); theta_shards: the shard inside
+    every rank's replica of theta, entries may be None (or the whole argument None) to skip the write."""
+    def addr(x):
+        return 0 if x is None else (int(x) if isinstance(x, int) else x.data_ptr())
+    R = len(acc_shards)
+    acc_arr = (C.c_void_p * R)(*[addr(a) for a in acc_shards])
+    th_arr = None if theta_shards is None else (C.c_void_p * R)(*[addr(x) for x in theta_shards])
+    _check("dp_reduce_noise_adamw_step",
+           lib().dp_reduce_noise_adamw_step(_ptr(theta), _ptr(m), _ptr(v), C.cast(acc_arr, C.c_void_p),
+                                            None if th_arr is None else C.cast(th_arr, C.c_void_p), R,
+                                            int(bool(zero_acc)), theta.numel(), int(elem_offset), float(sigma),
+                                            float(C_), int(batch_size), int(seed), int(step), float(lr), float(beta1),
+                                            float(beta2), float(xi), float(weight_decay), int(t), _stream(stream)))
 
 
 def dp_clip_stats(clip: torch.Tensor, out: torch.Tensor, stream=None) -> torch.Tensor:

@@ -355,6 +355,30 @@ int dp_noise_scale_adamw_step_snr(float* theta, float* m, float* v, float* acc, 
   return DP_OK;
 }
 
+int dp_reduce_noise_adamw_step(float* theta, float* m, float* v, float* const* acc_of_rank,
+                               float* const* theta_of_rank, int n_ranks, int zero_acc, int64_t n, int64_t elem_offset,
+                               double sigma, double C, int64_t batch_size, uint64_t seed, uint64_t step, double lr,
+                               double beta1, double beta2, double xi, double weight_decay, int64_t t,
+                               void* cuda_stream) {
+  NoiseArgs na;
+  AdamArgs aa;
+  int rc = make_noise_args(n, elem_offset, sigma, C, batch_size, seed, step, &na);
+  if (rc != DP_OK) return rc;
+  if ((rc = make_adam_args(lr, beta1, beta2, xi, weight_decay, t, &aa)) != DP_OK) return rc;
+  if (n_ranks < 1 || n_ranks > kMaxRanks || !acc_of_rank) return DP_ERR_ARG;
+  if (n == 0) return DP_OK;
+  if (!theta || !m || !v) return DP_ERR_ARG;
+  if ((elem_offset & 3) != 0 || misaligned(theta, 16) || misaligned(m, 16) || misaligned(v, 16)) return DP_ERR_ALIGN;
+  for (int r = 0; r < n_ranks; ++r) {
+    if (!acc_of_rank[r]) return DP_ERR_ARG;
+    if (misaligned(acc_of_rank[r], 16)) return DP_ERR_ALIGN;
+    if (theta_of_rank && theta_of_rank[r] && misaligned(theta_of_rank[r], 16)) return DP_ERR_ALIGN;
+  }
+  DP_CUDA(launch_reduce_update(theta, m, v, acc_of_rank, theta_of_rank, n_ranks, zero_acc, n, na, aa,
+                               static_cast<cudaStream_t>(cuda_stream)));
+  return DP_OK;
+}
+
 int dp_clip_stats(const float* clip, int B, float* out, void* cuda_stream) {
   if (!clip || !out || B <= 0) return DP_ERR_ARG;
   if (misaligned(clip, 4) || misaligned(out, 4)) return DP_ERR_ALIGN;

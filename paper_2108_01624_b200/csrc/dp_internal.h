@@ -41,6 +41,11 @@ cudaError_t launch_adamw(float* theta, float* m, float* v, const float* g, long 
 // sq_sums (optional, device double[2]): adds sum(acc^2) and sum((sigma C z)^2), the gradient-SNR terms.
 cudaError_t launch_noise_adamw(float* theta, float* m, float* v, float* acc, int zero_acc, long long n,
                                const NoiseArgs& na, const AdamArgs& aa, cudaStream_t s, double* sq_sums = nullptr);
+// Fused cross-rank sum + noise + AdamW + replica update on one shard (elem_offset % 4 == 0, 16-byte aligned pointers).
+constexpr int kMaxRanks = 16;
+cudaError_t launch_reduce_update(float* theta, float* m, float* v, float* const* acc_of_rank,
+                                 float* const* theta_of_rank, int n_ranks, int zero_acc, long long n,
+                                 const NoiseArgs& na, const AdamArgs& aa, cudaStream_t s);
 cudaError_t launch_clip_stats(const float* clip, int B, float* out, cudaStream_t s);
 cudaError_t launch_philox_u32(uint32_t* out, long long n, const NoiseArgs& na, cudaStream_t s);
 cudaError_t launch_equality_mask(const int32_t* ids, int B, int T, uint8_t* mask, cudaStream_t s);

@@ -213,6 +213,84 @@ cudaError_t launch_noise_adamw(float* theta, float* m, float* v, float* acc, int
   return launch_stream<2>(theta, m, v, acc, nullptr, zero_acc, n, na, aa, s, sq_sums);
 }
 
+// ---------------------------------------------------------------------------------------------
+// Macro-batch end of the data-parallel scheme in one pass over one shard of the flat vector:
+//   g = (sum over ranks of acc_r + sigma C z) / N, AdamW on this rank's theta / m / v, the new theta written into
+//   every rank's replica, every rank's accumulator shard zeroed.
+// The ranks' buffers are reached through plain loads and stores on peer-mapped addresses (no multicast, no
+// waiting on another rank inside the kernel: the caller orders the launches against the accumulate kernels of all
+// ranks).  The sum runs over the ranks in index order, so it does not depend on which rank computes it.
+// ---------------------------------------------------------------------------------------------
+struct PeerSet {
+  float* acc[kMaxRanks];       // shard start in rank r's accumulator
+  float* theta[kMaxRanks];     // shard start in rank r's parameter replica (nullptr: not written)
+  int n_ranks;
+};
+
+__global__ void __launch_bounds__(256)
+k_reduce_update(float* __restrict__ theta, float* __restrict__ m, float* __restrict__ v, const PeerSet P, int zero_acc,
+                long long n, unsigned long long j0, unsigned long long n_blocks, NoiseArgs na, AdamArgs aa) {
+  const unsigned long long stride = (unsigned long long)gridDim.x * blockDim.x;
+  for (unsigned long long b = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x; b < n_blocks; b += stride) {
+    const unsigned long long j = j0 + b;
+    const long long k0 = (long long)(4ull * j) - na.elem_offset;   // local index of lane 0 (a multiple of 4)
+    const float4 z = normals4(j, na);
+    if (k0 >= 0 && k0 + 4 <= n) {
+      float4 a4 = make_float4(0.f, 0.f, 0.f, 0.f);
+      for (int r = 0; r < P.n_ranks; ++r) {
+        const float4 x = *reinterpret_cast<const float4*>(P.acc[r] + k0);
+        a4.x += x.x; a4.y += x.y; a4.z += x.z; a4.w += x.w;
+      }
+      float4 t4 = *reinterpret_cast<const float4*>(theta + k0);
+      float4 m4 = *reinterpret_cast<const float4*>(m + k0);
+      float4 v4 = *reinterpret_cast<const float4*>(v + k0);
+      adam_update(t4.x, m4.x, v4.x, (a4.x + na.sigmaC * z.x) * na.inv_n, aa);
+      adam_update(t4.y, m4.y, v4.y, (a4.y + na.sigmaC * z.y) * na.inv_n, aa);
+      adam_update(t4.z, m4.z, v4.z, (a4.z + na.sigmaC * z.z) * na.inv_n, aa);
+      adam_update(t4.w, m4.w, v4.w, (a4.w + na.sigmaC * z.w) * na.inv_n, aa);
+      *reinterpret_cast<float4*>(theta + k0) = t4;
+      *reinterpret_cast<float4*>(m + k0) = m4;
+      *reinterpret_cast<float4*>(v + k0) = v4;
+      for (int r = 0; r < P.n_ranks; ++r) {
+        if (P.theta[r] && P.theta[r] != theta) *reinterpret_cast<float4*>(P.theta[r] + k0) = t4;
+        if (zero_acc) *reinterpret_cast<float4*>(P.acc[r] + k0) = make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+    } else {
+      const float zz[4] = {z.x, z.y, z.z, z.w};
+#pragma unroll
+      for (int l = 0; l < 4; ++l) {
+        const long long k = k0 + l;
+        if (k < 0 || k >= n) continue;
+        float a1 = 0.0f;
+        for (int r = 0; r < P.n_ranks; ++r) a1 += P.acc[r][k];
+        float t1 = theta[k], m1 = m[k], v1 = v[k];
+        adam_update(t1, m1, v1, (a1 + na.sigmaC * zz[l]) * na.inv_n, aa);
+        theta[k] = t1; m[k] = m1; v[k] = v1;
+        for (int r = 0; r < P.n_ranks; ++r) {
+          if (P.theta[r] && P.theta[r] != theta) P.theta[r][k] = t1;
+          if (zero_acc) P.acc[r][k] = 0.0f;
+        }
+      }
+    }
+  }
+}
+
+cudaError_t launch_reduce_update(float* theta, float* m, float* v, float* const* acc_of_rank,
+                                 float* const* theta_of_rank, int n_ranks, int zero_acc, long long n,
+                                 const NoiseArgs& na, const AdamArgs& aa, cudaStream_t s) {
+  if (n <= 0) return cudaSuccess;
+  PeerSet P;
+  P.n_ranks = n_ranks;
+  for (int r = 0; r < kMaxRanks; ++r) {
+    P.acc[r] = r < n_ranks ? acc_of_rank[r] : nullptr;
+    P.theta[r] = (r < n_ranks && theta_of_rank) ? theta_of_rank[r] : nullptr;
+  }
+  const unsigned long long j0 = (unsigned long long)na.elem_offset >> 2;
+  const unsigned long long j1 = ((unsigned long long)na.elem_offset + (unsigned long long)n + 3ull) >> 2;
+  k_reduce_update<<<stream_grid(j1 - j0), 256, 0, s>>>(theta, m, v, P, zero_acc, n, j0, j1 - j0, na, aa);
+  return counted(1);
+}
+
 // out[0] = fraction of examples with clip < 1, out[1] = mean clip factor.  One block, fixed order.
 __global__ void __launch_bounds__(256) k_clip_stats(const float* __restrict__ clip, int B, float* __restrict__ out) {
   __shared__ float red[2][8];

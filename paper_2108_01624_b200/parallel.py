@@ -31,13 +31,27 @@ class ShardedUpdate:
     t, examples_seen (already the global count) and the hyper-parameters.
     """
 
-    def __init__(self, state, dist, world: int, rank: int, update_fn: Optional[Callable] = None):
+    def __init__(self, state, dist, world: int, rank: int, update_fn: Optional[Callable] = None,
+                 peer_acc=None, peer_theta=None, fused_fn: Optional[Callable] = None):
+        """peer_acc / peer_theta (optional, one entry per rank): every rank's full accumulator and full replica of
+        theta as this GPU can address them (tensors, or raw device addresses of peer-mapped memory, e.g. the
+        buffer pointers of a symmetric-memory rendezvous).  With both given, the macro-batch ends with ONE kernel
+        per rank that sums the shard over all ranks, applies noise + AdamW and writes theta into every replica
+        (`fused_fn`, by default the library's dp_reduce_noise_adamw_step), between two barriers."""
         self.state, self.dist, self.world, self.rank = state, dist, world, rank
+        self.peer_acc, self.peer_theta = peer_acc, peer_theta
+        self.fused_fn = fused_fn or self._fused_reduce_kernel
+        if (peer_acc is None) != (peer_theta is None):
+            raise ValueError("peer_acc and peer_theta go together")
+        if peer_acc is not None and (len(peer_acc) != world or len(peer_theta) != world):
+            raise ValueError("one accumulator and one replica per rank")
         self.lo, self.hi = shard_bounds(state.acc.numel(), world, rank)
         self.per = shard_bounds(state.acc.numel(), world, 0)[1]
-        self.padded = torch.zeros(self.per * world, dtype=state.acc.dtype, device=state.acc.device)
         self.update_fn = update_fn or self._fused_kernel
         self.use_reduce_scatter = dist.get_backend() == "nccl"
+        # staging for the collectives of the two-step path (the fused path reads the peers' buffers in place)
+        self.padded = None if peer_acc is not None else torch.zeros(self.per * world, dtype=state.acc.dtype,
+                                                                     device=state.acc.device)
 
     def _fused_kernel(self, theta, m, v, acc, elem_offset, batch_size, t):
         from . import binding as b
@@ -45,7 +59,30 @@ class ShardedUpdate:
         b.dp_noise_scale_adamw_step(theta, m, v, acc, True, s.sigma, s.C, batch_size, s.seed, t, s.lr, s.beta1,
                                     s.beta2, s.xi, s.weight_decay, t, elem_offset)
 
+    def _fused_reduce_kernel(self, theta, m, v, acc_shards, theta_shards, elem_offset, batch_size, t):
+        from . import binding as b
+        s = self.state
+        b.dp_reduce_noise_adamw_step(theta, m, v, acc_shards, theta_shards, True, s.sigma, s.C, batch_size, s.seed, t,
+                                     s.lr, s.beta1, s.beta2, s.xi, s.weight_decay, t, elem_offset)
+
+    @staticmethod
+    def _shard_of(buf, lo, hi):
+        return buf + 4 * lo if isinstance(buf, int) else buf[lo:hi]      # fp32: 4 bytes per element
+
+    def _finish_fused(self):
+        s, dist = self.state, self.dist
+        s.t += 1
+        lo, hi = self.lo, self.hi
+        dist.barrier()          # stream-ordered: every rank's accumulate kernels precede the reads below
+        if hi > lo:
+            self.fused_fn(s.theta[lo:hi], s.m[lo:hi], s.v[lo:hi], [self._shard_of(a, lo, hi) for a in self.peer_acc],
+                          [self._shard_of(t, lo, hi) for t in self.peer_theta], lo, s.examples_seen, s.t)
+        dist.barrier()          # every shard of every replica is written, every accumulator is zero
+        s.examples_seen = 0
+
     def finish_macro_batch(self):
+        if self.peer_acc is not None:
+            return self._finish_fused()
         s, dist = self.state, self.dist
         n = s.acc.numel()
         s.t += 1

@@ -154,3 +154,23 @@ def test_accumulate_schedule_splits_large_groups_and_launches(lib):
     assert rc == 1 and start[1] == -1 and launch[1] == -1
     # argument checks
     assert lib.dp_accumulate_schedule(C.cast(L, C.c_void_p), 2, 0, 256, 256, 256, 256, 1) == -1
+
+
+def test_fused_cross_rank_update_argument_checks(lib):
+    ptrs2 = (C.c_void_p * 2)(4096, 8192)
+    p2 = C.cast(ptrs2, C.c_void_p)
+    ok = dict(n_ranks=2, zero=1, n=8, off=0)
+    def call(theta=256, m=512, v=768, acc=p2, th=None, n_ranks=2, n=8, off=0, lr=1e-3, t=1):
+        return lib.dp_reduce_noise_adamw_step(theta, m, v, acc, th, n_ranks, 1, n, off, 1.0, 1.0, 4, 0, 0, lr, 0.9, 0.999,
+                                              1e-11, 0.0, t, None)
+    assert call(acc=None) == -1
+    assert call(n_ranks=0) == -1 and call(n_ranks=17) == -1
+    assert call(t=0) == -1 and call(lr=float("nan")) == -1
+    assert call(n=0) == 0                                   # empty shard: nothing to do
+    assert call(theta=None) == -1
+    assert call(off=2) == -2                                # shard must start on a Philox block
+    assert call(theta=260) == -2                            # 16-byte alignment of every pointer
+    bad = (C.c_void_p * 2)(4096, 8196)
+    assert call(acc=C.cast(bad, C.c_void_p)) == -2
+    null = (C.c_void_p * 2)(4096, None)
+    assert call(acc=C.cast(null, C.c_void_p)) == -1

@@ -94,3 +94,73 @@ def test_shard_bounds_cover_and_align():
             for (a, b_), (c, d) in zip(spans[:-1], spans[1:]):
                 assert b_ == c and a <= b_
             assert all(lo % 4 == 0 or lo == n for lo, _ in spans)
+
+
+def _oracle_fused(state):
+    """CPU stand-in for dp_reduce_noise_adamw_step: rank-ordered sum of the accumulator shards, noise + AdamW,
+    theta into every replica, accumulator shards zeroed."""
+    from oracle import dp_oracle as O
+
+    def fn(theta, m, v, acc_shards, theta_shards, elem_offset, batch_size, t):
+        total = np.zeros(theta.numel())
+        for a in acc_shards:
+            total += a.numpy()
+        g = O.add_noise_and_scale(total, state.sigma, state.C, batch_size, state.seed, t, elem_offset)
+        th, mm, vv = O.adamw_step(theta.numpy(), m.numpy(), v.numpy(), g, state.lr, state.beta1, state.beta2,
+                                  state.xi, state.weight_decay, t)
+        m.copy_(torch.from_numpy(mm)); v.copy_(torch.from_numpy(vv))
+        for ts in theta_shards:
+            ts.copy_(torch.from_numpy(th))
+        for a in acc_shards:
+            a.zero_()
+    return fn
+
+
+def _fused_worker(rank, world, port, n, accs, thetas, out_dir):
+    """accs / thetas live in shared memory: every process addresses every rank's buffers, as peer-mapped GPU
+    memory would be."""
+    sys.path.insert(0, ROOT)
+    import torch.distributed as dist
+    from paper_2108_01624_b200.parallel import ShardedUpdate
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    g = torch.Generator().manual_seed(100 + rank)
+    local_acc = torch.randn(n, generator=g, dtype=torch.float64)
+    st = _State(n, local_acc)
+    st.acc, st.theta = accs[rank], thetas[rank]          # this rank's buffers are the shared ones
+    st.theta.copy_(torch.linspace(-1, 1, n, dtype=torch.float64))
+    sh = ShardedUpdate(st, dist, world, rank, peer_acc=accs, peer_theta=thetas, fused_fn=_oracle_fused(st))
+    for step in range(2):
+        st.acc.copy_(local_acc * (step + 1))
+        st.examples_seen = 64 * world
+        sh.finish_macro_batch()
+        assert st.examples_seen == 0 and st.t == step + 1
+    torch.save({"theta": st.theta.clone(), "acc": st.acc.clone(), "lo": sh.lo, "hi": sh.hi, "m": st.m},
+               f"{out_dir}/f{rank}.pt")
+    dist.destroy_process_group()
+
+
+@pytest.mark.parametrize("world,n", [(2, 1003), (3, 64)])
+def test_fused_peer_memory_update_equals_single_process(world, n, tmp_path):
+    accs = [torch.zeros(n, dtype=torch.float64).share_memory_() for _ in range(world)]
+    thetas = [torch.zeros(n, dtype=torch.float64).share_memory_() for _ in range(world)]
+    mp.spawn(_fused_worker, args=(world, _free_port(), n, accs, thetas, str(tmp_path)), nprocs=world, join=True)
+    outs = [torch.load(f"{tmp_path}/f{r}.pt") for r in range(world)]
+    src = [torch.randn(n, generator=torch.Generator().manual_seed(100 + r), dtype=torch.float64) for r in range(world)]
+    st = _State(n, sum(src))
+    fn = _oracle_update(st)
+    for step in range(2):
+        st.t += 1
+        fn(st.theta, st.m, st.v, (sum(src) * (step + 1)).clone(), 0, 64 * world, st.t)
+    for o in outs:
+        np.testing.assert_allclose(o["theta"].numpy(), st.theta.numpy(), rtol=1e-12, atol=1e-14)
+        assert float(o["acc"].abs().max()) == 0.0
+        np.testing.assert_allclose(o["m"][o["lo"]:o["hi"]].numpy(), st.m[o["lo"]:o["hi"]].numpy(), rtol=1e-12)
+
+
+def test_peer_buffers_given_as_addresses():
+    from paper_2108_01624_b200.parallel import ShardedUpdate
+    assert ShardedUpdate._shard_of(4096, 8, 16) == 4096 + 32
+    t = torch.arange(20.0)
+    assert torch.equal(ShardedUpdate._shard_of(t, 8, 16), t[8:16])

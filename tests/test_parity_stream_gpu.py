@@ -207,3 +207,50 @@ def test_clip_stats_matches_checker():
         out = torch.empty(2, dtype=torch.float32, device=DEV)
         b.dp_clip_stats(clip, out)
         np.testing.assert_allclose(to_np(out), O.clip_stats(to_np(clip)), rtol=1e-5)
+
+
+@pytest.mark.parametrize("n_flat,world", [(40_003, 3), (1 << 18, 8), (7, 2)])
+def test_fused_cross_rank_update_matches_checker(n_flat, world):
+    """Virtual ranks on one GPU: every rank has a full accumulator and a full replica of theta; the shard owners
+    run dp_reduce_noise_adamw_step one after the other (no launch waits for another).  Afterwards every replica
+    holds the checker's update of the SUMMED accumulator and every accumulator is zero."""
+    from paper_2108_01624_b200.parallel import shard_bounds
+    rng = np.random.default_rng(n_flat + world)
+    hp = dict(sigma=0.9, C=0.5, N=4096, seed=0x1234567, step=5, lr=1e-3, b1=0.9, b2=0.999, xi=1e-11, wd=0.1, t=3)
+    accs = [rng.standard_normal(n_flat).astype(np.float32) for _ in range(world)]
+    th0 = rng.standard_normal(n_flat).astype(np.float32)
+    m0 = (rng.standard_normal(n_flat) * 0.1).astype(np.float32)
+    v0 = (rng.random(n_flat) * 0.01).astype(np.float32)
+    acc_d = [torch.from_numpy(a).to(DEV) for a in accs]
+    th_d = [torch.from_numpy(th0).to(DEV) for _ in range(world)]
+    m_d = [torch.from_numpy(m0).to(DEV) for _ in range(world)]
+    v_d = [torch.from_numpy(v0).to(DEV) for _ in range(world)]
+    for r in range(world):
+        lo, hi = shard_bounds(n_flat, world, r)
+        if hi <= lo:
+            continue
+        b.dp_reduce_noise_adamw_step(th_d[r][lo:hi], m_d[r][lo:hi], v_d[r][lo:hi], [a[lo:hi] for a in acc_d],
+                                     [t[lo:hi] for t in th_d], True, hp["sigma"], hp["C"], hp["N"], hp["seed"],
+                                     hp["step"], hp["lr"], hp["b1"], hp["b2"], hp["xi"], hp["wd"], hp["t"],
+                                     elem_offset=lo)
+    torch.cuda.synchronize()
+    total = np.sum(np.stack([a.astype(np.float64) for a in accs]), axis=0)
+    g = O.add_noise_and_scale(total, hp["sigma"], hp["C"], hp["N"], seed=hp["seed"], step=hp["step"], elem_offset=0)
+    rt, rm, rv = O.adamw_step(th0.astype(np.float64), m0.astype(np.float64), v0.astype(np.float64), g, hp["lr"],
+                              hp["b1"], hp["b2"], hp["xi"], hp["wd"], hp["t"])
+    for r in range(world):
+        assert torch.equal(th_d[r], th_d[0])                      # every replica got the same bits
+        assert float(acc_d[r].abs().max()) == 0.0
+        lo, hi = shard_bounds(n_flat, world, r)
+        if hi > lo:
+            assert rel_max(to_np(m_d[r][lo:hi]), rm[lo:hi]) <= F32_TOL
+            assert rel_max(to_np(v_d[r][lo:hi]), rv[lo:hi]) <= F32_TOL
+    d, rd = to_np(th_d[0]) - th0, rt - th0
+    assert np.max(np.abs(d - rd)) <= F32_TOL * np.max(np.abs(rd)) + 1e-7 * np.max(np.abs(th0))
+    # and it is the single-GPU fused call on the summed accumulator, bit for bit, when the sum is exact
+    if world == 2:
+        th1, m1, v1 = (torch.from_numpy(x).to(DEV) for x in (th0, m0, v0))
+        s = torch.from_numpy(accs[0]).to(DEV) + torch.from_numpy(accs[1]).to(DEV)
+        b.dp_noise_scale_adamw_step(th1, m1, v1, s, True, hp["sigma"], hp["C"], hp["N"], hp["seed"], hp["step"],
+                                    hp["lr"], hp["b1"], hp["b2"], hp["xi"], hp["wd"], hp["t"], 0)
+        assert torch.equal(th1, th_d[0])
