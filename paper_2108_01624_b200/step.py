@@ -117,6 +117,20 @@ class DPStep:
             self.acc.zero_()
         self.examples_seen = 0
 
+    def state_dict(self) -> dict:
+        """Everything a run needs to resume in the middle of a macro-batch: parameters, Adam moments, the partly
+        filled accumulator, the macro-step counter (which also keys the noise) and the examples seen so far.
+        The noise generator is counter-based, so a resumed run draws exactly the noise the original would have."""
+        return {"theta": self.theta.clone(), "m": self.m.clone(), "v": self.v.clone(), "acc": self.acc.clone(),
+                "t": self.t, "examples_seen": self.examples_seen, "seed": self.seed, "n_flat": self.n_flat}
+
+    def load_state_dict(self, state: dict) -> None:
+        if int(state["n_flat"]) != self.n_flat:
+            raise ValueError("state belongs to another parameter layout")
+        for name in ("theta", "m", "v", "acc"):
+            getattr(self, name).copy_(state[name])
+        self.t, self.examples_seen, self.seed = int(state["t"]), int(state["examples_seen"]), int(state["seed"])
+
     def gradient_snr(self) -> float:
         """||aggregated clipped gradient|| / ||noise vector|| of the last finished macro-batch (host sync)."""
         if self.sq_sums is None:

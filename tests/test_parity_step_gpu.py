@@ -80,3 +80,80 @@ def test_bert_input_layer_three_embeddings():
     n1, _, _ = gpu_norms_clip(ll1, 1.0)
     np.testing.assert_allclose(to_np(n1), (G ** 2).sum((1, 2)), rtol=2e-3)
     assert b.dp_poll_status() == 0
+
+
+def test_checkpoint_resume_in_the_middle_of_a_macro_batch(tmp_path):
+    """Save after two of three microbatches, reload into a fresh object, finish: the linear and LayerNorm tensors
+    are bit-identical to the uninterrupted run (one owner per element and launch), the embedding rows agree within
+    fp32 atomics order, and the noise is the same draw (counter-based generator keyed by seed, step, element)."""
+    wl = synth.workload("bert_base_layer")
+    specs = list(wl.specs) + [synth.LayerSpec(synth.EMBEDDING, 300, 768, False, "emb")]
+    mk = lambda: DPStep(specs, DEV, wl.C, wl.sigma, wl.lr, wl.beta1, wl.beta2, wl.xi, wl.weight_decay, seed=9)
+    wl2 = synth.Workload("ckpt", 8, 64, torch.bfloat16, specs)
+    mbs = [synth.generate(wl2, seed=4, device=DEV, microbatch=k) for k in range(3)]
+    th0 = synth.initial_weights(mk().n_flat, 1, DEV)
+
+    full = mk()
+    full.theta.copy_(th0)
+    for d in mbs:
+        full.accumulate_microbatch(full.layer_list(d))
+    full.finish_macro_batch()
+
+    first = mk()
+    first.theta.copy_(th0)
+    for d in mbs[:2]:
+        first.accumulate_microbatch(first.layer_list(d))
+    torch.save(first.state_dict(), tmp_path / "ckpt.pt")
+    resumed = mk()
+    resumed.load_state_dict(torch.load(tmp_path / "ckpt.pt"))
+    assert resumed.examples_seen == 16 and resumed.t == 0
+    resumed.accumulate_microbatch(resumed.layer_list(mbs[2]))
+    resumed.finish_macro_batch()
+    torch.cuda.synchronize()
+    assert b.dp_poll_status() == 0
+    emb_lo = full.offsets[-1][0]
+    assert torch.equal(resumed.theta[:emb_lo], full.theta[:emb_lo])
+    assert torch.equal(resumed.m[:emb_lo], full.m[:emb_lo]) and torch.equal(resumed.v[:emb_lo], full.v[:emb_lo])
+    assert rel_l2(to_np(resumed.m[emb_lo:]), to_np(full.m[emb_lo:])) <= 1e-6
+    assert resumed.t == full.t == 1 and resumed.examples_seen == 0
+
+
+def test_outputs_stay_inside_their_buffers_and_repeat_bit_for_bit():
+    """Canary words around the accumulators, the norms and the clip factors survive a full microbatch, and a
+    second run of the same calls gives the same bits (the only order-dependent adds, the embedding atomics,
+    are left out of this list)."""
+    wl = synth.workload("bert_base_layer")
+    wl2 = synth.Workload("canary", 5, 100, torch.bfloat16, wl.specs)
+    data = synth.generate(wl2, seed=6, device=DEV)
+    results = []
+    for rep in range(2):
+        pad = 64
+        accs, raws = [], []
+        for ld in data:
+            acc = []
+            for shp in ([(ld.spec.d_in, ld.spec.d_out)] + ([(ld.spec.d_out,)] if ld.spec.has_bias else [])
+                        if ld.spec.kind == synth.LINEAR else [(ld.spec.d_out,), (ld.spec.d_out,)]):
+                n = int(np.prod(shp))
+                raw = torch.full((n + 2 * pad,), 12345.0, dtype=torch.float32, device=DEV)
+                raw[pad:pad + n].zero_()
+                raws.append((raw, n))
+                acc.append(raw[pad:pad + n].view(shp))
+            accs.append(acc)
+        ll = b.LayerList([b.Layer(kind=ld.spec.kind, G=ld.G, A=ld.A, ids=None, acc_w=a[0], acc_b=a[1] if len(a) > 1 else None,
+                                  has_bias=ld.spec.has_bias, vocab=0, path=b.DP_PATH_AUTO) for ld, a in zip(data, accs)])
+        nraw = torch.full((5 + 2 * pad,), 777.0, dtype=torch.float32, device=DEV)
+        craw = torch.full((5 + 2 * pad,), 777.0, dtype=torch.float32, device=DEV)
+        n, c = nraw[pad:pad + 5], craw[pad:pad + 5]
+        ws = b.alloc_workspace(ll)
+        b.dp_per_example_sqnorms(ll, n, False, ws)
+        b.dp_clip_factors(n, wl.C, c)
+        b.dp_clipped_accumulate_after_sqnorms(ll, c, ws)
+        torch.cuda.synchronize()
+        assert b.dp_poll_status() == 0
+        for raw, k in raws:
+            assert bool((raw[:pad] == 12345.0).all()) and bool((raw[pad + k:] == 12345.0).all())
+        for raw in (nraw, craw):
+            assert bool((raw[:pad] == 777.0).all()) and bool((raw[pad + 5:] == 777.0).all())
+        results.append([x.clone() for acc in accs for x in acc] + [n.clone(), c.clone()])
+    for x, y in zip(*results):
+        assert torch.equal(x, y)
