@@ -410,7 +410,7 @@ __global__ void __launch_bounds__(T_THREADS, 1) k_tile_sqnorm(const __grid_const
   }
 }
 
-struct AccumItem { int l, m0, n0, e0, e1, nt; bool valid; };
+struct AccumItem { int l, m0, n0, e0, e1, nt; bool valid, narrow; };
 
 // acc_w[(nb + j) * d_out + m] += v[j]: one lane owns row m (a d_out index), 32 columns per chunk.  The adds are
 // reductions performed at the L2 (no read-back into the SM); an element has one owner per launch unless the
@@ -440,6 +440,8 @@ __device__ __forceinline__ void accum_store_chunk(const UmmaLayer& L, int m, int
 // Every waiter waits for every phase of its barrier in order and whoever re-arms a barrier is gated on all
 // of its waiters (an mbarrier wait tells phases apart by parity only).  No TMA multicast is used.
 // Column c of N-half j of a CTA's accumulator is A feature n0 + 256 (c / 128) + 128 j + c % 128.
+// A tile with at most 256 A features left (the last one along d_in when d_in % 512 is in 1..256) is "narrow": CTA r
+// streams features [n0 + 128 r, +128) as its N-half 0 and the second UMMA of every k-step is skipped.
 // =================================================================================================
 constexpr int P_BK = 64;                                // tokens per stage
 constexpr int P_STAGES = 4;
@@ -468,6 +470,7 @@ __device__ __forceinline__ AccumItem pair_decode(const UmmaParams& P, int item) 
   t.nt = tile - mt * L.tiles_n;
   t.m0 = mt * 256;
   t.n0 = t.nt * 512;
+  t.narrow = L.d_in - t.n0 <= 256;     // at most 256 of the tile's 512 A features exist: one N-half carries them all
   t.e0 = (int)((long long)split * P.B / P.splits);
   t.e1 = (int)((long long)(split + 1) * P.B / P.splits);
   return t;
@@ -526,7 +529,7 @@ k_accum_pair(const __grid_constant__ UmmaParams P) {
         const AccumItem t = pair_decode(P, item);
         if (!t.valid) continue;
         const UmmaLayer& L = P.L[t.l];
-        const int mh = t.m0 + 128 * (int)rank, nh = t.n0 + 256 * (int)rank;
+        const int mh = t.m0 + 128 * (int)rank, nh = t.n0 + (t.narrow ? 128 : 256) * (int)rank;
         for (int e = t.e0; e < t.e1 && alive; ++e) {
           for (int tb = 0; tb < n_tb; ++tb) {
             const uint32_t slot = it % P_STAGES, ph = (it / P_STAGES) & 1u;
@@ -565,7 +568,7 @@ k_accum_pair(const __grid_constant__ UmmaParams P) {
             tc_fence_after();
             const uint32_t am = smem_u32(tiles + slot * P_STAGE_BYTES), an = am + P_M_BYTES;
             const int left = P.T - tb * P_BK;
-            if (left >= P_BK) {
+            if (left >= P_BK && !t.narrow) {
 #pragma unroll
               for (int k4 = 0; k4 < P_BK / 16; ++k4) {
                 const uint64_t adesc = smem_desc_sw128(am + k4 * 2048, P_ATOM_BYTES, 1024);
@@ -575,12 +578,12 @@ k_accum_pair(const __grid_constant__ UmmaParams P) {
                                  smem_desc_sw128(an + j * 2 * P_ATOM_BYTES + k4 * 2048, P_ATOM_BYTES, 1024), IDESC,
                                  acc | (uint32_t)k4);
               }
-            } else {                                   // ragged last stage: only the k-steps that hold tokens
-              const int nk = (left + 15) >> 4;
+            } else {                                   // ragged last stage or narrow tile: only the UMMAs that carry data
+              const int nk = left >= P_BK ? P_BK / 16 : (left + 15) >> 4, nj = t.narrow ? 1 : 2;
 #pragma unroll 1
               for (int k4 = 0; k4 < nk; ++k4) {
                 const uint64_t adesc = smem_desc_sw128(am + k4 * 2048, P_ATOM_BYTES, 1024);
-                for (int j = 0; j < 2; ++j)
+                for (int j = 0; j < nj; ++j)
                   umma_bf16_pair(tmem_base + (uint32_t)j * 256u, adesc,
                                  smem_desc_sw128(an + j * 2 * P_ATOM_BYTES + k4 * 2048, P_ATOM_BYTES, 1024), IDESC,
                                  acc | (uint32_t)k4);
@@ -669,12 +672,13 @@ k_accum_pair(const __grid_constant__ UmmaParams P) {
       if (!alive) continue;
       tc_fence_after();
       const int m = t.m0 + 128 * (int)rank + (int)q * 32 + lane;
+      // narrow tile: N-half 0 alone holds features n0 + 128 (c / 128) + c % 128; N-half 1 was never written
 #pragma unroll 1
-      for (int ch = 0; ch < 8; ++ch) {
+      for (int ch = 0; ch < ((t.narrow && h) ? 0 : 8); ++ch) {
         uint32_t v[32];
         tmem_ld_32x32(tmem_base + ((q * 32u) << 16) + (uint32_t)h * 256u + (uint32_t)ch * 32u, v);
         tmem_ld_wait();
-        accum_store_chunk(L, m, t.n0 + 256 * (ch >> 2) + 128 * h + (ch & 3) * 32, v);
+        accum_store_chunk(L, m, t.n0 + (t.narrow ? 128 : 256) * (ch >> 2) + 128 * h + (ch & 3) * 32, v);
       }
       tc_fence_before();
       __syncwarp();
