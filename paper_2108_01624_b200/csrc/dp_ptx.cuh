@@ -92,16 +92,9 @@ __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence:
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
 // ---- TMA ----------------------------------------------------------------------------------------
-// 3-D tiled load global -> shared, completion on an mbarrier (no multicast: every CTA fetches its own tile).
-__device__ __forceinline__ void tma_load_3d(void* smem_dst, const CUtensorMap* map, uint64_t* bar, int x, int y, int z) {
-  asm volatile(
-      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
-      ::"r"(smem_u32(smem_dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(smem_u32(bar)), "r"(x), "r"(y), "r"(z)
-      : "memory");
-}
-
-// 4-D variant.  The kernels view a [B, T, d] tensor as (x = 64 features, y = token, a = 64-feature group, z = example)
-// so that ONE copy brings several 64-feature groups of a token block: the cost of a tensor copy on the SM is per
+// 4-D tiled load global -> shared, completion on an mbarrier (no multicast: every CTA fetches its own tile).
+// The kernels view a [B, T, d] tensor as (x = 64 features, y = token, a = 64-feature group, z = example) so that
+// ONE copy brings several 64-feature groups of a token block: the cost of a tensor copy on the SM is per
 // instruction (about 130 cycles for a 3-D box, about 300 for a 4-D one, whatever its size), not per byte.
 __device__ __forceinline__ void tma_load_4d(void* smem_dst, const CUtensorMap* map, uint64_t* bar, int x, int y, int a, int z) {
   asm volatile(

@@ -78,8 +78,10 @@ __device__ __forceinline__ uint8_t* align1024(uint8_t* p) {
 // =================================================================================================
 // Gram kernel
 // =================================================================================================
-constexpr int G_SLOTS = 12;
-constexpr int G_SLOT_BYTES = 128 * 128;          // 128 tokens x 64 bf16 features, 128-byte swizzle
+constexpr int G_GROUPS = 2;                      // 64-feature tiles per TMA copy and ring slot
+constexpr int G_SLOTS = 6;
+constexpr int G_TILE_BYTES = 128 * 128;          // 128 tokens x 64 bf16 features, 128-byte swizzle
+constexpr int G_SLOT_BYTES = G_GROUPS * G_TILE_BYTES;
 constexpr int G_THREADS = 192;                   // warp 0: TMA, warp 1: MMA, warps 2..5: epilogue
 constexpr uint32_t G_IDESC = idesc_bf16_f32(128, 128, false, false);
 
@@ -123,8 +125,9 @@ __global__ void __launch_bounds__(G_THREADS, 1) k_gram_sqnorm(const __grid_const
   tc_fence_after();
   const uint32_t tmem_base = S->tmem_base;
   const int nblk = (P.T + 127) / 128, npairs = nblk * (nblk + 1) / 2;
-  // A box is always 128 tokens high: rows beyond T are outside the tensor and arrive as zeros.
-  constexpr uint32_t box_bytes = 128u * 128u;
+  // A box is always 128 tokens high and two 64-feature groups wide: rows beyond T and a group beyond the layer's
+  // width are outside the tensor and arrive as zeros.  One copy instruction per 32 KB keeps the producer (whose
+  // copies cost a fixed time each) well ahead of the 7 TB/s the ring can stream.
 
   if (warp == 0) {
     if (lane == 0) {   // ---------------- TMA producer ----------------
@@ -137,12 +140,12 @@ __global__ void __launch_bounds__(G_THREADS, 1) k_gram_sqnorm(const __grid_const
         for (int which = 0; which < 2 && alive; ++which) {
           const CUtensorMap* map = which ? &L.mapG : &L.mapA;
           const int d = which ? L.d_out : L.d_in;
-          for (int k0 = 0; k0 < d && alive; k0 += 64) {
+          for (int k0 = 0; k0 < d && alive; k0 += 64 * G_GROUPS) {
             for (int half = 0; half < (r == c ? 1 : 2); ++half) {
               const uint32_t slot = it % G_SLOTS, ph = (it / G_SLOTS) & 1u;
               if (!mbar_wait(&S->empty[slot], ph ^ 1u, abort_flag, P.status)) { alive = false; break; }
-              mbar_arrive_expect_tx(&S->full[slot], box_bytes);
-              tma_load_3d(tiles + slot * G_SLOT_BYTES, map, &S->full[slot], k0, (half ? c : r) * 128, i);
+              mbar_arrive_expect_tx(&S->full[slot], (uint32_t)G_SLOT_BYTES);
+              tma_load_4d(tiles + slot * G_SLOT_BYTES, map, &S->full[slot], 0, (half ? c : r) * 128, k0 / 64, i);
               ++it;
             }
           }
@@ -169,7 +172,7 @@ __global__ void __launch_bounds__(G_THREADS, 1) k_gram_sqnorm(const __grid_const
         for (int which = 0; which < 2 && alive; ++which) {
           const int d = which ? L.d_out : L.d_in;
           const uint32_t d_tmem = tmem_base + buf * 256u + (uint32_t)which * 128u;
-          for (int k0 = 0; k0 < d; k0 += 64) {
+          for (int k0 = 0; k0 < d; k0 += 64 * G_GROUPS) {
             const uint32_t sr = it % G_SLOTS, pr = (it / G_SLOTS) & 1u;
             ++it;
             if (!mbar_wait(&S->full[sr], pr, abort_flag, P.status)) { alive = false; break; }
@@ -183,9 +186,14 @@ __global__ void __launch_bounds__(G_THREADS, 1) k_gram_sqnorm(const __grid_const
             tc_fence_after();
             const uint32_t ar = smem_u32(tiles + sr * G_SLOT_BYTES), ac = smem_u32(tiles + sc * G_SLOT_BYTES);
 #pragma unroll
-            for (int k4 = 0; k4 < 4; ++k4) {
-              umma_bf16(d_tmem, smem_desc_sw128(ar + k4 * 32, 16, 1024), smem_desc_sw128(ac + k4 * 32, 16, 1024),
-                        G_IDESC, (k0 | k4) ? 1u : 0u);
+            for (int g = 0; g < G_GROUPS; ++g) {
+              if (k0 + 64 * g < d) {                   // a group beyond the layer's width holds zeros: skip it
+#pragma unroll
+                for (int k4 = 0; k4 < 4; ++k4) {
+                  umma_bf16(d_tmem, smem_desc_sw128(ar + g * G_TILE_BYTES + k4 * 32, 16, 1024),
+                            smem_desc_sw128(ac + g * G_TILE_BYTES + k4 * 32, 16, 1024), G_IDESC, (k0 | g | k4) ? 1u : 0u);
+                }
+              }
             }
             umma_commit(&S->empty[sr]);
             if (r != c) umma_commit(&S->empty[sc]);
@@ -714,23 +722,8 @@ static EncodeTiledFn encode_fn() {
   return fn;
 }
 
-// bf16 tensor [B, T, d] viewed as (x = feature, y = token, z = example); box = 64 features x box_rows tokens,
-// 128-byte swizzle, out-of-range elements read as zero.
-static bool encode_map(CUtensorMap* map, const void* base, int B, int T, int d, int box_rows) {
-  EncodeTiledFn fn = encode_fn();
-  if (!fn) return false;
-  const cuuint64_t dims[3] = {(cuuint64_t)d, (cuuint64_t)T, (cuuint64_t)B};
-  const cuuint64_t strides[2] = {(cuuint64_t)d * 2, (cuuint64_t)T * d * 2};
-  const cuuint32_t box[3] = {64u, (cuuint32_t)box_rows, 1u};
-  const cuuint32_t estr[3] = {1u, 1u, 1u};
-  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-            DP_TMA_L2_PROMOTION == 0 ? CU_TENSOR_MAP_L2_PROMOTION_NONE
-            : DP_TMA_L2_PROMOTION == 1 ? CU_TENSOR_MAP_L2_PROMOTION_L2_128B : CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
-// The same tensor as (x = 64 features, y = token, a = 64-feature group, z = example); box = 64 x box_rows x groups x 1.
+// bf16 tensor [B, T, d] viewed as (x = 64 features, y = token, a = 64-feature group, z = example);
+// box = 64 x box_rows x groups x 1, 128-byte swizzle, out-of-range elements read as zero.
 static bool encode_map4(CUtensorMap* map, const void* base, int B, int T, int d, int box_rows, int groups) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) return false;
@@ -783,18 +776,13 @@ static bool ensure_smem(K kernel, int bytes) {
   return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) == cudaSuccess;
 }
 
-// groups_g / groups_a > 0: 4-D maps whose box spans that many 64-feature groups (tile kernels); 0: 3-D maps (Gram).
+// groups_g / groups_a: 64-feature groups that a box of the G / A map spans.
 // A box may be taller than T or span more groups than the layer has: what lies outside the tensor is zero-filled.
-static bool fill_layer(UmmaLayer& U, const dp_layer& L, int box_rows, int groups_g = 0, int groups_a = 0) {
+static bool fill_layer(UmmaLayer& U, const dp_layer& L, int box_rows, int groups_g, int groups_a) {
   const bool emb = L.kind == DP_EMBEDDING;
-  if (groups_g > 0) {
-    if (!encode_map4(&U.mapG, L.G, L.B, L.T, L.d_out, box_rows, groups_g)) return false;
-    if (!encode_map4(&U.mapA, L.A, L.B, L.T, L.d_in, box_rows, groups_a)) return false;
-  } else {
-    if (!encode_map(&U.mapG, L.G, L.B, L.T, L.d_out, box_rows)) return false;
-    if (emb) U.mapA = U.mapG;      // never used: an embedding streams no A operand (d_in = 0 below)
-    else if (!encode_map(&U.mapA, L.A, L.B, L.T, L.d_in, box_rows)) return false;
-  }
+  if (!encode_map4(&U.mapG, L.G, L.B, L.T, L.d_out, box_rows, groups_g)) return false;
+  if (emb) U.mapA = U.mapG;      // never used: an embedding streams no A operand (d_in = 0 below)
+  else if (!encode_map4(&U.mapA, L.A, L.B, L.T, L.d_in, box_rows, groups_a)) return false;
   U.acc_w = L.acc_w;
   U.acc_b = L.acc_b;
   U.ids = emb ? L.ids : nullptr;
@@ -835,7 +823,7 @@ int launch_umma_sqnorms(const dp_layer* layers, const int* idx, int n, const int
         const long long add = (long long)B * (gram ? gram_pairs(T) : tile_count(L));
         if (items + add > 0x7fffffffll) break;
         UmmaLayer& U = P.L[P.n_layers];
-        if (!(gram ? fill_layer(U, L, 128) : fill_layer(U, L, T_BK, 2, 4))) return DP_ERR_CUDA;
+        if (!(gram ? fill_layer(U, L, 128, G_GROUPS, G_GROUPS) : fill_layer(U, L, T_BK, 2, 4))) return DP_ERR_CUDA;
         U.item_start = (int)items;
         U.partial_base = base[k];
         items += add;
