@@ -7,7 +7,7 @@ import torch
 
 from paper_2108_01624_b200 import DPStep, synth
 
-from .helpers import (LINEAR, O, b, gpu_norms_clip, make_layer_list, rel_l2, to_np, to_oracle_layers)
+from .helpers import (LAYERNORM, LINEAR, O, b, gpu_norms_clip, make_layer_list, rel_l2, to_np, to_oracle_layers)
 
 pytestmark = pytest.mark.gpu
 
@@ -49,6 +49,29 @@ def _sampled_entries_check(data, accs, clip, n_samples, seed):
             assert abs(float(acc[1][q]) - ref) <= BF16_TOL * (abs(ref) + scale)
 
 
+def _full_size_ln_and_embedding_check(data, accs, clip, n_ln, seed):
+    """At the full launch size: a few LayerNorm layers (every element of gain and bias sums) and the embedding
+    (every row) recomputed in fp64 on the host with the GPU's clip factors."""
+    rng = np.random.default_rng(seed)
+    c = to_np(clip)
+    ln_idx = [k for k, ld in enumerate(data) if ld.spec.kind == LAYERNORM]
+    for k in rng.choice(ln_idx, size=min(n_ln, len(ln_idx)), replace=False):
+        ld, acc = data[int(k)], accs[int(k)]
+        G, X = to_np(ld.G), to_np(ld.A)
+        gain = np.einsum("i,itd->d", c, X * G)
+        bias = np.einsum("i,itd->d", c, G)
+        assert rel_l2(to_np(acc[0]), gain) <= 1e-3 and rel_l2(to_np(acc[1]), bias) <= 1e-3, ld.spec.name
+    for ld, acc in zip(data, accs):
+        if ld.spec.kind != synth.EMBEDDING:
+            continue
+        G = to_np(ld.G) * c[:, None, None]
+        ref = np.zeros((ld.spec.d_in, ld.spec.d_out))
+        np.add.at(ref, ld.ids.cpu().numpy().reshape(-1), G.reshape(-1, ld.spec.d_out))
+        assert rel_l2(to_np(acc[0]), ref) <= 1e-3, ld.spec.name
+        untouched = np.setdiff1d(np.arange(ld.spec.d_in), ld.ids.cpu().numpy().reshape(-1))
+        assert float(acc[0][torch.from_numpy(untouched).to(acc[0].device)].abs().max()) == 0.0
+
+
 def test_bert_base_block_full_batch():
     wl = synth.workload("bert_base_layer")
     data = synth.generate(wl, seed=0, device=DEV)
@@ -79,8 +102,18 @@ def test_bert_large_stack_subset_and_samples(n_layers):
     data = synth.generate(wl, seed=0, device=DEV, specs=specs)
     assert len(data) == 6 * n_layers + 1
     ll, accs = make_layer_list(data, DEV)
-    n, c, ws = gpu_norms_clip(ll, wl.C)
-    b.dp_clipped_accumulate(ll, c, ws)
+    # the call sequence bench.py times: the model in two lists (linear layers; LayerNorm + embedding), each with
+    # its own workspace, the second accumulate reusing the column sums of its norm call
+    lin = b.LayerList([l for l in ll.layers if l.kind == "linear"])
+    rest = b.LayerList([l for l in ll.layers if l.kind != "linear"])
+    ws, ws_rest = b.alloc_workspace(lin), b.alloc_workspace(rest)
+    n = torch.empty(wl.B, dtype=torch.float32, device=DEV)
+    c = torch.empty(wl.B, dtype=torch.float32, device=DEV)
+    b.dp_per_example_sqnorms(lin, n, False, ws)
+    b.dp_per_example_sqnorms(rest, n, True, ws_rest)
+    b.dp_clip_factors(n, wl.C, c)
+    b.dp_clipped_accumulate(lin, c, ws)
+    b.dp_clipped_accumulate_after_sqnorms(rest, c, ws_rest)
     torch.cuda.synchronize()
     assert b.dp_poll_status() == 0
     # (a) checker on eight examples spread over the batch (first, last, and both sides of the half-way and
@@ -94,6 +127,7 @@ def test_bert_large_stack_subset_and_samples(n_layers):
     np.testing.assert_allclose(to_np(c[rows]), c_ref, rtol=CLIP_TOL)
     # (b) full launch size: sampled accumulator entries in fp64
     _sampled_entries_check(data, accs, c, n_samples=6, seed=1)
+    _full_size_ln_and_embedding_check(data, accs, c, n_ln=3, seed=2)
     # (c) the same eight examples as a microbatch of their own through the GPU path, element by element
     ll8, acc8 = make_layer_list(sub, DEV)
     n8, c8, ws8 = gpu_norms_clip(ll8, wl.C)
