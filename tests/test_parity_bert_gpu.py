@@ -128,6 +128,16 @@ def test_bert_large_stack_subset_and_samples(n_layers):
     # (b) full launch size: sampled accumulator entries in fp64
     _sampled_entries_check(data, accs, c, n_samples=6, seed=1)
     _full_size_ln_and_embedding_check(data, accs, c, n_ln=3, seed=2)
+    # (b') all 256 norms of the linear layers: the Gram kernel against the materialised-tile kernel, two different
+    # algorithms for the same quantity (the identity of Section 4.3 holds at any size)
+    n_gram = torch.empty(wl.B, dtype=torch.float32, device=DEV)
+    b.dp_per_example_sqnorms(lin, n_gram, False, ws)
+    lin_mat = b.LayerList([b.Layer(kind=l.kind, G=l.G, A=l.A, ids=None, acc_w=l.acc_w, acc_b=l.acc_b, has_bias=l.has_bias,
+                                   vocab=0, path=b.DP_PATH_MATERIALIZED) for l in lin.layers])
+    n_mat = torch.empty(wl.B, dtype=torch.float32, device=DEV)
+    b.dp_per_example_sqnorms(lin_mat, n_mat, False, b.alloc_workspace(lin_mat))
+    assert b.dp_poll_status() == 0
+    np.testing.assert_allclose(to_np(n_gram), to_np(n_mat), rtol=2 * CLIP_TOL)
     # (c) the same eight examples as a microbatch of their own through the GPU path, element by element
     ll8, acc8 = make_layer_list(sub, DEV)
     n8, c8, ws8 = gpu_norms_clip(ll8, wl.C)
