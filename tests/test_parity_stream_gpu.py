@@ -254,3 +254,28 @@ def test_fused_cross_rank_update_matches_checker(n_flat, world):
         b.dp_noise_scale_adamw_step(th1, m1, v1, s, True, hp["sigma"], hp["C"], hp["N"], hp["seed"], hp["step"],
                                     hp["lr"], hp["b1"], hp["b2"], hp["xi"], hp["wd"], hp["t"], 0)
         assert torch.equal(th1, th_d[0])
+
+
+def test_fused_update_at_full_parameter_count_on_sampled_windows():
+    """One fused launch over 333,563,904 parameters (the BERT-Large vector of the benchmark); the checker
+    recomputes windows at the start, around 2^28 and 2^32 bytes into the vector, and at the ragged end."""
+    n = 333_563_904
+    hp = dict(sigma=0.9, C=0.5, N=2_097_152, seed=0xC0FFEE, step=7, lr=1e-3, b1=0.9, b2=0.999, xi=1e-11, wd=0.5, t=2)
+    g = torch.Generator(device=DEV).manual_seed(5)
+    acc = torch.randn(n, generator=g, device=DEV) * 100.0
+    theta = torch.randn(n, generator=g, device=DEV) * 0.02
+    m = torch.randn(n, generator=g, device=DEV) * 1e-5
+    v = torch.rand(n, generator=g, device=DEV) * 1e-9
+    windows = [(0, 4096), ((1 << 26) - 100, 300), ((1 << 28) + 1, 2047), (n - 4099, 4099)]
+    before = {lo: tuple(to_np(x[lo:lo + k]) for x in (acc, theta, m, v)) for lo, k in windows}
+    b.dp_noise_scale_adamw_step(theta, m, v, acc, True, hp["sigma"], hp["C"], hp["N"], hp["seed"], hp["step"],
+                                hp["lr"], hp["b1"], hp["b2"], hp["xi"], hp["wd"], hp["t"], 0)
+    torch.cuda.synchronize()
+    assert float(acc.abs().max()) == 0.0
+    for lo, k in windows:
+        a0, t0, m0, v0 = before[lo]
+        gref = O.add_noise_and_scale(a0, hp["sigma"], hp["C"], hp["N"], seed=hp["seed"], step=hp["step"], elem_offset=lo)
+        rt, rm, rv = O.adamw_step(t0, m0, v0, gref, hp["lr"], hp["b1"], hp["b2"], hp["xi"], hp["wd"], hp["t"])
+        assert rel_max(to_np(m[lo:lo + k]), rm) <= F32_TOL and rel_max(to_np(v[lo:lo + k]), rv) <= F32_TOL
+        d, rd = to_np(theta[lo:lo + k]) - t0, rt - t0
+        assert np.max(np.abs(d - rd)) <= F32_TOL * np.max(np.abs(rd)) + 1e-7 * np.max(np.abs(t0))
