@@ -681,12 +681,18 @@ k_accum_pair(const __grid_constant__ UmmaParams P) {
       tc_fence_after();
       const int m = t.m0 + 128 * (int)rank + (int)q * 32 + lane;
       // narrow tile: N-half 0 alone holds features n0 + 128 (c / 128) + c % 128; N-half 1 was never written
-#pragma unroll 1
-      for (int ch = 0; ch < ((t.narrow && h) ? 0 : 8); ++ch) {
-        uint32_t v[32];
-        tmem_ld_32x32(tmem_base + ((q * 32u) << 16) + (uint32_t)h * 256u + (uint32_t)ch * 32u, v);
-        tmem_ld_wait();
-        accum_store_chunk(L, m, t.n0 + (t.narrow ? 128 : 256) * (ch >> 2) + 128 * h + (ch & 3) * 32, v);
+      if (!(t.narrow && h)) {
+        // two register buffers: the TMEM load of chunk ch + 1 is in flight while chunk ch goes out as L2 reductions
+        uint32_t v[2][32];
+        const uint32_t tsrc = tmem_base + ((q * 32u) << 16) + (uint32_t)h * 256u;
+        const int nstep = t.narrow ? 128 : 256;
+        tmem_ld_32x32(tsrc, v[0]);
+#pragma unroll
+        for (int ch = 0; ch < 8; ++ch) {
+          tmem_ld_wait();
+          if (ch + 1 < 8) tmem_ld_32x32(tsrc + (uint32_t)(ch + 1) * 32u, v[(ch + 1) & 1]);
+          accum_store_chunk(L, m, t.n0 + nstep * (ch >> 2) + 128 * h + (ch & 3) * 32, v[ch & 1]);
+        }
       }
       tc_fence_before();
       __syncwarp();
