@@ -61,6 +61,11 @@ typedef enum { DP_F32 = 0, DP_BF16 = 1 } dp_dtype;
  *   AUTO          linear: GRAM iff T * (d_in + d_out) <= d_in * d_out, the flop count of either way;
  *                 embedding: GRAM whenever the tensor-core kernel accepts the layer (bf16, d_out % 64 == 0). */
 typedef enum { DP_PATH_AUTO = 0, DP_PATH_GRAM = 1, DP_PATH_MATERIALIZED = 2 } dp_path;
+/* Which kernels a layer gets.  A bf16 LINEAR layer whose d_in and d_out are multiples of 64 and whose A and G are
+ * 16-byte aligned runs on the tensor cores (norms and clipped sum); every other linear layer (fp32, other widths,
+ * e.g. a vocabulary-sized output that was not padded to a multiple of 64) runs on plain CUDA-core kernels, which
+ * give the same results and are far slower.  LAYERNORM and the EMBEDDING accumulate are bandwidth-bound kernels
+ * for any width; they use 16-byte loads when d is a multiple of 8 (bf16) or 4 (fp32) and the tensors are aligned. */
 
 /* One trainable layer of one microbatch.  B and T must be equal across the layers of a call. */
 typedef struct dp_layer {
