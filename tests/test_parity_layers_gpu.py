@@ -194,6 +194,16 @@ def test_layer_with_more_tiles_than_one_wave():
     check_against_checker(data, C)
 
 
+def test_vocabulary_sized_output_layer():
+    """An output projection onto a vocabulary padded to a multiple of 64 (30528): 120 x 1 accumulate tiles, 477
+    feature tiles per example in the Gram kernel."""
+    specs = [LayerSpec(LINEAR, 256, 30528, True, "mlm_head")]
+    data = random_layers(specs, 3, 48, torch.bfloat16, DEV, seed=17, g_scale=0.01)
+    ol = to_oracle_layers(data)
+    C = float(np.sqrt(np.median(O.per_example_sqnorms(ol))))
+    check_against_checker(data, C)
+
+
 def test_accumulate_twice_adds_twice():
     """acc += ...: a second call over the same microbatch doubles every accumulator (the GEMM adds through L2
     reductions, the other kernels read-modify-write)."""
