@@ -3,7 +3,7 @@
 //   k_gram_sqnorm  per-example squared norm by the token-Gram identity
 //                  |A_i^T G_i|_F^2 + |1^T G_i|^2 = < A_i A_i^T + [bias] 1 1^T , G_i G_i^T >.
 //                  Both 128x128 fp32 Grams of a token-block pair live in TMEM (2 x 128 columns,
-//                  double-buffered); operands are K-major 128x64 tiles fetched by TMA.  For a token
+//                  double-buffered); operands are K-major 128x64 tiles, two per TMA copy.  For a token
 //                  embedding the input is one-hot, so A_i A_i^T is the token-id equality mask: only
 //                  G_i G_i^T is formed on the tensor cores and the epilogue multiplies it by
 //                  [id_t == id_s] (integer compares).
@@ -36,6 +36,7 @@ constexpr int kMaxLayers = kUmmaMaxLayers;
 #ifndef DP_TMA_L2_PROMOTION
 #define DP_TMA_L2_PROMOTION 2          // 0 none, 1 128 B, 2 256 B
 #endif
+
 struct alignas(64) UmmaLayer {
   CUtensorMap mapG;   // [B, T, d_out] bf16
   CUtensorMap mapA;   // [B, T, d_in]  bf16
@@ -47,8 +48,7 @@ struct alignas(64) UmmaLayer {
   int partial_base;       // first per-example partial slot of this layer
   uint16_t tiles_m, tiles_n;   // tile kernels: tiles over d_out and over d_in
   uint8_t has_bias, is_emb;
-  uint16_t pad;
-  int pad2[4];
+  uint8_t pad[18];        // to 320 bytes (a multiple of the tensor maps' 64-byte alignment)
 };
 static_assert(sizeof(UmmaLayer) == 320, "UmmaLayer grew: 96 of them must fit the kernel parameter block");
 
@@ -798,8 +798,7 @@ static bool fill_layer(UmmaLayer& U, const dp_layer& L, int box_rows, int groups
   U.tiles_n = (uint16_t)ceil_div(L.d_in, 256);
   U.has_bias = emb ? 0 : L.has_bias;
   U.is_emb = emb ? 1 : 0;
-  U.pad = 0;
-  U.pad2[0] = U.pad2[1] = U.pad2[2] = U.pad2[3] = 0;
+  for (uint8_t& x : U.pad) x = 0;
   return true;
 }
 
