@@ -9,6 +9,7 @@ stay resident in HBM (32 GB per microbatch, far larger than L2, so no flush is n
   python bench.py [--gpus N] [--steps K] [--warmup W]          device-timed line (+ e2e, roofline, cpu_baseline)
   python bench.py --impl reference ...                         the CPU checker timed on the host cores
   python bench.py --macro-microbatches 8192                    one whole macro-step of the 2,097,152-example mega-batch
+  python bench.py --long-sequence-paths                        T=512 block: Gram vs materialised vs auto-selected norms
 
 Under torchrun (N > 1) each rank processes its own microbatches (weak scaling); the accumulators are
 reduce-scattered once per step, the noise/AdamW pass runs on the local shard and theta is all-gathered.
@@ -210,6 +211,9 @@ def main():
     ap.add_argument("--macro-microbatches", type=int, default=0,
                     help="instead of the per-microbatch line: time ONE macro-step of this many microbatches "
                          "(8192 = the 2,097,152-example mega-batch of Section 5.3) and print its line")
+    ap.add_argument("--long-sequence-paths", action="store_true",
+                    help="instead of the per-microbatch line: the T=512 BERT-Large block (B=64) with the norm path of "
+                         "its linear layers forced to Gram, forced to materialised tiles, and chosen automatically")
     ap.add_argument("--pool", type=int, default=2,
                     help="distinct resident microbatches the macro-step rotates over (32 GB each)")
     args = ap.parse_args()
@@ -217,6 +221,9 @@ def main():
         run_reference(args)
         return
     args.warmup = max(args.warmup, 3)
+    if args.long_sequence_paths:
+        run_long_sequence_paths(args)
+        return
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -367,6 +374,61 @@ def main():
         print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()
+
+
+def run_long_sequence_paths(args):
+    """The long-sequence crossover: one BERT-Large block at T=512, B=64.  Norms of the four linear layers with the
+    path forced per layer (token Gram / materialised tiles) and auto-selected, then the clipped accumulate; each
+    call device-timed alone over `--steps` repetitions (inputs 1.07 GB, larger than L2)."""
+    import paper_2108_01624_b200 as pkg
+    from paper_2108_01624_b200 import binding as b
+    from paper_2108_01624_b200 import synth
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    wl = synth.workload("bert_large_layer_t512")
+    data = [ld for ld in synth.generate(wl, seed=0, device=dev) if ld.spec.kind == "linear"]
+    accs = [(torch.zeros(ld.spec.d_in, ld.spec.d_out, device=dev), torch.zeros(ld.spec.d_out, device=dev)) for ld in data]
+    sq = torch.empty(wl.B, dtype=torch.float32, device=dev)
+    clip = torch.empty_like(sq)
+    stream = torch.cuda.current_stream()
+    reps = max(args.steps, 10)
+
+    def timed(fn):
+        for _ in range(args.warmup):
+            fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(reps):
+            fn()
+        e1.record(stream)
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / reps
+
+    T, B = wl.T, wl.B
+    nbytes = sum(2.0 * B * T * (ld.spec.d_in + ld.spec.d_out) for ld in data)
+    nblk = (T + 127) // 128
+    flops = {"gram": sum(2.0 * B * (ld.spec.d_in + ld.spec.d_out) * 128 * 128 * nblk * (nblk + 1) / 2 for ld in data),
+             "materialized": sum(2.0 * B * T * ld.spec.d_in * ld.spec.d_out for ld in data)}
+    out = {}
+    l0 = pkg.dp_launch_count()
+    for name, path in (("gram", b.DP_PATH_GRAM), ("materialized", b.DP_PATH_MATERIALIZED), ("auto", b.DP_PATH_AUTO)):
+        ll = pkg.LayerList([b.Layer(kind="linear", G=ld.G, A=ld.A, acc_w=a[0], acc_b=a[1], has_bias=True, path=path)
+                            for ld, a in zip(data, accs)])
+        ws = b.alloc_workspace(ll)
+        ms = timed(lambda: pkg.dp_per_example_sqnorms(ll, sq, False, ws))
+        out[name] = {"ms": ms, "GB/s": nbytes / ms / 1e6}
+        if name in flops:       # flops the kernel executes (upper-triangle block pairs for the Gram path)
+            out[name]["TFLOP/s"] = flops[name] / ms / 1e9
+    pkg.dp_clip_factors(sq, wl.C, clip)
+    ms = timed(lambda: pkg.dp_clipped_accumulate(ll, clip, ws))
+    out["accumulate"] = {"ms": ms, "TFLOP/s": flops["materialized"] / ms / 1e9}
+    torch.cuda.synchronize()
+    if pkg.dp_poll_status() != 0:
+        raise RuntimeError("device status not clean")
+    print(json.dumps({"workload": "bert_large_layer_t512", "B": B, "T": T, "linear_layers": len(data),
+                      "input_bytes": nbytes, "repetitions": reps, "timings": out,
+                      "gpu_launches": int(pkg.dp_launch_count() - l0), "peaks": measured_peaks()}))
 
 
 def run_macro_step(args, pkg, synth, wl, step, sharded, dist, world, rank, dev, data0, lin_idx, rest_idx, bufs, stream):

@@ -267,6 +267,226 @@ __global__ void __launch_bounds__(G_THREADS, 1) k_gram_sqnorm(const __grid_const
 }
 
 // =================================================================================================
+// Gram kernel for examples longer than one token block (T > 128, linear layers)
+//
+// With several 128-token blocks the Gram of an example is a grid of nblk x nblk blocks, of which the upper
+// triangle is computed.  An item here is a row block r and TWO neighbouring column blocks (c0, c0 + 1), one
+// 128 x 256 x 16 UMMA per 16 features: per 64-feature stage the SM receives the row tile (16 KB, not needed
+// when r = c0: the first half of the column tile is the row tile) and the column tile (32 KB) for 512 tensor
+// cycles, where the one-block-pair kernel above needs two 16 KB tiles per 256 cycles (and its 128 x 128 UMMAs read
+// shared memory at the full 128 B/clk).  The last column block of a row with an odd count runs alone (N = 128).
+// TMEM holds P = A_r A_c^T (256 columns) and Q = G_r G_c^T (256 columns), one buffer each; the pipeline is kept
+// full by splitting the epilogue: as soon as P is complete the eight epilogue warps copy it to registers (128
+// per thread) and release its columns, so the UMMAs of the next item's P overlap this item's Q and product-sum.
+// =================================================================================================
+constexpr int W_STAGES = 4;
+constexpr int W_ROW_BYTES = 128 * 128;                  // 128 tokens x 64 bf16 features, 128-byte swizzle
+constexpr int W_COL_BYTES = 256 * 128;                  // 256 tokens x 64 features
+constexpr int W_STAGE_BYTES = W_ROW_BYTES + W_COL_BYTES;
+constexpr int W_THREADS = 320;                          // warp 0 TMA, warp 1 UMMA issue, warps 2..9 epilogue
+constexpr int kWideMaxLayers = 48;
+
+struct alignas(64) WideLayer {
+  CUtensorMap rowA, colA, rowG, colG;   // [B, T, d] bf16 as (feature, token, example); boxes 64 x 128 and 64 x 256
+  int d_out, d_in;
+  int item_start, partial_base;
+  int has_bias;
+  int pad[11];
+};
+static_assert(sizeof(WideLayer) == 576, "WideLayer: 48 of them must fit the kernel parameter block");
+
+struct WideParams {
+  WideLayer L[kWideMaxLayers];
+  int n_layers, total_items, B, T;
+  int partial_stride, pad;
+  float* partial;
+  int* status;
+};
+static_assert(sizeof(WideParams) <= 32000, "kernel parameter block too large");
+
+struct WideCtl {
+  uint64_t full[W_STAGES], empty[W_STAGES], x_full, x_empty, y_full, y_empty, drain;
+  uint32_t tmem_base;
+  int abort;
+};
+constexpr int W_SMEM = 1024 + W_STAGES * W_STAGE_BYTES + (int)sizeof(WideCtl);
+
+// items of one example: for every row block r the column blocks r, r+1, ... in pairs
+__host__ __device__ inline int wide_items(int nblk) {
+  int n = 0;
+  for (int r = 0; r < nblk; ++r) n += (nblk - r + 1) / 2;
+  return n;
+}
+
+struct WideItem { int l, i, idx, r, c0, ncol; };
+
+__device__ __forceinline__ WideItem wide_decode(const WideParams& P, int item, int per_example, int nblk) {
+  WideItem t;
+  t.l = 0;
+  while (t.l + 1 < P.n_layers && item >= P.L[t.l + 1].item_start) ++t.l;
+  const int rem = item - P.L[t.l].item_start;
+  t.i = rem / per_example;
+  t.idx = rem - t.i * per_example;
+  int p = t.idx;
+  t.r = 0;
+  while (p >= (nblk - t.r + 1) / 2) { p -= (nblk - t.r + 1) / 2; ++t.r; }
+  t.c0 = t.r + 2 * p;
+  t.ncol = (nblk - t.c0) < 2 ? (nblk - t.c0) : 2;
+  return t;
+}
+
+__global__ void __launch_bounds__(W_THREADS, 1) k_gram_sqnorm_wide(const __grid_constant__ WideParams P) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* tiles = align1024(smem_raw);
+  WideCtl* S = reinterpret_cast<WideCtl*>(tiles + W_STAGES * W_STAGE_BYTES);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  volatile int* abort_flag = &S->abort;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < W_STAGES; ++s) { mbar_init(&S->full[s], 1); mbar_init(&S->empty[s], 1); }
+    mbar_init(&S->x_full, 1);
+    mbar_init(&S->y_full, 1);
+    mbar_init(&S->x_empty, 8);
+    mbar_init(&S->y_empty, 8);
+    mbar_init(&S->drain, 1);
+    S->abort = 0;
+    fence_mbar_init();
+  }
+  if (warp == 1) { tmem_alloc(&S->tmem_base, 512); tmem_relinquish(); }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = S->tmem_base;
+  const int nblk = (P.T + 127) / 128, per_example = wide_items(nblk);
+
+  if (warp == 0) {
+    if (lane == 0) {   // ---------------- TMA producer ----------------
+      uint32_t it = 0;
+      bool alive = true;
+      for (int item = blockIdx.x; item < P.total_items && alive; item += gridDim.x) {
+        const WideItem t = wide_decode(P, item, per_example, nblk);
+        const WideLayer& L = P.L[t.l];
+        const bool diag = t.c0 == t.r;
+        // a lone column block is fetched with the 128-token box; rows beyond T arrive as zeros either way
+        const uint32_t bytes = (uint32_t)((diag ? 0 : W_ROW_BYTES) + (t.ncol == 2 ? W_COL_BYTES : W_ROW_BYTES));
+        for (int which = 0; which < 2 && alive; ++which) {
+          const CUtensorMap* rowmap = which ? &L.rowG : &L.rowA;
+          const CUtensorMap* colmap = t.ncol == 2 ? (which ? &L.colG : &L.colA) : rowmap;
+          const int d = which ? L.d_out : L.d_in;
+          for (int k0 = 0; k0 < d; k0 += 64) {
+            const uint32_t slot = it % W_STAGES, ph = (it / W_STAGES) & 1u;
+            if (!mbar_wait(&S->empty[slot], ph ^ 1u, abort_flag, P.status, 21, (int)it)) { alive = false; break; }
+            uint8_t* st = tiles + slot * W_STAGE_BYTES;
+            mbar_arrive_expect_tx(&S->full[slot], bytes);
+            if (!diag) tma_load_3d(st, rowmap, &S->full[slot], k0, t.r * 128, t.i);
+            tma_load_3d(st + W_ROW_BYTES, colmap, &S->full[slot], k0, t.c0 * 128, t.i);
+            ++it;
+          }
+        }
+      }
+      const uint32_t pending = it < (uint32_t)W_STAGES ? it : (uint32_t)W_STAGES;
+      for (uint32_t k = 0; k < pending; ++k) {
+        const uint32_t j = it - 1 - k;
+        mbar_wait_drain(&S->full[j % W_STAGES], (j / W_STAGES) & 1u, P.status);
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {   // ---------------- MMA issuer ----------------
+      constexpr uint32_t IDESC_N256 = idesc_bf16_f32(128, 256, false, false);
+      constexpr uint32_t IDESC_N128 = idesc_bf16_f32(128, 128, false, false);
+      uint32_t it = 0, tile_it = 0;
+      bool alive = true;
+      for (int item = blockIdx.x; item < P.total_items && alive; item += gridDim.x, ++tile_it) {
+        const WideItem t = wide_decode(P, item, per_example, nblk);
+        const WideLayer& L = P.L[t.l];
+        const bool diag = t.c0 == t.r;
+        const uint32_t idesc = t.ncol == 2 ? IDESC_N256 : IDESC_N128;
+        const uint32_t tph = tile_it & 1u;
+        for (int which = 0; which < 2 && alive; ++which) {
+          if (!mbar_wait(which ? &S->y_empty : &S->x_empty, tph ^ 1u, abort_flag, P.status, 22, (int)tile_it)) {
+            alive = false;
+            break;
+          }
+          tc_fence_after();
+          const int d = which ? L.d_out : L.d_in;
+          const uint32_t d_tmem = tmem_base + (uint32_t)which * 256u;
+          for (int k0 = 0; k0 < d; k0 += 64) {
+            const uint32_t slot = it % W_STAGES, ph = (it / W_STAGES) & 1u;
+            ++it;
+            if (!mbar_wait(&S->full[slot], ph, abort_flag, P.status, 23, (int)it)) { alive = false; break; }
+            tc_fence_after();
+            const uint32_t colb = smem_u32(tiles + slot * W_STAGE_BYTES) + W_ROW_BYTES;
+            const uint32_t rowb = diag ? colb : colb - W_ROW_BYTES;
+#pragma unroll
+            for (int k4 = 0; k4 < 4; ++k4)
+              umma_bf16(d_tmem, smem_desc_sw128(rowb + k4 * 32, 16, 1024), smem_desc_sw128(colb + k4 * 32, 16, 1024),
+                        idesc, (k0 | k4) ? 1u : 0u);
+            umma_commit(&S->empty[slot]);
+          }
+          if (alive) umma_commit(which ? &S->y_full : &S->x_full);
+        }
+      }
+      umma_commit(&S->drain);
+      mbar_wait_drain(&S->drain, 0u, P.status);
+    }
+  } else {   // ---------------- epilogue warps 2..9: lanes [32 q, +32), column block h of the pair ----------------
+    const uint32_t q = (uint32_t)warp & 3u;
+    const int h = warp >= 6 ? 1 : 0;
+    uint32_t tile_it = 0;
+    bool alive = true;
+    for (int item = blockIdx.x; item < P.total_items; item += gridDim.x, ++tile_it) {
+      const WideItem t = wide_decode(P, item, per_example, nblk);
+      const WideLayer& L = P.L[t.l];
+      const uint32_t tph = tile_it & 1u;
+      const bool active = h < t.ncol;
+      const uint32_t tsrc = tmem_base + ((q * 32u) << 16) + (uint32_t)h * 128u;
+      if (alive) alive = __all_sync(0xffffffffu, mbar_wait(&S->x_full, tph, abort_flag, P.status, 24, (int)tile_it));
+      if (!alive) continue;
+      tc_fence_after();
+      uint32_t pv[4][32];
+      if (active) {
+#pragma unroll
+        for (int ch = 0; ch < 4; ++ch) tmem_ld_32x32(tsrc + (uint32_t)ch * 32u, pv[ch]);
+        tmem_ld_wait();
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&S->x_empty);
+      alive = __all_sync(0xffffffffu, mbar_wait(&S->y_full, tph, abort_flag, P.status, 25, (int)tile_it));
+      if (!alive) continue;
+      tc_fence_after();
+      const float bias1 = L.has_bias ? 1.0f : 0.0f;
+      float sum = 0.0f;
+      if (active) {
+#pragma unroll
+        for (int ch = 0; ch < 4; ++ch) {
+          uint32_t qv[32];
+          tmem_ld_32x32(tsrc + 256u + (uint32_t)ch * 32u, qv);
+          tmem_ld_wait();
+#pragma unroll
+          for (int j = 0; j < 32; ++j) sum = fmaf(__uint_as_float(pv[ch][j]) + bias1, __uint_as_float(qv[j]), sum);
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&S->y_empty);
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) sum += __shfl_down_sync(0xffffffffu, sum, o);
+      if (lane == 0)
+        P.partial[(size_t)t.i * P.partial_stride + L.partial_base + t.idx * 8 + h * 4 + (int)q] =
+            (t.c0 + h == t.r) ? sum : 2.0f * sum;
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    __syncwarp();
+    tc_fence_after();
+    tmem_dealloc(tmem_base, 512);
+  }
+}
+
+// =================================================================================================
 // Tile kernel: 128 (d_out) x 256 (d_in) output tiles, K = tokens
 // =================================================================================================
 constexpr int T_BK = 128;                              // tokens per stage: one box per operand covers 8 k-steps
@@ -744,6 +964,22 @@ static bool encode_map4(CUtensorMap* map, const void* base, int B, int T, int d,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// bf16 tensor [B, T, d] as (x = feature, y = token, z = example); box = 64 features x box_rows tokens of one
+// example, 128-byte swizzle, out-of-range elements read as zero.
+static bool encode_map3(CUtensorMap* map, const void* base, int B, int T, int d, int box_rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[3] = {(cuuint64_t)d, (cuuint64_t)T, (cuuint64_t)B};
+  const cuuint64_t strides[2] = {(cuuint64_t)d * 2, (cuuint64_t)T * d * 2};
+  const cuuint32_t box[3] = {64u, (cuuint32_t)box_rows, 1u};
+  const cuuint32_t estr[3] = {1u, 1u, 1u};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+            DP_TMA_L2_PROMOTION == 0 ? CU_TENSOR_MAP_L2_PROMOTION_NONE
+            : DP_TMA_L2_PROMOTION == 1 ? CU_TENSOR_MAP_L2_PROMOTION_L2_128B : CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 bool umma_supported(const dp_layer& L) {
   if (L.kind == DP_EMBEDDING) {   // mask-Gram norm only (the accumulate is a scatter, not a contraction)
     return L.dtype == DP_BF16 && L.d_out % 64 == 0 && (reinterpret_cast<uintptr_t>(L.G) & 15u) == 0 &&
@@ -758,11 +994,18 @@ bool umma_supported(const dp_layer& L) {
 
 static int gram_pairs(int T) { const int nb = (T + 127) / 128; return nb * (nb + 1) / 2; }
 static int tile_count(const dp_layer& L) { return ceil_div(L.d_out, 128) * ceil_div(L.d_in, 256); }
+// Gram layers with more than one token block run on the two-column-block kernel (linear layers only: the
+// id-equality mask of an embedding is applied by the one-block-pair kernel).
+static bool gram_wide(const dp_layer& L) { return L.kind == DP_LINEAR && L.T > 128; }
+// fp32 partial sums per example that a layer's norm kernel writes
+static int sqnorm_partials(const dp_layer& L, bool gram) {
+  if (!gram) return 8 * tile_count(L);
+  return gram_wide(L) ? 8 * wide_items((L.T + 127) / 128) : 4 * gram_pairs(L.T);
+}
 
 size_t umma_sqnorm_partials_per_example(const dp_layer* layers, const int* idx, int n, const int* use_gram) {
   size_t c = 0;
-  for (int k = 0; k < n; ++k)
-    c += use_gram[k] ? 4 * (size_t)gram_pairs(layers[idx[k]].T) : 8 * (size_t)tile_count(layers[idx[k]]);
+  for (int k = 0; k < n; ++k) c += (size_t)sqnorm_partials(layers[idx[k]], use_gram[k] != 0);
   return c;
 }
 
@@ -806,16 +1049,55 @@ int launch_umma_sqnorms(const dp_layer* layers, const int* idx, int n, const int
                         int partial_stride, int partial_base, int* status, cudaStream_t s) {
   if (n <= 0) return DP_OK;
   const int B = layers[idx[0]].B, T = layers[idx[0]].T;
-  static bool attr_ok = ensure_smem(k_gram_sqnorm, G_SMEM) && ensure_smem(k_tile_sqnorm, T_SMEM);
+  static bool attr_ok = ensure_smem(k_gram_sqnorm, G_SMEM) && ensure_smem(k_tile_sqnorm, T_SMEM) &&
+                        ensure_smem(k_gram_sqnorm_wide, W_SMEM);
   if (!attr_ok) return DP_ERR_CUDA;
   // Partial slots are assigned in the caller's layer order, whichever kernel fills them.
   std::vector<int> base(n);
   int pos = partial_base;
   for (int k = 0; k < n; ++k) {
     base[k] = pos;
-    pos += use_gram[k] ? 4 * gram_pairs(T) : 8 * tile_count(layers[idx[k]]);
+    pos += sqnorm_partials(layers[idx[k]], use_gram[k] != 0);
   }
-  for (int pass = 0; pass < 2; ++pass) {             // pass 0: Gram layers, pass 1: materialised tiles
+  {   // Gram layers with several token blocks
+    const int per_example = wide_items((T + 127) / 128);
+    int k = 0;
+    while (k < n) {
+      WideParams P;
+      P.n_layers = 0;
+      long long items = 0;
+      for (; k < n && P.n_layers < kWideMaxLayers; ++k) {
+        const dp_layer& L = layers[idx[k]];
+        if (!use_gram[k] || !gram_wide(L)) continue;
+        const long long add = (long long)B * per_example;
+        if (items + add > 0x7fffffffll) break;
+        WideLayer& W = P.L[P.n_layers];
+        if (!encode_map3(&W.rowA, L.A, B, T, L.d_in, 128) || !encode_map3(&W.colA, L.A, B, T, L.d_in, 256) ||
+            !encode_map3(&W.rowG, L.G, B, T, L.d_out, 128) || !encode_map3(&W.colG, L.G, B, T, L.d_out, 256))
+          return DP_ERR_CUDA;
+        W.d_out = L.d_out;
+        W.d_in = L.d_in;
+        W.item_start = (int)items;
+        W.partial_base = base[k];
+        W.has_bias = L.has_bias;
+        for (int& x : W.pad) x = 0;
+        items += add;
+        ++P.n_layers;
+      }
+      if (P.n_layers == 0) continue;
+      P.total_items = (int)items;
+      P.B = B;
+      P.T = T;
+      P.partial_stride = partial_stride;
+      P.pad = 0;
+      P.partial = partial;
+      P.status = status;
+      const int grid = P.total_items < sm_count() ? P.total_items : sm_count();
+      k_gram_sqnorm_wide<<<grid, W_THREADS, W_SMEM, s>>>(P);
+      if (counted(1) != cudaSuccess) return DP_ERR_CUDA;
+    }
+  }
+  for (int pass = 0; pass < 2; ++pass) {             // pass 0: one-block-pair Gram layers, pass 1: materialised tiles
     const bool gram = pass == 0;
     int k = 0;
     while (k < n) {
@@ -824,6 +1106,7 @@ int launch_umma_sqnorms(const dp_layer* layers, const int* idx, int n, const int
       long long items = 0;
       for (; k < n && P.n_layers < kMaxLayers; ++k) {
         if ((use_gram[k] != 0) != gram) continue;
+        if (gram && gram_wide(layers[idx[k]])) continue;
         const dp_layer& L = layers[idx[k]];
         const long long add = (long long)B * (gram ? gram_pairs(T) : tile_count(L));
         if (items + add > 0x7fffffffll) break;
