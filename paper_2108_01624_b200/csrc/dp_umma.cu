@@ -279,10 +279,16 @@ __global__ void __launch_bounds__(G_THREADS, 1) k_gram_sqnorm(const __grid_const
 // full by splitting the epilogue: as soon as P is complete the eight epilogue warps copy it to registers (128
 // per thread) and release its columns, so the UMMAs of the next item's P overlap this item's Q and product-sum.
 // =================================================================================================
-constexpr int W_STAGES = 4;
-constexpr int W_ROW_BYTES = 128 * 128;                  // 128 tokens x 64 bf16 features, 128-byte swizzle
-constexpr int W_COL_BYTES = 256 * 128;                  // 256 tokens x 64 features
-constexpr int W_STAGE_BYTES = W_ROW_BYTES + W_COL_BYTES;
+// Shared memory is a ring of 16 KB units; a stage takes the units it needs (row tile 1, column tile 2 or 1), so
+// the stages of an item whose row tile is also its first column tile occupy 32 KB instead of 48 KB and more of
+// them are in flight.  A stage never straddles the end of the ring: the units left there are skipped.
+#ifndef DP_WIDE_UNITS
+#define DP_WIDE_UNITS 14
+#endif
+constexpr int W_UNITS = DP_WIDE_UNITS;
+constexpr int W_UNIT_BYTES = 128 * 128;                 // 128 tokens x 64 bf16 features, 128-byte swizzle
+constexpr int W_BARS = 16;                              // stage barriers (more than stages can be in flight)
+static_assert(W_UNITS >= 3 && W_UNITS < W_BARS, "a stage of three units must fit, and every stage in flight needs a barrier");
 constexpr int W_THREADS = 320;                          // warp 0 TMA, warp 1 UMMA issue, warps 2..9 epilogue
 constexpr int kWideMaxLayers = 48;
 
@@ -305,11 +311,12 @@ struct WideParams {
 static_assert(sizeof(WideParams) <= 32000, "kernel parameter block too large");
 
 struct WideCtl {
-  uint64_t full[W_STAGES], empty[W_STAGES], x_full, x_empty, y_full, y_empty, drain;
+  uint64_t full[W_BARS], empty[W_BARS], x_full, x_empty, y_full, y_empty, drain;
   uint32_t tmem_base;
   int abort;
 };
-constexpr int W_SMEM = 1024 + W_STAGES * W_STAGE_BYTES + (int)sizeof(WideCtl);
+constexpr int W_SMEM = 1024 + W_UNITS * W_UNIT_BYTES + (int)sizeof(WideCtl);
+static_assert(W_SMEM <= 232448, "over the shared memory of one CTA");
 
 // items of one example: for every row block r the column blocks r, r+1, ... in pairs
 __host__ __device__ inline int wide_items(int nblk) {
@@ -338,12 +345,12 @@ __device__ __forceinline__ WideItem wide_decode(const WideParams& P, int item, i
 __global__ void __launch_bounds__(W_THREADS, 1) k_gram_sqnorm_wide(const __grid_constant__ WideParams P) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* tiles = align1024(smem_raw);
-  WideCtl* S = reinterpret_cast<WideCtl*>(tiles + W_STAGES * W_STAGE_BYTES);
+  WideCtl* S = reinterpret_cast<WideCtl*>(tiles + W_UNITS * W_UNIT_BYTES);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   volatile int* abort_flag = &S->abort;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < W_STAGES; ++s) { mbar_init(&S->full[s], 1); mbar_init(&S->empty[s], 1); }
+    for (int s = 0; s < W_BARS; ++s) { mbar_init(&S->full[s], 1); mbar_init(&S->empty[s], 1); }
     mbar_init(&S->x_full, 1);
     mbar_init(&S->y_full, 1);
     mbar_init(&S->x_empty, 8);
@@ -361,45 +368,62 @@ __global__ void __launch_bounds__(W_THREADS, 1) k_gram_sqnorm_wide(const __grid_
 
   if (warp == 0) {
     if (lane == 0) {   // ---------------- TMA producer ----------------
-      uint32_t it = 0;
+      // Stage n uses barrier n % W_BARS; stages [tail, n) are in flight or unread, `foot` holds the units each of
+      // them took (those skipped at the end of the ring included); they are released in order.
+      uint32_t n = 0, tail = 0;
+      int pos = 0, free_units = W_UNITS;
+      uint8_t foot[W_BARS];
       bool alive = true;
       for (int item = blockIdx.x; item < P.total_items && alive; item += gridDim.x) {
         const WideItem t = wide_decode(P, item, per_example, nblk);
         const WideLayer& L = P.L[t.l];
         const bool diag = t.c0 == t.r;
         // a lone column block is fetched with the 128-token box; rows beyond T arrive as zeros either way
-        const uint32_t bytes = (uint32_t)((diag ? 0 : W_ROW_BYTES) + (t.ncol == 2 ? W_COL_BYTES : W_ROW_BYTES));
+        const int u = (diag ? 0 : 1) + (t.ncol == 2 ? 2 : 1);
         for (int which = 0; which < 2 && alive; ++which) {
           const CUtensorMap* rowmap = which ? &L.rowG : &L.rowA;
           const CUtensorMap* colmap = t.ncol == 2 ? (which ? &L.colG : &L.colA) : rowmap;
           const int d = which ? L.d_out : L.d_in;
-          for (int k0 = 0; k0 < d; k0 += 64) {
-            const uint32_t slot = it % W_STAGES, ph = (it / W_STAGES) & 1u;
-            if (!mbar_wait(&S->empty[slot], ph ^ 1u, abort_flag, P.status, 21, (int)it)) { alive = false; break; }
-            uint8_t* st = tiles + slot * W_STAGE_BYTES;
-            mbar_arrive_expect_tx(&S->full[slot], bytes);
-            if (!diag) tma_load_3d(st, rowmap, &S->full[slot], k0, t.r * 128, t.i);
-            tma_load_3d(st + W_ROW_BYTES, colmap, &S->full[slot], k0, t.c0 * 128, t.i);
-            ++it;
+          for (int k0 = 0; k0 < d && alive; k0 += 64) {
+            const int skip = pos + u > W_UNITS ? W_UNITS - pos : 0;
+            while (free_units < skip + u) {
+              if (!mbar_wait(&S->empty[tail % W_BARS], (tail / W_BARS) & 1u, abort_flag, P.status, 21, (int)tail)) {
+                alive = false;
+                break;
+              }
+              free_units += foot[tail % W_BARS];
+              ++tail;
+            }
+            if (!alive) break;
+            if (skip) pos = 0;
+            uint8_t* st = tiles + pos * W_UNIT_BYTES;
+            uint64_t* bar = &S->full[n % W_BARS];
+            mbar_arrive_expect_tx(bar, (uint32_t)(u * W_UNIT_BYTES));
+            if (!diag) tma_load_3d(st, rowmap, bar, k0, t.r * 128, t.i);
+            tma_load_3d(st + (diag ? 0 : W_UNIT_BYTES), colmap, bar, k0, t.c0 * 128, t.i);
+            foot[n % W_BARS] = (uint8_t)(skip + u);
+            free_units -= skip + u;
+            pos += u;
+            if (pos == W_UNITS) pos = 0;
+            ++n;
           }
         }
       }
-      const uint32_t pending = it < (uint32_t)W_STAGES ? it : (uint32_t)W_STAGES;
-      for (uint32_t k = 0; k < pending; ++k) {
-        const uint32_t j = it - 1 - k;
-        mbar_wait_drain(&S->full[j % W_STAGES], (j / W_STAGES) & 1u, P.status);
-      }
+      // Leave no copy in flight: every stage not yet released must have landed before shared memory is given up.
+      for (uint32_t j = tail; j < n; ++j) mbar_wait_drain(&S->full[j % W_BARS], (j / W_BARS) & 1u, P.status);
     }
   } else if (warp == 1) {
     if (lane == 0) {   // ---------------- MMA issuer ----------------
       constexpr uint32_t IDESC_N256 = idesc_bf16_f32(128, 256, false, false);
       constexpr uint32_t IDESC_N128 = idesc_bf16_f32(128, 128, false, false);
-      uint32_t it = 0, tile_it = 0;
+      uint32_t n = 0, tile_it = 0;
+      int pos = 0;
       bool alive = true;
       for (int item = blockIdx.x; item < P.total_items && alive; item += gridDim.x, ++tile_it) {
         const WideItem t = wide_decode(P, item, per_example, nblk);
         const WideLayer& L = P.L[t.l];
         const bool diag = t.c0 == t.r;
+        const int u = (diag ? 0 : 1) + (t.ncol == 2 ? 2 : 1);
         const uint32_t idesc = t.ncol == 2 ? IDESC_N256 : IDESC_N128;
         const uint32_t tph = tile_it & 1u;
         for (int which = 0; which < 2 && alive; ++which) {
@@ -411,17 +435,20 @@ __global__ void __launch_bounds__(W_THREADS, 1) k_gram_sqnorm_wide(const __grid_
           const int d = which ? L.d_out : L.d_in;
           const uint32_t d_tmem = tmem_base + (uint32_t)which * 256u;
           for (int k0 = 0; k0 < d; k0 += 64) {
-            const uint32_t slot = it % W_STAGES, ph = (it / W_STAGES) & 1u;
-            ++it;
-            if (!mbar_wait(&S->full[slot], ph, abort_flag, P.status, 23, (int)it)) { alive = false; break; }
+            if (pos + u > W_UNITS) pos = 0;              // the same walk over the unit ring as the producer's
+            const uint32_t rowb = smem_u32(tiles + pos * W_UNIT_BYTES);
+            const uint32_t colb = diag ? rowb : rowb + W_UNIT_BYTES;
+            pos += u;
+            if (pos == W_UNITS) pos = 0;
+            const uint32_t b = n % W_BARS, ph = (n / W_BARS) & 1u;
+            ++n;
+            if (!mbar_wait(&S->full[b], ph, abort_flag, P.status, 23, (int)n)) { alive = false; break; }
             tc_fence_after();
-            const uint32_t colb = smem_u32(tiles + slot * W_STAGE_BYTES) + W_ROW_BYTES;
-            const uint32_t rowb = diag ? colb : colb - W_ROW_BYTES;
 #pragma unroll
             for (int k4 = 0; k4 < 4; ++k4)
               umma_bf16(d_tmem, smem_desc_sw128(rowb + k4 * 32, 16, 1024), smem_desc_sw128(colb + k4 * 32, 16, 1024),
                         idesc, (k0 | k4) ? 1u : 0u);
-            umma_commit(&S->empty[slot]);
+            umma_commit(&S->empty[b]);
           }
           if (alive) umma_commit(which ? &S->y_full : &S->x_full);
         }
