@@ -1086,16 +1086,23 @@ int launch_umma_sqnorms(const dp_layer* layers, const int* idx, int n, const int
     base[k] = pos;
     pos += sqnorm_partials(layers[idx[k]], use_gram[k] != 0);
   }
-  {   // Gram layers with several token blocks
+  {   // Gram layers with several token blocks, widest first: items go to the CTAs round-robin, so the last,
+      // partly filled round then holds the shortest items
     const int per_example = wide_items((T + 127) / 128);
-    int k = 0;
-    while (k < n) {
+    std::vector<int> wide;
+    for (int k = 0; k < n; ++k)
+      if (use_gram[k] && gram_wide(layers[idx[k]])) wide.push_back(k);
+    std::stable_sort(wide.begin(), wide.end(), [&](int a, int b) {
+      return layers[idx[a]].d_in + layers[idx[a]].d_out > layers[idx[b]].d_in + layers[idx[b]].d_out;
+    });
+    size_t w = 0;
+    while (w < wide.size()) {
       WideParams P;
       P.n_layers = 0;
       long long items = 0;
-      for (; k < n && P.n_layers < kWideMaxLayers; ++k) {
+      for (; w < wide.size() && P.n_layers < kWideMaxLayers; ++w) {
+        const int k = wide[w];
         const dp_layer& L = layers[idx[k]];
-        if (!use_gram[k] || !gram_wide(L)) continue;
         const long long add = (long long)B * per_example;
         if (items + add > 0x7fffffffll) break;
         WideLayer& W = P.L[P.n_layers];
@@ -1111,7 +1118,7 @@ int launch_umma_sqnorms(const dp_layer* layers, const int* idx, int n, const int
         items += add;
         ++P.n_layers;
       }
-      if (P.n_layers == 0) continue;
+      if (P.n_layers == 0) return DP_ERR_UNSUPPORTED;     // one layer alone has more items than an int holds
       P.total_items = (int)items;
       P.B = B;
       P.T = T;
