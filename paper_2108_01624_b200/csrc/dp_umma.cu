@@ -1,20 +1,21 @@
 // tcgen05 / TMEM / TMA kernels for bf16 linear layers (sm_100a).
 //
-//   k_gram_sqnorm  per-example squared norm by the token-Gram identity
-//                  |A_i^T G_i|_F^2 + |1^T G_i|^2 = < A_i A_i^T + [bias] 1 1^T , G_i G_i^T >.
-//                  Both 128x128 fp32 Grams of a token-block pair live in TMEM (2 x 128 columns,
-//                  double-buffered); operands are K-major 128x64 tiles, two per TMA copy.  For a token
-//                  embedding the input is one-hot, so A_i A_i^T is the token-id equality mask: only
-//                  G_i G_i^T is formed on the tensor cores and the epilogue multiplies it by
-//                  [id_t == id_s] (integer compares).
-//   k_tile_sqnorm  the materialised-tile norm: 128 (d_out) x 256 (d_in) tiles of ONE example's A_i^T G_i
-//                  (one 128x256x16 UMMA per 16 tokens, both operands MN-major straight from the
-//                  row-major activations), squared and summed in the epilogue; the tile never leaves TMEM.
-//   k_accum_pair   the clipped sum acc_w += sum_i c_i A_i^T G_i on CTA pairs (cta_group::2): 256 x 512
-//                  tiles, the per-example factor applied to the G rows in shared memory by the worker
-//                  warps, which also form the bias column sums, so A and G are read from HBM once.
+//   k_gram_sqnorm       per-example squared norm by the token-Gram identity
+//                       |A_i^T G_i|_F^2 + |1^T G_i|^2 = < A_i A_i^T + [bias] 1 1^T , G_i G_i^T >, for T <= 128.
+//                       Both 128x128 fp32 Grams live in TMEM (2 x 128 columns, double-buffered); operands are
+//                       K-major 128x64 tiles, two per TMA copy.  For a token embedding the input is one-hot, so
+//                       A_i A_i^T is the token-id equality mask: only G_i G_i^T is formed on the tensor cores and
+//                       the epilogue multiplies it by [id_t == id_s] (integer compares; any T).
+//   k_gram_sqnorm_wide  the same identity for T > 128: a row block against two column blocks per item
+//                       (128x256 UMMAs), upper triangle of the block grid only.
+//   k_tile_sqnorm_pair  the materialised-tile norm on CTA pairs: 256 (d_out) x 256 (d_in) tiles of ONE example's
+//                       A_i^T G_i (one 256x256x16 UMMA per 16 tokens, both operands MN-major straight from the
+//                       row-major activations), squared and summed in the epilogue; the tile never leaves TMEM.
+//   k_accum_pair        the clipped sum acc_w += sum_i c_i A_i^T G_i on CTA pairs (cta_group::2): 256 x 512
+//                       tiles, the per-example factor applied to the G rows in shared memory by the worker
+//                       warps, which also form the bias column sums, so A and G are read from HBM once.
 //
-// All three are persistent kernels (grid = number of SMs) over a work list decoded on the device from
+// All are persistent kernels (grid = number of SMs) over a work list decoded on the device from
 // per-layer tile counts; roles are warp-specialised (TMA producer / MMA issuer / epilogue or worker warps).
 #include <cuda.h>
 
@@ -513,28 +514,33 @@ __global__ void __launch_bounds__(W_THREADS, 1) k_gram_sqnorm_wide(const __grid_
   }
 }
 
-// =================================================================================================
-// Tile kernel: 128 (d_out) x 256 (d_in) output tiles, K = tokens
-// =================================================================================================
-constexpr int T_BK = 128;                              // tokens per stage: one box per operand covers 8 k-steps
-constexpr int T_STAGES = 2;
-constexpr int T_THREADS = 320;                          // warp 0 TMA, warp 1 UMMA issue, warps 2..9 epilogue
-constexpr int T_ATOM_BYTES = T_BK * 128;               // 128 tokens x 64 bf16 features
-constexpr int T_M_BYTES = 2 * T_ATOM_BYTES;            // G tile: 128 features of d_out
-constexpr int T_N_BYTES = 4 * T_ATOM_BYTES;            // A tile: 256 features of d_in
-constexpr int T_STAGE_BYTES = T_M_BYTES + T_N_BYTES;   // 96 KB
-constexpr uint32_t T_IDESC = idesc_bf16_f32(128, 256, true, true);
+struct TileItem { int l, m0, n0, e, slot; };
+constexpr int T_THREADS = 320;                          // warp 0 TMA, warp 1 UMMA issue (or forwarding), warps 2..9 epilogue
 
-struct TileCtl {
-  uint64_t full[T_STAGES], empty[T_STAGES], tmem_full[2], tmem_empty[2], drain;
+// =================================================================================================
+// Tile kernel on CTA pairs: 256 (d_out) x 256 (d_in) tiles of ONE example's A_i^T G_i (cta_group::2).
+// CTA r of the pair streams G features [m0 + 128 r, +128) (its rows of the tile) and A features
+// [n0 + 128 r, +128) (its half of the N operand): 64 KB per 128-token stage and CTA for 1024 tensor cycles, where
+// a lone CTA with a 128 x 256 tile needs 96 KB (measured: 932 -> 964 TFLOP/s at T=128, 1000 -> 1080 at T=512).  Two 256-column TMEM accumulators per CTA: the square-sum of a
+// tile overlaps the UMMAs of the next.  The odd CTA's warp 1 forwards "my stage has landed" to the even CTA,
+// whose warp 1 issues the UMMAs for both.
+// =================================================================================================
+constexpr int Q_BK = 128;                               // tokens per stage: one box per operand covers 8 k-steps (64-token
+                                                        // stages, twice as many, measured 5-10 % slower: a copy has a fixed cost)
+constexpr int Q_STAGES = 3;
+constexpr int Q_ATOM_BYTES = Q_BK * 128;                // Q_BK tokens x 64 bf16 features
+constexpr int Q_HALF_BYTES = 2 * Q_ATOM_BYTES;          // 128 features
+constexpr int Q_STAGE_BYTES = 2 * Q_HALF_BYTES;         // G rows + A half
+struct TilePairCtl {
+  uint64_t full[Q_STAGES], empty[Q_STAGES], ready[Q_STAGES], tmem_full[2], tmem_empty[2], drain;
   uint32_t tmem_base;
   int abort;
 };
-constexpr int T_SMEM = 1024 + T_STAGES * T_STAGE_BYTES + (int)sizeof(TileCtl);
+constexpr int Q_SMEM = 1024 + Q_STAGES * Q_STAGE_BYTES + (int)sizeof(TilePairCtl);
+static_assert(Q_SMEM <= 232448, "over the shared memory of one CTA");
 
-struct TileItem { int l, m0, n0, e, slot; };
-
-__device__ __forceinline__ TileItem tile_decode(const UmmaParams& P, int item) {
+// tiles_m / tiles_n count 256-wide tiles here; 16 partial sums per tile
+__device__ __forceinline__ TileItem tile_pair_decode(const UmmaParams& P, int item) {
   TileItem t;
   t.l = find_layer(P, item);
   const UmmaLayer& L = P.L[t.l];
@@ -542,101 +548,116 @@ __device__ __forceinline__ TileItem tile_decode(const UmmaParams& P, int item) {
   t.e = rem / tiles;
   const int tile = rem - t.e * tiles;
   const int mt = tile / L.tiles_n;
-  t.m0 = mt * 128;
+  t.m0 = mt * 256;
   t.n0 = (tile - mt * L.tiles_n) * 256;
-  t.slot = L.partial_base + tile * 8;
+  t.slot = L.partial_base + tile * 16;
   return t;
 }
 
-__global__ void __launch_bounds__(T_THREADS, 1) k_tile_sqnorm(const __grid_constant__ UmmaParams P) {
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(T_THREADS, 1)
+k_tile_sqnorm_pair(const __grid_constant__ UmmaParams P) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* tiles = align1024(smem_raw);
-  TileCtl* S = reinterpret_cast<TileCtl*>(tiles + T_STAGES * T_STAGE_BYTES);
+  TilePairCtl* S = reinterpret_cast<TilePairCtl*>(tiles + Q_STAGES * Q_STAGE_BYTES);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   volatile int* abort_flag = &S->abort;
+  const uint32_t rank = cluster_ctarank();
+  const int first_item = (int)cluster_id_x(), item_stride = (int)cluster_count_x();
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < T_STAGES; ++s) {
-      mbar_init(&S->full[s], 1);
-      mbar_init(&S->empty[s], 1);
-    }
-    for (int b = 0; b < 2; ++b) { mbar_init(&S->tmem_full[b], 1); mbar_init(&S->tmem_empty[b], 8); }
+    for (int s = 0; s < Q_STAGES; ++s) { mbar_init(&S->full[s], 1); mbar_init(&S->empty[s], 1); mbar_init(&S->ready[s], 1); }
+    for (int b = 0; b < 2; ++b) { mbar_init(&S->tmem_full[b], 1); mbar_init(&S->tmem_empty[b], 16); }
     mbar_init(&S->drain, 1);
     S->abort = 0;
     fence_mbar_init();
   }
-  if (warp == 1) { tmem_alloc(&S->tmem_base, 512); tmem_relinquish(); }
+  if (warp == 1) { tmem_alloc_pair(&S->tmem_base, 512); tmem_relinquish_pair(); }
   tc_fence_before();
   __syncthreads();
+  cluster_sync_all();           // the peer's barriers are initialised before anyone signals them
   tc_fence_after();
   const uint32_t tmem_base = S->tmem_base;
-  const int n_tb = (P.T + T_BK - 1) / T_BK;
+  const int n_tb = (P.T + Q_BK - 1) / Q_BK;
 
   if (warp == 0) {
-    if (lane == 0) {   // ---------------- TMA producer ----------------
+    if (lane == 0) {   // ---------------- TMA producer (each CTA, its own slices) ----------------
       uint32_t it = 0;
       bool alive = true;
-      for (int item = blockIdx.x; item < P.total_items && alive; item += gridDim.x) {
-        const TileItem t = tile_decode(P, item);
+      for (int item = first_item; item < P.total_items && alive; item += item_stride) {
+        const TileItem t = tile_pair_decode(P, item);
         const UmmaLayer& L = P.L[t.l];
-        const int e = t.e;
         for (int tb = 0; tb < n_tb; ++tb) {
-          const uint32_t slot = it % T_STAGES, ph = (it / T_STAGES) & 1u;
-          if (!mbar_wait(&S->empty[slot], ph ^ 1u, abort_flag, P.status)) { alive = false; break; }
-          uint8_t* st = tiles + slot * T_STAGE_BYTES;
-          // two boxes of 64 features x 128 tokens x (2 | 4) feature groups; tokens beyond T arrive as zeros
-          mbar_arrive_expect_tx(&S->full[slot], (uint32_t)T_STAGE_BYTES);
-          tma_load_4d(st, &L.mapG, &S->full[slot], 0, tb * T_BK, t.m0 / 64, e);
-          tma_load_4d(st + T_M_BYTES, &L.mapA, &S->full[slot], 0, tb * T_BK, t.n0 / 64, e);
+          const uint32_t slot = it % Q_STAGES, ph = (it / Q_STAGES) & 1u;
+          if (!mbar_wait(&S->empty[slot], ph ^ 1u, abort_flag, P.status, 41, (int)it)) { alive = false; break; }
+          uint8_t* st = tiles + slot * Q_STAGE_BYTES;
+          // two boxes of 64 features x Q_BK tokens x 2 feature groups; tokens beyond T and groups beyond the
+          // layer's width arrive as zeros
+          mbar_arrive_expect_tx(&S->full[slot], (uint32_t)Q_STAGE_BYTES);
+          tma_load_4d(st, &L.mapG, &S->full[slot], 0, tb * Q_BK, (t.m0 + 128 * (int)rank) / 64, t.e);
+          tma_load_4d(st + Q_HALF_BYTES, &L.mapA, &S->full[slot], 0, tb * Q_BK, (t.n0 + 128 * (int)rank) / 64, t.e);
           ++it;
         }
       }
-      const uint32_t pending = it < (uint32_t)T_STAGES ? it : (uint32_t)T_STAGES;
+      const uint32_t pending = it < (uint32_t)Q_STAGES ? it : (uint32_t)Q_STAGES;
       for (uint32_t k = 0; k < pending; ++k) {
         const uint32_t j = it - 1 - k;
-        mbar_wait_drain(&S->full[j % T_STAGES], (j / T_STAGES) & 1u, P.status);
+        mbar_wait_drain(&S->full[j % Q_STAGES], (j / Q_STAGES) & 1u, P.status);
       }
     }
   } else if (warp == 1) {
-    if (lane == 0) {   // ---------------- MMA issuer ----------------
+    if (lane == 0 && rank == 1) {   // ---------------- odd CTA: forward "stage landed" to the issuer ----------------
+      uint32_t it = 0;
+      bool alive = true;
+      for (int item = first_item; item < P.total_items && alive; item += item_stride) {
+        for (int tb = 0; tb < n_tb; ++tb, ++it) {
+          const uint32_t slot = it % Q_STAGES, ph = (it / Q_STAGES) & 1u;
+          if (!mbar_wait(&S->full[slot], ph, abort_flag, P.status, 46, (int)it)) { alive = false; break; }
+          mbar_arrive_cluster(&S->ready[slot], 0u);
+        }
+      }
+    } else if (lane == 0) {   // ---------------- even CTA: UMMA issuer ----------------
+      constexpr uint32_t IDESC = idesc_bf16_f32(256, 256, true, true);
       uint32_t it = 0, tile_it = 0;
       bool alive = true;
-      for (int item = blockIdx.x; item < P.total_items && alive; item += gridDim.x, ++tile_it) {
-        const TileItem t = tile_decode(P, item);
+      for (int item = first_item; item < P.total_items && alive; item += item_stride, ++tile_it) {
         const uint32_t buf = tile_it & 1u, tph = (tile_it >> 1) & 1u;
-        if (!mbar_wait(&S->tmem_empty[buf], tph ^ 1u, abort_flag, P.status)) { alive = false; break; }
+        if (!mbar_wait(&S->tmem_empty[buf], tph ^ 1u, abort_flag, P.status, 42, (int)tile_it)) { alive = false; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + buf * 256u;
         uint32_t first = 0;
         for (int tb = 0; tb < n_tb; ++tb) {
-          const uint32_t slot = it % T_STAGES, ph = (it / T_STAGES) & 1u;
+          const uint32_t slot = it % Q_STAGES, ph = (it / Q_STAGES) & 1u;
           ++it;
-          if (!mbar_wait(&S->full[slot], ph, abort_flag, P.status)) { alive = false; break; }
+          if (!mbar_wait(&S->full[slot], ph, abort_flag, P.status, 43, (int)it) ||
+              !mbar_wait(&S->ready[slot], ph, abort_flag, P.status, 47, (int)it)) {
+            alive = false;
+            break;
+          }
           tc_fence_after();
-          const uint32_t am = smem_u32(tiles + slot * T_STAGE_BYTES), an = am + T_M_BYTES;
-          const int left = P.T - tb * T_BK, nk = left >= T_BK ? T_BK / 16 : (left + 15) >> 4;   // k-steps that hold tokens
+          const uint32_t am = smem_u32(tiles + slot * Q_STAGE_BYTES), an = am + Q_HALF_BYTES;
+          const int left = P.T - tb * Q_BK, nk = left >= Q_BK ? Q_BK / 16 : (left + 15) >> 4;   // k-steps that hold tokens
 #pragma unroll
-          for (int k8 = 0; k8 < T_BK / 16; ++k8) {
+          for (int k8 = 0; k8 < Q_BK / 16; ++k8) {
             if (k8 < nk)
-              umma_bf16(d_tmem, smem_desc_sw128(am + k8 * 2048, T_ATOM_BYTES, 1024),
-                        smem_desc_sw128(an + k8 * 2048, T_ATOM_BYTES, 1024), T_IDESC, first | (uint32_t)k8);
+              umma_bf16_pair(d_tmem, smem_desc_sw128(am + k8 * 2048, Q_ATOM_BYTES, 1024),
+                             smem_desc_sw128(an + k8 * 2048, Q_ATOM_BYTES, 1024), IDESC, first | (uint32_t)k8);
           }
           first = 1;
-          umma_commit(&S->empty[slot]);
+          umma_commit_pair(&S->empty[slot], (uint16_t)3);
         }
-        if (alive) umma_commit(&S->tmem_full[buf]);
+        if (alive) umma_commit_pair(&S->tmem_full[buf], (uint16_t)3);
       }
-      umma_commit(&S->drain);
+      umma_commit_pair(&S->drain, (uint16_t)1);
       mbar_wait_drain(&S->drain, 0u, P.status);
     }
   } else {   // ---------------- epilogue warps 2..9: lanes [32 q, +32), accumulator columns [128 h, +128) ----------------
     const uint32_t q = (uint32_t)warp & 3u, h = warp >= 6 ? 1u : 0u;
     uint32_t tile_it = 0;
     bool alive = true;
-    for (int item = blockIdx.x; item < P.total_items; item += gridDim.x, ++tile_it) {
-      const TileItem t = tile_decode(P, item);
+    for (int item = first_item; item < P.total_items; item += item_stride, ++tile_it) {
+      const TileItem t = tile_pair_decode(P, item);
       const uint32_t buf = tile_it & 1u, tph = (tile_it >> 1) & 1u;
-      if (alive) alive = __all_sync(0xffffffffu, mbar_wait(&S->tmem_full[buf], tph, abort_flag, P.status));
+      if (alive) alive = __all_sync(0xffffffffu, mbar_wait(&S->tmem_full[buf], tph, abort_flag, P.status, 44, (int)tile_it));
       if (!alive) continue;
       tc_fence_after();
       float sum = 0.0f;
@@ -646,22 +667,22 @@ __global__ void __launch_bounds__(T_THREADS, 1) k_tile_sqnorm(const __grid_const
         tmem_ld_32x32(tmem_base + ((q * 32u) << 16) + buf * 256u + h * 128u + (uint32_t)ch * 32u, v);
         tmem_ld_wait();
 #pragma unroll
-          for (int j = 0; j < 32; ++j) sum = fmaf(__uint_as_float(v[j]), __uint_as_float(v[j]), sum);
+        for (int j = 0; j < 32; ++j) sum = fmaf(__uint_as_float(v[j]), __uint_as_float(v[j]), sum);
       }
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(&S->tmem_empty[buf]);
+      if (lane == 0) mbar_arrive_cluster(&S->tmem_empty[buf], 0u);
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) sum += __shfl_down_sync(0xffffffffu, sum, o);
-      if (lane == 0) P.partial[(size_t)t.e * P.partial_stride + t.slot + (int)(h * 4u + q)] = sum;
+      if (lane == 0) P.partial[(size_t)t.e * P.partial_stride + t.slot + (int)(rank * 8u + h * 4u + q)] = sum;
     }
   }
   tc_fence_before();
   __syncthreads();
+  cluster_sync_all();           // neither CTA leaves while the other may still read its memory or signal it
   if (warp == 1) {
-    __syncwarp();
     tc_fence_after();
-    tmem_dealloc(tmem_base, 512);
+    tmem_dealloc_pair(tmem_base, 512);
   }
 }
 
@@ -1020,13 +1041,14 @@ bool umma_supported(const dp_layer& L) {
 }
 
 static int gram_pairs(int T) { const int nb = (T + 127) / 128; return nb * (nb + 1) / 2; }
-static int tile_count(const dp_layer& L) { return ceil_div(L.d_out, 128) * ceil_div(L.d_in, 256); }
+static int tile_count(const dp_layer& L) { return ceil_div(L.d_out, 256) * ceil_div(L.d_in, 256); }
+static int tile_partials(const dp_layer& L) { return 16 * tile_count(L); }
 // Gram layers with more than one token block run on the two-column-block kernel (linear layers only: the
 // id-equality mask of an embedding is applied by the one-block-pair kernel).
 static bool gram_wide(const dp_layer& L) { return L.kind == DP_LINEAR && L.T > 128; }
 // fp32 partial sums per example that a layer's norm kernel writes
 static int sqnorm_partials(const dp_layer& L, bool gram) {
-  if (!gram) return 8 * tile_count(L);
+  if (!gram) return tile_partials(L);
   return gram_wide(L) ? 8 * wide_items((L.T + 127) / 128) : 4 * gram_pairs(L.T);
 }
 
@@ -1076,8 +1098,8 @@ int launch_umma_sqnorms(const dp_layer* layers, const int* idx, int n, const int
                         int partial_stride, int partial_base, int* status, cudaStream_t s) {
   if (n <= 0) return DP_OK;
   const int B = layers[idx[0]].B, T = layers[idx[0]].T;
-  static bool attr_ok = ensure_smem(k_gram_sqnorm, G_SMEM) && ensure_smem(k_tile_sqnorm, T_SMEM) &&
-                        ensure_smem(k_gram_sqnorm_wide, W_SMEM);
+  static bool attr_ok = ensure_smem(k_gram_sqnorm, G_SMEM) &&
+                        ensure_smem(k_gram_sqnorm_wide, W_SMEM) && ensure_smem(k_tile_sqnorm_pair, Q_SMEM);
   if (!attr_ok) return DP_ERR_CUDA;
   // Partial slots are assigned in the caller's layer order, whichever kernel fills them.
   std::vector<int> base(n);
@@ -1145,7 +1167,11 @@ int launch_umma_sqnorms(const dp_layer* layers, const int* idx, int n, const int
         const long long add = (long long)B * (gram ? gram_pairs(T) : tile_count(L));
         if (items + add > 0x7fffffffll) break;
         UmmaLayer& U = P.L[P.n_layers];
-        if (!(gram ? fill_layer(U, L, 128, G_GROUPS, G_GROUPS) : fill_layer(U, L, T_BK, 2, 4))) return DP_ERR_CUDA;
+        if (!(gram ? fill_layer(U, L, 128, G_GROUPS, G_GROUPS) : fill_layer(U, L, Q_BK, 2, 2))) return DP_ERR_CUDA;
+        if (!gram) {
+          U.tiles_m = (uint16_t)ceil_div(L.d_out, 256);
+          U.tiles_n = (uint16_t)ceil_div(L.d_in, 256);
+        }
         U.item_start = (int)items;
         U.partial_base = base[k];
         items += add;
@@ -1163,8 +1189,12 @@ int launch_umma_sqnorms(const dp_layer* layers, const int* idx, int n, const int
       P.partial = partial;
       P.status = status;
       const int grid = P.total_items < sm_count() ? P.total_items : sm_count();
-      if (gram) k_gram_sqnorm<<<grid, G_THREADS, G_SMEM, s>>>(P);
-      else      k_tile_sqnorm<<<grid, T_THREADS, T_SMEM, s>>>(P);
+      if (gram) {
+        k_gram_sqnorm<<<grid, G_THREADS, G_SMEM, s>>>(P);
+      } else {
+        const int units = sm_count() / 2;
+        k_tile_sqnorm_pair<<<2 * (P.total_items < units ? P.total_items : units), T_THREADS, Q_SMEM, s>>>(P);
+      }
       if (counted(1) != cudaSuccess) return DP_ERR_CUDA;
     }
   }
