@@ -154,6 +154,31 @@ def test_tensor_core_tile_edges(B, T):
     check_against_checker(data, C, [b.DP_PATH_MATERIALIZED] * len(WIDE))
 
 
+@pytest.mark.parametrize("B,T", [(3, 129), (2, 256), (3, 300), (2, 384), (2, 640), (1, 700)])
+def test_long_examples_gram_and_tiles(B, T):
+    """More than one 128-token block per example: the Gram kernel pairs the column blocks of every row block
+    (two blocks = one item; three and five blocks leave a lone last column, with and without the row block in it;
+    token counts that end inside a block), and the tile kernel runs several token stages per tile.  Both forced
+    paths against the checker, with embedding and LayerNorm layers beside the linear ones."""
+    specs = [LayerSpec(LINEAR, 192, 320, True, "w192x320"), LayerSpec(LINEAR, 64, 128, False, "w64x128"),
+             LayerSpec(LAYERNORM, 128, 128, False, "ln"), LayerSpec(EMBEDDING, 50, 64, False, "emb")]
+    data = random_layers(specs, B, T, torch.bfloat16, DEV, seed=7 * T + B, g_scale=0.02, vocab_dup=12)
+    ol = to_oracle_layers(data)
+    C = float(np.sqrt(np.median(O.per_example_sqnorms(ol))))
+    check_against_checker(data, C, [b.DP_PATH_GRAM] * len(specs))
+    check_against_checker(data, C, [b.DP_PATH_MATERIALIZED] * len(specs))
+
+
+def test_more_long_gram_layers_than_one_launch_holds():
+    """60 linear layers at T = 160: the Gram launch for examples of several token blocks takes 48 layers, so this
+    needs two, widest layers first; the partial sums still land in the caller's layer order."""
+    specs = [LayerSpec(LINEAR, 64 * (1 + k % 3), 64 * (1 + (k // 3) % 2), k % 2 == 0, f"l{k}") for k in range(60)]
+    data = random_layers(specs, 2, 160, torch.bfloat16, DEV, seed=9, g_scale=0.02)
+    ol = to_oracle_layers(data)
+    C = float(np.sqrt(np.median(O.per_example_sqnorms(ol))))
+    check_against_checker(data, C, [b.DP_PATH_GRAM] * len(specs))
+
+
 def test_more_linear_layers_than_one_launch_holds():
     """130 small linear layers: the tensor-core launches take at most 96 layers each, and the accumulate GEMM packs
     every launch's layers into waves of its own."""
