@@ -29,6 +29,9 @@ the Box-Muller transform, with the uniforms formed in IEEE binary32 so that a
 GPU can reproduce the same uniforms bit for bit and the transcendental part
 evaluated in fp64.
 
+A table shared by the embedding and the output projection (BERT's masked-LM
+head) is clipped by the norm of its summed gradient (shared_table_*).
+
 Pins (tests/test_oracle_pins.py): C -> infinity equals the batch GEMM; every
 clipped contribution has norm <= C; Gram-identity norm equals brute force on
 tiny inputs; rank-one closed form; Philox known-answer vectors and an
@@ -110,6 +113,62 @@ def per_example_sqnorms(layers: Sequence[OracleLayer]) -> np.ndarray:
         for layer in layers:
             for g in per_example_gradient(layer, i):
                 total += float(np.sum(g * g))
+        n[i] = total
+    return n
+
+
+# ---------------------------------------------------------------------------
+# A table shared by the token embedding and the output projection
+# ---------------------------------------------------------------------------
+# The paper trains BERT-Large (Section 4) and does not restate its architecture;
+# in that model the masked-LM output projection reuses the word-piece table E
+# of Section 4.3's embeddings: logits[s, v] = <h[s, :], E[v, :]>.  Example i's
+# gradient for E is then ONE tensor, the sum of the embedding's scatter and of
+# the projection's dlogits_i^T h_i, and Algorithm 1 clips by the norm of that
+# sum, not by the two parts' norms added up.
+
+def shared_table_gradient(emb: OracleLayer, proj: OracleLayer, i: int) -> np.ndarray:
+    """[V, d] gradient of example i for a table used by both layers.
+
+    emb   EMBEDDING layer (ids [B, T], G [B, T, d]).
+    proj  LINEAR layer without bias whose A is dlogits [B, T_out, V] and whose
+          G is the projection's input h [B, T_out, d], so that its A_i^T G_i is
+          the [V, d] gradient of the table.
+    """
+    scatter = per_example_gradient(emb, i)[0]
+    dense = per_example_gradient(proj, i)[0]
+    assert scatter.shape == dense.shape
+    return scatter + dense
+
+
+def shared_table_cross_terms(emb: OracleLayer, proj: OracleLayer) -> np.ndarray:
+    """x_i = <scatter_i, dense_i> (sum of elementwise products of the two
+    materialised [V, d] parts): ||scatter_i + dense_i||^2 exceeds the two
+    parts' squared norms by 2 x_i."""
+    B = emb.B
+    x = np.zeros(B, dtype=np.float64)
+    for i in range(B):
+        scatter = per_example_gradient(emb, i)[0]
+        dense = per_example_gradient(proj, i)[0]
+        x[i] = float(np.sum(scatter * dense))
+    return x
+
+
+def per_example_sqnorms_shared_table(layers: Sequence[OracleLayer], emb_index: int, proj_index: int) -> np.ndarray:
+    """n_i over all layers when layers[emb_index] and layers[proj_index] train
+    the same table: every other layer as in per_example_sqnorms, the shared
+    table once, by the norm of its summed gradient."""
+    B = layers[0].B
+    n = np.zeros(B, dtype=np.float64)
+    for i in range(B):
+        total = 0.0
+        for k, layer in enumerate(layers):
+            if k in (emb_index, proj_index):
+                continue
+            for g in per_example_gradient(layer, i):
+                total += float(np.sum(g * g))
+        g = shared_table_gradient(layers[emb_index], layers[proj_index], i)
+        total += float(np.sum(g * g))
         n[i] = total
     return n
 

@@ -370,3 +370,84 @@ def test_gradient_snr_sums_closed_forms(rng):
 def test_clip_stats_values():
     assert O.clip_stats(np.array([1.0, 1.0, 0.5, 0.25])) == (0.5, 0.6875)
     assert O.clip_stats(np.ones(7)) == (0.0, 1.0)
+
+
+# ------------------------------------------------------------------ a table shared by embedding and output projection
+
+def _shared_table_case(rng, B=3, T=5, T_out=4, V=7, d=6):
+    emb = O.OracleLayer(kind=O.EMBEDDING, G=rng.standard_normal((B, T, d)), ids=rng.integers(0, V, (B, T)), vocab=V)
+    proj = O.OracleLayer(kind=O.LINEAR, A=rng.standard_normal((B, T_out, V)), G=rng.standard_normal((B, T_out, d)))
+    return emb, proj
+
+
+def test_shared_table_gradient_matches_scalar_loops(rng):
+    """dE[v, :] = sum_{t: id_t = v} G_emb[t, :] + sum_s dlogits[s, v] h[s, :], written out with scalar loops."""
+    emb, proj = _shared_table_case(rng)
+    B, T, d = emb.G.shape
+    T_out, V = proj.A.shape[1], proj.A.shape[2]
+    for i in range(B):
+        ref = np.zeros((V, d))
+        for t in range(T):
+            for q in range(d):
+                ref[emb.ids[i, t], q] += emb.G[i, t, q]
+        for s in range(T_out):
+            for v in range(V):
+                for q in range(d):
+                    ref[v, q] += proj.A[i, s, v] * proj.G[i, s, q]
+        np.testing.assert_allclose(O.shared_table_gradient(emb, proj, i), ref, rtol=1e-12, atol=1e-12)
+
+
+def test_shared_table_norm_is_the_parts_plus_twice_the_cross_term(rng):
+    """Polarisation: ||s + d||^2 = ||s||^2 + ||d||^2 + 2 <s, d>, with the parts' norms taken from the functions
+    pinned above, and <s, d> also by the token-pair form sum_{t,s} dlogits[s, id_t] <h[s], G_emb[t]>."""
+    emb, proj = _shared_table_case(rng, B=4, T=6, T_out=3, V=5, d=8)     # V < T: ids repeat
+    other = O.OracleLayer(kind=O.LAYERNORM, A=rng.standard_normal((4, 6, 8)), G=rng.standard_normal((4, 6, 8)))
+    x = O.shared_table_cross_terms(emb, proj)
+    n_sep = O.per_example_sqnorms([emb, other, proj])
+    n_tied = O.per_example_sqnorms_shared_table([emb, other, proj], 0, 2)
+    np.testing.assert_allclose(n_tied, n_sep + 2.0 * x, rtol=1e-12)
+    for i in range(4):
+        pair = 0.0
+        for t in range(6):
+            for s in range(3):
+                pair += proj.A[i, s, emb.ids[i, t]] * float(np.dot(proj.G[i, s], emb.G[i, t]))
+        assert abs(pair - x[i]) <= 1e-12 * max(1.0, abs(x[i]))
+    assert np.max(np.abs(x)) > 1e-3            # the term is not negligible on random inputs
+
+
+def test_shared_table_cross_term_closed_forms(rng):
+    """One token with id k and one output position whose dlogits is alpha on vocabulary entry k': the scatter is
+    g at row k, the dense part alpha h at row k', so <s, d> = alpha <h, g> if k' = k and 0 otherwise."""
+    d, V = 5, 4
+    g, h = rng.standard_normal(d), rng.standard_normal(d)
+    for k, kp in ((2, 2), (2, 3)):
+        emb = O.OracleLayer(kind=O.EMBEDDING, G=g.reshape(1, 1, d), ids=np.array([[k]]), vocab=V)
+        A = np.zeros((1, 1, V))
+        A[0, 0, kp] = 0.7
+        proj = O.OracleLayer(kind=O.LINEAR, A=A, G=h.reshape(1, 1, d))
+        x = O.shared_table_cross_terms(emb, proj)[0]
+        assert abs(x - (0.7 * float(h @ g) if k == kp else 0.0)) <= 1e-14
+    # zero output gradients: the shared table's norm is the embedding's alone
+    emb, proj = _shared_table_case(rng)
+    proj.A[:] = 0.0
+    np.testing.assert_allclose(O.per_example_sqnorms_shared_table([emb, proj], 0, 1), O.per_example_sqnorms([emb]),
+                               rtol=1e-12)
+
+
+def test_shared_table_accumulates_into_one_tensor(rng):
+    """Both layers add into the same [V, d] accumulator; with C -> infinity the result is the batch gradient of
+    the table, scatter of all rows plus dlogits^T h over all examples and positions."""
+    emb, proj = _shared_table_case(rng, B=5)
+    accs = O.zero_accumulators([emb, proj])
+    accs[1][0] = accs[0][0]                     # one tensor, two contributors
+    O.clipped_accumulate([emb, proj], np.ones(5), accs)
+    V, d = accs[0][0].shape
+    ref = np.zeros((V, d))
+    np.add.at(ref, emb.ids.reshape(-1), emb.G.reshape(-1, d))
+    ref += proj.A.reshape(-1, V).T @ proj.G.reshape(-1, d)
+    np.testing.assert_allclose(accs[0][0], ref, rtol=1e-12, atol=1e-12)
+    # every clipped contribution of the shared table stays within C
+    n = O.per_example_sqnorms_shared_table([emb, proj], 0, 1)
+    c = O.clip_factors(n, 0.5)
+    for i in range(5):
+        assert c[i] * np.linalg.norm(O.shared_table_gradient(emb, proj, i)) <= 0.5 * (1 + 1e-12)
