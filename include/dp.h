@@ -180,6 +180,25 @@ DP_API int dp_reduce_noise_adamw_step(float* theta, float* m, float* v, float* c
  * Section 5.2.1): out[0] = fraction of examples with clip_i < 1, out[1] = mean clip_i.  out: device float[2]. */
 DP_API int dp_clip_stats(const float* clip, int B, float* out, void* cuda_stream);
 
+/* A table trained through two layers: the token embedding and an output projection onto the same table.
+ * (Section 4.3 names the word-piece embedding; the model of Section 4 is BERT-Large, whose masked-LM head
+ * projects onto that table, logits[s, v] = <h[s, :], E[v, :]>; the paper does not restate this.)  Example i's gradient
+ * for the table is then ONE tensor, scatter_i + dlogits_i^T h_i, and Algorithm 1's clip acts on the norm of that sum:
+ * the two parts' squared norms, plus twice their inner product.  Pass the embedding as a DP_EMBEDDING layer and the
+ * projection as a DP_LINEAR layer without bias whose A is dlogits [B, T_out, V] (d_in = V) and whose G is the
+ * projection's input h [B, T_out, d] (d_out = d), both with acc_w = the table's [V, d] accumulator (each in a call
+ * with its own token count, the second with accumulate_into = 1): dp_per_example_sqnorms then adds the two parts
+ * and dp_clipped_accumulate sums both into the table.  This call adds the inner product,
+ *   sqnorm[i] += 2 * sum_{t < T} sum_{s < T_out} dlogits[i, s, ids[i, t]] * <h[i, s, :], G_emb[i, t, :]>,
+ * and must run before dp_clip_factors.  ids int32 [B, T]; G_emb [B, T, d]; dlogits [B, T_out, V]; h [B, T_out, d];
+ * all three of `dtype` (DP_F32 or DP_BF16), row-major, device pointers owned by the caller; sqnorm fp32 [B].
+ * fp32 accumulation in a fixed order.  A token id outside [0, V) is skipped and reported by dp_poll_status
+ * (DP_ERR_BAD_ID).  DP_ERR_ARG on null pointers or non-positive sizes, DP_ERR_ALIGN on pointers not aligned to
+ * their element size. */
+DP_API int dp_shared_table_cross_sqnorms(const int32_t* ids, const void* G_emb, int B, int T, const void* dlogits,
+                                         const void* h, int T_out, int d, int V, int dtype, float* sqnorm,
+                                         void* cuda_stream);
+
 /* Test utility: out[k] = the raw Philox word of element elem_offset + k (lane (e & 3) of block e >> 2). */
 DP_API int dp_philox_u32(uint32_t* out, int64_t n_words, int64_t elem_offset, uint64_t seed, uint64_t step,
                   void* cuda_stream);

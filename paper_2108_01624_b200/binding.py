@@ -24,7 +24,7 @@ _KINDS = {"linear": DP_LINEAR, "layernorm": DP_LAYERNORM, "embedding": DP_EMBEDD
 
 EXPORTS = ["dp_workspace_bytes", "dp_per_example_sqnorms", "dp_clip_factors", "dp_clipped_accumulate", "dp_clipped_accumulate_after_sqnorms", "dp_accumulate_schedule", "dp_reduce_noise_adamw_step",
            "dp_add_noise_and_scale", "dp_adamw_step", "dp_noise_scale_adamw_step", "dp_noise_scale_adamw_step_snr",
-           "dp_clip_stats", "dp_philox_u32",
+           "dp_clip_stats", "dp_philox_u32", "dp_shared_table_cross_sqnorms",
            "dp_token_equality_mask", "dp_layernorm_sqnorms_static", "dp_poll_status", "dp_last_timeout_info", "dp_launch_count",
            "dp_status_string", "dp_version"]
 
@@ -72,6 +72,7 @@ def lib() -> C.CDLL:
         L.dp_clip_stats.argtypes = [vp, i32, vp, vp]
         L.dp_philox_u32.argtypes = [vp, i64, i64, u64, u64, vp]
         L.dp_token_equality_mask.argtypes = [vp, i32, i32, vp, vp]
+        L.dp_shared_table_cross_sqnorms.argtypes = [vp, vp, i32, i32, vp, vp, i32, i32, i32, i32, vp, vp]
         L.dp_layernorm_sqnorms_static.argtypes = [vp, vp, i32, vp]
         L.dp_poll_status.argtypes = [vp]
         L.dp_status_string.restype = C.c_char_p
@@ -185,6 +186,22 @@ def dp_per_example_sqnorms(layers: LayerList, sqnorm: torch.Tensor, accumulate_i
     _check("dp_per_example_sqnorms",
            lib().dp_per_example_sqnorms(layers.ptr, len(layers), _ptr(sqnorm), int(accumulate_into), ws_p, ws_n,
                                         _stream(stream)))
+    return sqnorm
+
+
+def dp_shared_table_cross_sqnorms(emb: Layer, proj: Layer, sqnorm: torch.Tensor, stream=None) -> torch.Tensor:
+    """sqnorm[i] += 2 <scatter_i, dlogits_i^T h_i> for a table trained through the embedding layer `emb` and the
+    output projection `proj` (a linear layer whose A is dlogits [B, T_out, V] and whose G is h [B, T_out, d])."""
+    B, T, d = emb.G.shape
+    _, T_out, V = proj.A.shape
+    if emb.ids is None or emb.ids.dtype != torch.int32 or proj.A.dtype != emb.G.dtype or proj.G.dtype != emb.G.dtype:
+        raise ValueError("embedding ids (int32) and one dtype for G_emb, dlogits and h expected")
+    if proj.G.shape != (B, T_out, d) or int(emb.vocab) != V:
+        raise ValueError("the projection must map [B, T_out, V] x [B, T_out, d] onto the embedding's [V, d] table")
+    dtype = DP_F32 if emb.G.dtype == torch.float32 else DP_BF16
+    _check("dp_shared_table_cross_sqnorms",
+           lib().dp_shared_table_cross_sqnorms(_ptr(emb.ids), _ptr(emb.G), B, T, _ptr(proj.A), _ptr(proj.G), T_out, d, V,
+                                               dtype, _ptr(sqnorm), _stream(stream)))
     return sqnorm
 
 

@@ -400,6 +400,21 @@ int dp_philox_u32(uint32_t* out, int64_t n_words, int64_t elem_offset, uint64_t 
   return DP_OK;
 }
 
+int dp_shared_table_cross_sqnorms(const int32_t* ids, const void* G_emb, int B, int T, const void* dlogits,
+                                  const void* h, int T_out, int d, int V, int dtype, float* sqnorm, void* cuda_stream) {
+  if (!ids || !G_emb || !dlogits || !h || !sqnorm) return DP_ERR_ARG;
+  if (B <= 0 || T <= 0 || T_out <= 0 || d <= 0 || V <= 0) return DP_ERR_ARG;
+  if (dtype != DP_F32 && dtype != DP_BF16) return DP_ERR_ARG;
+  const size_t es = dtype == DP_F32 ? 4 : 2;
+  if (misaligned(ids, 4) || misaligned(sqnorm, 4) || misaligned(G_emb, es) || misaligned(dlogits, es) || misaligned(h, es))
+    return DP_ERR_ALIGN;
+  int* status = status_ptr();
+  if (!status) return DP_ERR_CUDA;
+  DP_CUDA(launch_shared_table_cross(ids, G_emb, B, T, dlogits, h, T_out, d, V, dtype, sqnorm, status,
+                                    static_cast<cudaStream_t>(cuda_stream)));
+  return DP_OK;
+}
+
 int dp_token_equality_mask(const int32_t* ids, int B, int T, uint8_t* mask, void* cuda_stream) {
   if (!ids || !mask || B <= 0 || T <= 0) return DP_ERR_ARG;
   if (misaligned(ids, 4)) return DP_ERR_ALIGN;

@@ -567,4 +567,87 @@ cudaError_t launch_embedding_accum(const dp_layer& L, const float* clip, int* st
   return counted(1);
 }
 
+// ---------------------------------------------------------------------------------------------
+// Cross term of a table shared by a token embedding and an output projection: example i's gradient for the table
+// is scatter_i + dlogits_i^T h_i, and <scatter_i, dlogits_i^T h_i> = sum_{t,s} dlogits[s, id_t] <h[s,:], G_emb[t,:]>.
+// One CTA per example walks the T_out x T grid of token pairs in 64 x 64 blocks (a 4 x 4 micro-tile per thread,
+// the feature dimension staged through shared memory 32 at a time) and weighs every inner product with the
+// gathered output gradient.  Fixed order of summation: the result does not depend on the launch.
+// ---------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void __launch_bounds__(256)
+k_shared_table_cross(const int32_t* __restrict__ ids, const T* __restrict__ Gemb, const T* __restrict__ dlogits,
+                     const T* __restrict__ H, int Tn, int Tout, int d, int V, float* __restrict__ sqnorm,
+                     int* __restrict__ status) {
+  __shared__ float Hs[64][33], Gs[64][33];
+  __shared__ float red[32];
+  const int i = blockIdx.x;
+  const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
+  const T* Hi = H + (size_t)i * Tout * d;
+  const T* Gi = Gemb + (size_t)i * Tn * d;
+  const T* Di = dlogits + (size_t)i * Tout * V;
+  const int32_t* idi = ids + (size_t)i * Tn;
+  float total = 0.0f;
+  for (int s0 = 0; s0 < Tout; s0 += 64) {
+    for (int t0 = 0; t0 < Tn; t0 += 64) {
+      float acc[4][4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u)
+#pragma unroll
+        for (int v = 0; v < 4; ++v) acc[u][v] = 0.0f;
+      for (int k0 = 0; k0 < d; k0 += 32) {
+        for (int e = threadIdx.x; e < 64 * 32; e += 256) {
+          const int r = e >> 5, c = e & 31;
+          const bool kin = k0 + c < d;
+          Hs[r][c] = (kin && s0 + r < Tout) ? ldf(Hi + (size_t)(s0 + r) * d + k0 + c) : 0.0f;
+          Gs[r][c] = (kin && t0 + r < Tn) ? ldf(Gi + (size_t)(t0 + r) * d + k0 + c) : 0.0f;
+        }
+        __syncthreads();
+#pragma unroll 8
+        for (int c = 0; c < 32; ++c) {
+          float a[4], bb[4];
+#pragma unroll
+          for (int u = 0; u < 4; ++u) { a[u] = Hs[ty * 4 + u][c]; bb[u] = Gs[tx * 4 + u][c]; }
+#pragma unroll
+          for (int u = 0; u < 4; ++u)
+#pragma unroll
+            for (int v = 0; v < 4; ++v) acc[u][v] = fmaf(a[u], bb[v], acc[u][v]);
+        }
+        __syncthreads();
+      }
+#pragma unroll
+      for (int v = 0; v < 4; ++v) {
+        const int t = t0 + tx * 4 + v;
+        if (t >= Tn) continue;
+        const int id = idi[t];
+        if (id < 0 || id >= V) {                     // skipped and reported, like the embedding kernels
+          atomicCAS(status, STATUS_OK, STATUS_BAD_ID);
+          continue;
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const int sx = s0 + ty * 4 + u;
+          if (sx < Tout) total = fmaf(acc[u][v], ldf(Di + (size_t)sx * V + id), total);
+        }
+      }
+    }
+  }
+  total = block_sum(total, red);
+  if (threadIdx.x == 0) sqnorm[i] += 2.0f * total;
+}
+
+cudaError_t launch_shared_table_cross(const int32_t* ids, const void* G_emb, int B, int T, const void* dlogits,
+                                      const void* h, int T_out, int d, int V, int dtype, float* sqnorm, int* status,
+                                      cudaStream_t s) {
+  if (dtype == DP_F32)
+    k_shared_table_cross<float><<<B, 256, 0, s>>>(ids, static_cast<const float*>(G_emb), static_cast<const float*>(dlogits),
+                                                  static_cast<const float*>(h), T, T_out, d, V, sqnorm, status);
+  else
+    k_shared_table_cross<__nv_bfloat16><<<B, 256, 0, s>>>(ids, static_cast<const __nv_bfloat16*>(G_emb),
+                                                          static_cast<const __nv_bfloat16*>(dlogits),
+                                                          static_cast<const __nv_bfloat16*>(h), T, T_out, d, V, sqnorm,
+                                                          status);
+  return counted(1);
+}
+
 }  // namespace dpk

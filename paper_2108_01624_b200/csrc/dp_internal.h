@@ -65,6 +65,10 @@ cudaError_t launch_weighted_rows_sum_batched(const ColTaskHost* tasks, int n, co
 // Embedding by grouping equal ids inside an example.
 cudaError_t launch_embedding_sqnorm(const dp_layer& L, float* sqnorm, int* status, cudaStream_t s);
 cudaError_t launch_embedding_accum(const dp_layer& L, const float* clip, int* status, cudaStream_t s);
+// sqnorm[i] += 2 <scatter_i, dlogits_i^T h_i> for a table shared by an embedding and an output projection.
+cudaError_t launch_shared_table_cross(const int32_t* ids, const void* G_emb, int B, int T, const void* dlogits,
+                                      const void* h, int T_out, int d, int V, int dtype, float* sqnorm, int* status,
+                                      cudaStream_t s);
 cudaError_t launch_fill_zero(float* p, long long n, cudaStream_t s);
 // sqnorm[i] (+)= sum of partial[i * stride + j], j < count, in a fixed order.
 cudaError_t launch_reduce_partials(const float* partial, int B, int count, float* sqnorm, cudaStream_t s);

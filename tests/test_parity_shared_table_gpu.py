@@ -1,0 +1,129 @@
+"""GPU parity for a table trained through two layers (token embedding + output projection onto the same table, the
+masked-LM head of BERT): the cross term of the squared norm, the whole norm -> clip -> accumulate flow into one
+accumulator, the BERT-Large-sized case on sampled examples, and the report of an out-of-range token id."""
+import numpy as np
+import pytest
+import torch
+
+from .helpers import EMBEDDING, LINEAR, LayerData, LayerSpec, O, b, rel_l2, to_np, to_oracle_layers
+
+pytestmark = pytest.mark.gpu
+
+if not torch.cuda.is_available():
+    pytest.skip("needs a CUDA device", allow_module_level=True)
+
+DEV = "cuda:0"
+CLIP_TOL = 1e-3
+BF16_TOL = 2e-2
+
+
+def _case(B, T, T_out, V, d, dtype, seed, scale=1.0, correlated=False):
+    """Embedding (ids repeat when V < T) and projection (A = dlogits, G = h) on the device, as LayerData.
+    correlated: position s of the projection sees a hidden state aligned with token s's embedding gradient and
+    pushes on that token's own vocabulary entry, so that the two parts of the table's gradient overlap."""
+    g = torch.Generator().manual_seed(seed)
+    ids = torch.randint(0, V, (B, T), generator=g, dtype=torch.int32)
+    G_emb = torch.randn(B, T, d, generator=g) * scale
+    dlogits = torch.randn(B, T_out, V, generator=g) * scale
+    h = torch.randn(B, T_out, d, generator=g)
+    if correlated:
+        h = h + 2.0 * G_emb[:, :T_out, :] / scale
+        dlogits.scatter_add_(2, ids[:, :T_out, None].long(), torch.full((B, T_out, 1), 3.0 * scale))
+    ids, G_emb, dlogits, h = ids.to(DEV), G_emb.to(dtype).to(DEV), dlogits.to(dtype).to(DEV), h.to(dtype).to(DEV)
+    emb = LayerData(LayerSpec(EMBEDDING, V, d, False, "tok_emb"), G=G_emb, ids=ids)
+    proj = LayerData(LayerSpec(LINEAR, V, d, False, "mlm_decoder"), G=h, A=dlogits)
+    return emb, proj
+
+
+def _layers(emb, proj, acc):
+    le = b.Layer(kind=EMBEDDING, G=emb.G, ids=emb.ids, acc_w=acc, vocab=emb.spec.d_in)
+    lp = b.Layer(kind=LINEAR, G=proj.G, A=proj.A, acc_w=acc, has_bias=False)
+    return le, lp
+
+
+@pytest.mark.parametrize("dtype,tol", [(torch.float32, 1e-4), (torch.bfloat16, 1e-3)])
+@pytest.mark.parametrize("B,T,T_out,V,d", [(3, 37, 20, 50, 96), (2, 150, 130, 40, 72), (1, 1, 1, 3, 5), (4, 64, 65, 700, 33)])
+def test_cross_term_matches_checker(dtype, tol, B, T, T_out, V, d):
+    emb, proj = _case(B, T, T_out, V, d, dtype, seed=T + T_out)
+    oe, op = to_oracle_layers([emb, proj])
+    x_ref = O.shared_table_cross_terms(oe, op)
+    scale = np.sqrt(O.per_example_sqnorms([oe]) * O.per_example_sqnorms([op]))     # |<s, d>| <= ||s|| ||d||
+    le, lp = _layers(emb, proj, torch.zeros(V, d, device=DEV))
+    sq = torch.full((B,), 3.0, dtype=torch.float32, device=DEV)                     # adds into what is there
+    b.dp_shared_table_cross_sqnorms(le, lp, sq)
+    assert b.dp_poll_status() == 0
+    assert np.max(np.abs(to_np(sq) - 3.0 - 2.0 * x_ref) / (scale + 3.0)) <= tol
+
+
+@pytest.mark.parametrize("dtype,V,d", [(torch.float32, 50, 40), (torch.bfloat16, 128, 64), (torch.bfloat16, 100, 64)])
+def test_shared_table_norm_clip_accumulate(dtype, V, d):
+    """Two calls with different token counts, the cross term, one clip, both layers summed into ONE accumulator."""
+    B, T, T_out = 6, 48, 20
+    emb, proj = _case(B, T, T_out, V, d, dtype, seed=11, scale=0.05, correlated=True)
+    oe, op = to_oracle_layers([emb, proj])
+    n_ref = O.per_example_sqnorms_shared_table([oe, op], 0, 1)
+    C = float(np.sqrt(np.median(n_ref)))
+    c_ref = O.clip_factors(n_ref, C)
+    acc = torch.zeros(V, d, device=DEV)
+    le, lp = _layers(emb, proj, acc)
+    ll_e, ll_p = b.LayerList([le]), b.LayerList([lp])
+    ws_e, ws_p = b.alloc_workspace(ll_e), b.alloc_workspace(ll_p)
+    sq = torch.empty(B, dtype=torch.float32, device=DEV)
+    clip = torch.empty_like(sq)
+    b.dp_per_example_sqnorms(ll_e, sq, False, ws_e)
+    b.dp_per_example_sqnorms(ll_p, sq, True, ws_p)
+    b.dp_shared_table_cross_sqnorms(le, lp, sq)
+    b.dp_clip_factors(sq, C, clip)
+    b.dp_clipped_accumulate(ll_e, clip, ws_e)
+    b.dp_clipped_accumulate(ll_p, clip, ws_p)
+    assert b.dp_poll_status() == 0
+    np.testing.assert_allclose(to_np(sq), n_ref, rtol=2 * CLIP_TOL)
+    np.testing.assert_allclose(to_np(clip), c_ref, rtol=CLIP_TOL)
+    assert 0 < int((c_ref < 1).sum()) < B                      # both branches of the clip
+    accs = O.zero_accumulators([oe, op])
+    accs[1][0] = accs[0][0]
+    O.clipped_accumulate([oe, op], c_ref, accs)
+    assert rel_l2(to_np(acc), accs[0][0]) <= (1e-4 if dtype == torch.float32 else BF16_TOL)
+    # without the cross term the norms would be visibly off on these inputs
+    assert np.max(np.abs(O.per_example_sqnorms([oe, op]) / n_ref - 1.0)) > 10 * CLIP_TOL
+
+
+def test_bert_large_sized_table_on_sampled_examples():
+    """30528 x 1024 table (the vocabulary padded to a multiple of 64), 128 tokens, 20 masked positions, B = 256 in
+    one launch; the checker materialises the [V, d] gradient of three examples spread over the batch."""
+    B, T, T_out, V, d = 256, 128, 20, 30528, 1024
+    emb, proj = _case(B, T, T_out, V, d, torch.bfloat16, seed=5, scale=0.01)
+    ids = emb.ids.clone()
+    ids[:, ::3] = ids[:, ::3] % 50                              # frequent ids, as under a Zipf law: rows repeat
+    emb = LayerData(emb.spec, G=emb.G, ids=ids.contiguous())
+    le, lp = _layers(emb, proj, None)
+    sq = torch.zeros(B, dtype=torch.float32, device=DEV)
+    b.dp_shared_table_cross_sqnorms(le, lp, sq)
+    assert b.dp_poll_status() == 0
+    got = to_np(sq)
+    for i in (0, 131, 255):
+        sub = [LayerData(emb.spec, G=emb.G[i:i + 1].contiguous(), ids=emb.ids[i:i + 1].contiguous()),
+               LayerData(proj.spec, G=proj.G[i:i + 1].contiguous(), A=proj.A[i:i + 1].contiguous())]
+        oe, op = to_oracle_layers(sub)
+        x = O.shared_table_cross_terms(oe, op)[0]
+        scale = float(np.sqrt(O.per_example_sqnorms([oe])[0] * O.per_example_sqnorms([op])[0]))
+        assert abs(got[i] - 2.0 * x) <= 1e-3 * scale, (i, got[i], 2.0 * x, scale)
+
+
+def test_out_of_range_id_is_skipped_and_reported():
+    emb, proj = _case(2, 9, 4, 10, 8, torch.float32, seed=3)
+    ids = emb.ids.clone()
+    ids[1, 4] = 10                                              # == V
+    oe, op = to_oracle_layers([emb, proj])
+    # the checker with that token's row zeroed = the token skipped
+    G0 = emb.G.clone()
+    G0[1, 4] = 0
+    oe0 = to_oracle_layers([LayerData(emb.spec, G=G0, ids=emb.ids)])[0]
+    x_ref = O.shared_table_cross_terms(oe0, op)
+    bad = LayerData(emb.spec, G=emb.G, ids=ids.contiguous())
+    le, lp = _layers(bad, proj, None)
+    sq = torch.zeros(2, dtype=torch.float32, device=DEV)
+    b.dp_shared_table_cross_sqnorms(le, lp, sq)
+    assert b.dp_poll_status() == -7                             # DP_ERR_BAD_ID
+    assert b.dp_poll_status() == 0                              # the report is read once
+    np.testing.assert_allclose(to_np(sq), 2.0 * x_ref, rtol=1e-4, atol=1e-5)
