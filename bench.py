@@ -205,7 +205,7 @@ def main():
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--blocks", type=int, default=24,
                     help="encoder blocks of the stack (24 = the benchmark workload; fewer only for profiler captures)")
     ap.add_argument("--macro-microbatches", type=int, default=0,
@@ -273,18 +273,23 @@ def main():
             dist.destroy_process_group()
         return
 
-    def one_step(ev=None):
+    def make_lists(d):
+        ll = step.layer_list(d)
+        return pkg.LayerList([ll.layers[k] for k in lin_idx]), pkg.LayerList([ll.layers[k] for k in rest_idx])
+
+    def one_step(ev=None, lists=None):
+        lin, rest = (ll_lin, ll_rest) if lists is None else lists
         if ev:
             ev[0].record(stream)
-        pkg.dp_per_example_sqnorms(ll_lin, sq, False, ws)
-        pkg.dp_per_example_sqnorms(ll_rest, sq, True, ws_rest)
+        pkg.dp_per_example_sqnorms(lin, sq, False, ws)
+        pkg.dp_per_example_sqnorms(rest, sq, True, ws_rest)
         pkg.dp_clip_factors(sq, wl.C, clip)
         if ev:
             ev[1].record(stream)
-        pkg.dp_clipped_accumulate(ll_lin, clip, ws)
+        pkg.dp_clipped_accumulate(lin, clip, ws)
         if ev:
             ev[2].record(stream)
-        pkg.dp_clipped_accumulate_after_sqnorms(ll_rest, clip, ws_rest)
+        pkg.dp_clipped_accumulate_after_sqnorms(rest, clip, ws_rest)
         if ev:
             ev[3].record(stream)
         step.examples_seen = wl.B * world
@@ -354,7 +359,7 @@ def main():
 
     e2e = None
     if not args.no_e2e and world == 1:
-        e2e = run_e2e(pkg, wl, data, one_step, clip, stream, args.e2e_steps)
+        e2e = run_e2e(pkg, synth, wl, data, one_step, make_lists, clip, stream, args.e2e_steps)
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         cpu_baseline = time_oracle(wl, data, n_params)
@@ -504,38 +509,59 @@ def run_macro_step(args, pkg, synth, wl, step, sharded, dist, world, rank, dev, 
             "gpu_launches": int(launches), "clocks": clocks}))
 
 
-def run_e2e(pkg, wl, data, one_step, clip, stream, n_steps):
-    """Same step through the public API with HOST buffers: every step copies all layer inputs from pinned host
-    memory to the device and reads the clip factors back."""
+def run_e2e(pkg, synth, wl, data, one_step, make_lists, clip, stream, n_steps):
+    """Same step through the public API with HOST buffers: every step copies all of its layer inputs from pinned
+    host memory to the device and reads the clip factors back.  The inputs of step k + 1 are copied (on a second
+    stream, into a second set of device buffers) while step k computes, as a training loop would prefetch them;
+    the link is the bound either way (32 GB per step)."""
     host = []
     try:
         for ld in data:
             host.append([None if t is None else torch.empty(t.shape, dtype=t.dtype, pin_memory=True).copy_(t)
                          for t in (ld.A, ld.G, ld.ids)])
-        mirror = "full pinned mirror of every layer's inputs"
+        mirror = "full pinned mirror of every layer's inputs; two device input sets, copy of step k+1 under step k"
+        sets = [data, [synth.LayerData(ld.spec, G=torch.empty_like(ld.G), A=None if ld.A is None else torch.empty_like(ld.A),
+                                       ids=None if ld.ids is None else torch.empty_like(ld.ids)) for ld in data]]
     except RuntimeError:
-        host = None
-    if host is None:
         return None
+    lists = [None, make_lists(sets[1])]
     clip_h = torch.empty(clip.shape, dtype=clip.dtype, pin_memory=True)
     h2d = sum(t.numel() * t.element_size() for h in host for t in h if t is not None)
     d2h = clip_h.numel() * clip_h.element_size()
+    copier = torch.cuda.Stream()
+    copied = [torch.cuda.Event(), torch.cuda.Event()]
+    done = [torch.cuda.Event(), torch.cuda.Event()]
 
-    def e2e_step():
-        for ld, h in zip(data, host):
-            for dst, src in zip((ld.A, ld.G, ld.ids), h):
-                if dst is not None:
-                    dst.copy_(src, non_blocking=True)
-        one_step()
+    def copy_in(k):          # inputs of step k into set k % 2, once the step that last used that set has finished
+        with torch.cuda.stream(copier):
+            copier.wait_event(done[k % 2])
+            for ld, h in zip(sets[k % 2], host):
+                for dst, src in zip((ld.A, ld.G, ld.ids), h):
+                    if dst is not None:
+                        dst.copy_(src, non_blocking=True)
+            copied[k % 2].record(copier)
+
+    def compute(k):
+        stream.wait_event(copied[k % 2])
+        one_step(lists=lists[k % 2])
         clip_h.copy_(clip, non_blocking=True)
+        done[k % 2].record(stream)
 
-    e2e_step()
+    def run(n):
+        for ev in done:
+            ev.record(stream)
+        copy_in(0)
+        for k in range(n):
+            if k + 1 < n:
+                copy_in(k + 1)
+            compute(k)
+            stream.synchronize()      # the host reads the step's result before it goes on
+
+    run(1)
     torch.cuda.synchronize()
     a, b_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     a.record(stream)
-    for _ in range(n_steps):
-        e2e_step()
-        stream.synchronize()
+    run(n_steps)
     b_.record(stream)
     torch.cuda.synchronize()
     ms = a.elapsed_time(b_) / n_steps
