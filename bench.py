@@ -214,6 +214,9 @@ def main():
     ap.add_argument("--long-sequence-paths", action="store_true",
                     help="instead of the per-microbatch line: the T=512 BERT-Large block (B=64) with the norm path of "
                          "its linear layers forced to Gram, forced to materialised tiles, and chosen automatically")
+    ap.add_argument("--verify", action="store_true",
+                    help="with --macro-microbatches: check the accumulator after the loop (untimed) against the "
+                         "counted sum of single passes over the pool, and against the bound N C")
     ap.add_argument("--pool", type=int, default=2,
                     help="distinct resident microbatches the macro-step rotates over (32 GB each)")
     args = ap.parse_args()
@@ -476,20 +479,40 @@ def run_macro_step(args, pkg, synth, wl, step, sharded, dist, world, rank, dev, 
     sampler = ClockSampler(dev.index or 0)
     sampler.start()
     l0 = pkg.dp_launch_count()
-    t0, t1, t2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+    t0, t1, t1b, t2 = (torch.cuda.Event(enable_timing=True) for _ in range(4))
     barrier()
     t0.record(stream)
     for k in range(M):
         microbatch(k)
     t1.record(stream)
+    launches = pkg.dp_launch_count() - l0
+    verify = None
+    if args.verify:
+        # Untimed: the accumulator after M microbatches against count_p x (one pass over pool entry p), summed in
+        # fp64; and the bound ||sum of clipped gradients|| <= N C that clipping guarantees.
+        acc_loop = step.acc.clone()
+        ref = torch.zeros(step.n_flat, dtype=torch.float64, device=dev)
+        for p_ in range(len(lists)):
+            step.acc.zero_()
+            microbatch(p_)
+            ref += step.acc.double() * float(len(range(p_, M, len(lists))))
+        step.acc.copy_(acc_loop)
+        diff = float((acc_loop.double() - ref).norm() / ref.norm())
+        norm = float(acc_loop.double().norm())
+        verify = {"rel_l2_vs_counted_single_passes": diff, "acc_norm": norm, "bound_N_times_C": wl.B * M * wl.C,
+                  "within_bound": bool(norm <= wl.B * M * wl.C * (1 + 1e-3))}
+        del acc_loop, ref
+    l1 = pkg.dp_launch_count()
+    t1b.record(stream)
     finish()
     t2.record(stream)
     barrier()
-    launches = pkg.dp_launch_count() - l0
+    launches += pkg.dp_launch_count() - l1
     clocks = sampler.stop()
     if pkg.dp_poll_status() != 0:
         raise RuntimeError("device status not clean after the macro-step")
-    total_ms, upd_ms = t0.elapsed_time(t2), t1.elapsed_time(t2)
+    upd_ms = t1b.elapsed_time(t2)
+    total_ms = t0.elapsed_time(t1) + upd_ms
     if dist is not None:
         t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
@@ -506,7 +529,7 @@ def run_macro_step(args, pkg, synth, wl, step, sharded, dist, world, rank, dev, 
             "config": {"workload": name, "B": wl.B, "T": wl.T, "microbatches_per_step": M, "examples_per_step": N,
                        "resident_microbatch_pool": len(lists), "params": wl.n_params(), "parallelism": f"dp{world}",
                        "l2": "inputs (32 GB per microbatch) far exceed L2; no flush"},
-            "gpu_launches": int(launches), "clocks": clocks}))
+            "verify": verify, "gpu_launches": int(launches), "clocks": clocks}))
 
 
 def run_e2e(pkg, synth, wl, data, one_step, make_lists, clip, stream, n_steps):
