@@ -44,7 +44,7 @@ typedef enum {
   DP_OK = 0,
   DP_ERR_ARG = -1,         /* null pointer, non-positive size, non-finite scalar, bad enum */
   DP_ERR_ALIGN = -2,       /* pointer not aligned as required */
-  DP_ERR_UNSUPPORTED = -3, /* valid request this build cannot run (e.g. forced path on a shape it excludes) */
+  DP_ERR_UNSUPPORTED = -3, /* valid request the library cannot run (e.g. forced path on a shape it excludes) */
   DP_ERR_CUDA = -4,        /* a CUDA runtime/driver call failed */
   DP_ERR_TIMEOUT = -5,     /* a bounded device-side wait ran out (reported by dp_poll_status) */
   DP_ERR_WORKSPACE = -6,   /* workspace missing, misaligned or too small */
