@@ -127,3 +127,73 @@ def test_out_of_range_id_is_skipped_and_reported():
     assert b.dp_poll_status() == -7                             # DP_ERR_BAD_ID
     assert b.dp_poll_status() == 0                              # the report is read once
     np.testing.assert_allclose(to_np(sq), 2.0 * x_ref, rtol=1e-4, atol=1e-5)
+
+
+def test_bert_heads_in_three_token_groups_with_tied_decoder():
+    """The tensors of BERT outside the encoder stack, through the C ABI in three calls with their own token counts:
+    per token (word-piece table, a stand-in encoder layer), per masked position (MLM transform, its LayerNorm, the
+    decoder tied to the word-piece table, the output bias as a 1 x V linear layer over a column of ones), per
+    example (pooler and next-sentence classifier on the first token).  One norm over everything, one clip, every
+    tensor's clipped sum against the checker; the table receives both of its contributions."""
+    B, T, T_out, V, d = 5, 24, 20, 128, 64
+    g = torch.Generator().manual_seed(21)
+    dt = torch.bfloat16
+
+    def rnd(*shape, scale=1.0):
+        return (torch.randn(*shape, generator=g) * scale).to(dt).to(DEV)
+
+    ids = torch.randint(0, V, (B, T), generator=g, dtype=torch.int32).to(DEV)
+    dlogits = rnd(B, T_out, V, scale=0.05)
+    ones = torch.ones(B, T_out, 1, dtype=dt, device=DEV)
+    specs = {
+        "tok_emb": LayerData(LayerSpec(EMBEDDING, V, d, False, "tok_emb"), G=rnd(B, T, d, scale=0.05), ids=ids),
+        "enc": LayerData(LayerSpec(LINEAR, d, d, True, "enc"), G=rnd(B, T, d, scale=0.02), A=rnd(B, T, d)),
+        "mlm_dense": LayerData(LayerSpec(LINEAR, d, d, True, "mlm_dense"), G=rnd(B, T_out, d, scale=0.05), A=rnd(B, T_out, d)),
+        "mlm_ln": LayerData(LayerSpec("layernorm", d, d, False, "mlm_ln"), G=rnd(B, T_out, d, scale=0.05), A=rnd(B, T_out, d)),
+        "decoder": LayerData(LayerSpec(LINEAR, V, d, False, "decoder"), G=rnd(B, T_out, d), A=dlogits),
+        "out_bias": LayerData(LayerSpec(LINEAR, 1, V, False, "out_bias"), G=dlogits, A=ones),
+        "pooler": LayerData(LayerSpec(LINEAR, d, d, True, "pooler"), G=rnd(B, 1, d, scale=0.3), A=rnd(B, 1, d)),
+        "nsp": LayerData(LayerSpec(LINEAR, d, 2, True, "nsp"), G=rnd(B, 1, 2, scale=0.3), A=rnd(B, 1, d)),
+    }
+    groups = [["tok_emb", "enc"], ["mlm_dense", "mlm_ln", "decoder", "out_bias"], ["pooler", "nsp"]]
+    names = [n for grp in groups for n in grp]
+    table = torch.zeros(V, d, device=DEV)
+
+    def acc_for(name):
+        sp = specs[name].spec
+        if name in ("tok_emb", "decoder"):
+            return [table]
+        if sp.kind == LINEAR:
+            return [torch.zeros(sp.d_in, sp.d_out, device=DEV)] + ([torch.zeros(sp.d_out, device=DEV)] if sp.has_bias else [])
+        return [torch.zeros(d, device=DEV), torch.zeros(d, device=DEV)]
+
+    accs = {n: acc_for(n) for n in names}
+    layer = {}
+    for n in names:
+        ld, a = specs[n], accs[n]
+        layer[n] = b.Layer(kind=ld.spec.kind, G=ld.G, A=ld.A, ids=ld.ids, acc_w=a[0], acc_b=a[1] if len(a) > 1 else None,
+                           has_bias=ld.spec.has_bias, vocab=V if ld.spec.kind == EMBEDDING else 0)
+    lists = [b.LayerList([layer[n] for n in grp]) for grp in groups]
+    wss = [b.alloc_workspace(ll) for ll in lists]
+    sq = torch.empty(B, dtype=torch.float32, device=DEV)
+    clip = torch.empty_like(sq)
+    for k, (ll, ws) in enumerate(zip(lists, wss)):
+        b.dp_per_example_sqnorms(ll, sq, k > 0, ws)
+    b.dp_shared_table_cross_sqnorms(layer["tok_emb"], layer["decoder"], sq)
+
+    ol = to_oracle_layers([specs[n] for n in names])
+    n_ref = O.per_example_sqnorms_shared_table(ol, names.index("tok_emb"), names.index("decoder"))
+    C = float(np.sqrt(np.median(n_ref)))
+    c_ref = O.clip_factors(n_ref, C)
+    b.dp_clip_factors(sq, C, clip)
+    for ll, ws in zip(lists, wss):
+        b.dp_clipped_accumulate(ll, clip, ws)
+    assert b.dp_poll_status() == 0
+    np.testing.assert_allclose(to_np(sq), n_ref, rtol=2 * CLIP_TOL)
+    np.testing.assert_allclose(to_np(clip), c_ref, rtol=CLIP_TOL)
+    ref = O.zero_accumulators(ol)
+    ref[names.index("decoder")][0] = ref[names.index("tok_emb")][0]
+    O.clipped_accumulate(ol, c_ref, ref)
+    for k, n in enumerate(names):
+        for x, y in zip(accs[n], ref[k]):
+            assert x.shape == y.shape and rel_l2(to_np(x), y) <= BF16_TOL, n
