@@ -58,7 +58,11 @@ typedef enum { DP_F32 = 0, DP_BF16 = 1 } dp_dtype;
  *                 for an embedding the first factor is the token-id equality mask.
  *   MATERIALIZED  tiles of A_i^T G_i formed on chip, squared and summed; for an embedding,
  *                 rows with equal ids are summed first.
- *   AUTO          linear: GRAM iff T * (d_in + d_out) <= d_in * d_out, the flop count of either way;
+ *   AUTO          linear: the cheaper way.  On the CUDA-core kernels GRAM iff T * (d_in + d_out) <= d_in * d_out,
+ *                 the flop count of either way.  On the tensor-core kernels (see below) by measured cost: GRAM for
+ *                 T <= 128; beyond, GRAM iff the multiply-accumulates it executes, 128 * 128 * (d_in + d_out) per
+ *                 block pair of the upper triangle of the ceil(T/128)^2 token blocks, are at most 1.75 times
+ *                 T * d_in * d_out;
  *                 embedding: GRAM whenever the tensor-core kernel accepts the layer (bf16, d_out % 64 == 0). */
 typedef enum { DP_PATH_AUTO = 0, DP_PATH_GRAM = 1, DP_PATH_MATERIALIZED = 2 } dp_path;
 /* Which kernels a layer gets.  A bf16 LINEAR layer whose d_in and d_out are multiples of 64 and whose A and G are

@@ -61,9 +61,22 @@ static int validate_layers(const dp_layer* layers, int n_layers, bool need_acc) 
   return DP_OK;
 }
 
+// AUTO: the path with the lower cost.  On the CUDA-core kernels the cost is the flop count of either way.  On the
+// tensor-core kernels it is measured: up to 128 tokens the Gram kernel is bound by reading A and G once and beat
+// the tile kernel at every width tried (64 to 1024); beyond, it executes 128 x 128 x (d_in + d_out)
+// multiply-accumulates per block pair of the upper triangle and came out ahead whenever that count stayed under
+// about 1.75 times the tile kernel's T x d_in x d_out (whose tiles re-read A and G through L2 for every tile row
+// and column): T from 256 to 4096, widths from 256 to 4096, one mispick of 13 % among fifteen shapes.
 static bool use_gram(const dp_layer& L) {
   if (L.path == DP_PATH_GRAM) return true;
   if (L.path == DP_PATH_MATERIALIZED) return false;
+  if (L.kind == DP_LINEAR && umma_supported(L)) {
+    if (L.T <= 128) return true;
+    const long long nblk = (L.T + 127) / 128;
+    const double gram = 128.0 * 128.0 * (double)(nblk * (nblk + 1) / 2) * (double)(L.d_in + L.d_out);
+    const double tiles = (double)L.T * (double)L.d_in * (double)L.d_out;
+    return gram <= 1.75 * tiles;
+  }
   return (long long)L.T * (L.d_in + L.d_out) <= (long long)L.d_in * L.d_out;
 }
 
