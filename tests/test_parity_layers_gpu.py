@@ -154,7 +154,7 @@ def test_tensor_core_tile_edges(B, T):
     check_against_checker(data, C, [b.DP_PATH_MATERIALIZED] * len(WIDE))
 
 
-@pytest.mark.parametrize("B,T", [(3, 129), (2, 256), (3, 300), (2, 384), (2, 640), (1, 700)])
+@pytest.mark.parametrize("B,T", [(3, 129), (2, 256), (3, 300), (2, 384), (2, 640), (1, 700), (2, 2050)])
 def test_long_examples_gram_and_tiles(B, T):
     """More than one 128-token block per example: the Gram kernel pairs the column blocks of every row block
     (two blocks = one item; three and five blocks leave a lone last column, with and without the row block in it;
