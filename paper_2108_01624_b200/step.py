@@ -24,15 +24,30 @@ class DPStep:
 
     def __init__(self, specs: Sequence[LayerSpec], device, C: float, sigma: float, lr: float, beta1: float,
                  beta2: float, xi: float, weight_decay: float, seed: int = 0, theta: Optional[torch.Tensor] = None,
-                 track_snr: bool = False):
+                 track_snr: bool = False, shared_tables: Optional[dict] = None):
+        """shared_tables maps the index of an output-projection spec (a bias-free LINEAR layer with d_in = V whose
+        A is dlogits and whose G is the projection's input) to the index of the EMBEDDING spec whose [V, d] table it
+        also trains (BERT's masked-LM decoder): the projection gets no storage of its own, both layers accumulate into
+        the table, and the per-example norm includes the inner product of their two contributions."""
         self.specs = list(specs)
+        self.shared_tables = dict(shared_tables or {})
+        for p_li, e_li in self.shared_tables.items():
+            sp, se = self.specs[p_li], self.specs[e_li]
+            if not (e_li < p_li and se.kind == EMBEDDING and sp.kind == LINEAR and not sp.has_bias
+                    and sp.d_in == se.d_in and sp.d_out == se.d_out):
+                raise ValueError("a shared table needs an EMBEDDING [V, d] listed before a bias-free LINEAR V -> d")
         self.device = torch.device(device)
         self.C, self.sigma, self.lr, self.beta1, self.beta2 = C, sigma, lr, beta1, beta2
         self.xi, self.weight_decay, self.seed = xi, weight_decay, seed
         self.offsets: List[List[int]] = []
         self.shapes: List[List[tuple]] = []
         pos = 0
-        for sp in self.specs:
+        for li, sp in enumerate(self.specs):
+            if li in self.shared_tables:              # alias of the embedding's table
+                e_li = self.shared_tables[li]
+                self.offsets.append(list(self.offsets[e_li]))
+                self.shapes.append(list(self.shapes[e_li]))
+                continue
             if sp.kind == LINEAR:
                 shp = [(sp.d_in, sp.d_out)] + ([(sp.d_out,)] if sp.has_bias else [])
             elif sp.kind == LAYERNORM:
@@ -82,18 +97,43 @@ class DPStep:
                                path=b.DP_PATH_AUTO if paths is None else paths[li]))
         return b.LayerList(out)
 
-    def accumulate_microbatch(self, layers: b.LayerList, stream=None):
-        """norms -> clip factors -> clipped accumulate for one microbatch (all enqueued, no sync)."""
-        B = layers.B
+    def layer_lists(self, data: Sequence[LayerData], paths: Optional[Sequence[int]] = None) -> List[b.LayerList]:
+        """Descriptors for one microbatch whose layers do not all see the same number of tokens (encoder layers per
+        token, the masked-LM head per masked position, pooler and sentence classifier per example): one list per
+        token count, in order of first appearance; accumulate_microbatch takes the result."""
+        whole = self.layer_list(data, paths)
+        groups: dict = {}
+        for L in whole.layers:
+            groups.setdefault(int(L.G.shape[1]), []).append(L)
+        return [b.LayerList(ls) for ls in groups.values()]
+
+    def accumulate_microbatch(self, layers, stream=None):
+        """norms -> clip factors -> clipped accumulate for one microbatch (all enqueued, no sync).
+        `layers` is a LayerList, or a list of them (layer_lists) when token counts differ between layers."""
+        lists = [layers] if isinstance(layers, b.LayerList) else list(layers)
+        B = lists[0].B
         if self._sqnorm is None or self._sqnorm.numel() != B:
             self._sqnorm = torch.empty(B, dtype=torch.float32, device=self.device)
             self._clip = torch.empty(B, dtype=torch.float32, device=self.device)
-        need = b.dp_workspace_bytes(layers)
-        if self._ws is None or self._ws.numel() < need:
-            self._ws = torch.empty(max(need, 256), dtype=torch.uint8, device=self.device)
-        b.dp_per_example_sqnorms(layers, self._sqnorm, False, self._ws, stream)
+        if self._ws is None or len(self._ws) != len(lists):
+            self._ws = [None] * len(lists)
+        for k, ll in enumerate(lists):
+            need = b.dp_workspace_bytes(ll)
+            if self._ws[k] is None or self._ws[k].numel() < need:
+                self._ws[k] = torch.empty(max(need, 256), dtype=torch.uint8, device=self.device)
+            b.dp_per_example_sqnorms(ll, self._sqnorm, k > 0, self._ws[k], stream)
+        if self.shared_tables:
+            by_acc = {}
+            for ll in lists:
+                for L in ll.layers:
+                    by_acc.setdefault(L.acc_w.data_ptr(), []).append(L)
+            for pair in by_acc.values():          # an embedding and the projection that shares its accumulator
+                if len(pair) == 2:
+                    emb, proj = (pair[0], pair[1]) if pair[0].kind == EMBEDDING else (pair[1], pair[0])
+                    b.dp_shared_table_cross_sqnorms(emb, proj, self._sqnorm, stream)
         b.dp_clip_factors(self._sqnorm, self.C, self._clip, stream)
-        b.dp_clipped_accumulate_after_sqnorms(layers, self._clip, self._ws, stream)
+        for k, ll in enumerate(lists):
+            b.dp_clipped_accumulate_after_sqnorms(ll, self._clip, self._ws[k], stream)
         self.examples_seen += B
         return self._sqnorm, self._clip
 

@@ -197,3 +197,68 @@ def test_bert_heads_in_three_token_groups_with_tied_decoder():
     for k, n in enumerate(names):
         for x, y in zip(accs[n], ref[k]):
             assert x.shape == y.shape and rel_l2(to_np(x), y) <= BF16_TOL, n
+
+
+def test_dpstep_with_token_groups_and_a_shared_table():
+    """The same model through DPStep: layers grouped by token count, the decoder aliased onto the word-piece table
+    (no storage of its own in the flat parameter vector), two microbatches, then noise + AdamW over the flat vector
+    against the checker."""
+    from paper_2108_01624_b200 import DPStep, synth
+    B, T, T_out, V, d = 4, 24, 20, 128, 64
+    dt = torch.bfloat16
+    spec_list = [LayerSpec(EMBEDDING, V, d, False, "tok_emb"), LayerSpec(LINEAR, d, d, True, "enc"),
+                 LayerSpec(LINEAR, d, d, True, "mlm_dense"), LayerSpec("layernorm", d, d, False, "mlm_ln"),
+                 LayerSpec(LINEAR, V, d, False, "decoder"), LayerSpec(LINEAR, 1, V, False, "out_bias"),
+                 LayerSpec(LINEAR, d, d, True, "pooler"), LayerSpec(LINEAR, d, 2, True, "nsp")]
+    tokens = [T, T, T_out, T_out, T_out, T_out, 1, 1]
+    hp = dict(C=0.3, sigma=0.7, lr=1e-2, beta1=0.9, beta2=0.999, xi=1e-11, weight_decay=0.5)
+    step = DPStep(spec_list, DEV, seed=5, shared_tables={4: 0}, **hp)
+    assert step.offsets[4] == step.offsets[0]
+    assert step.n_flat == sum((sp.n_params() + 3) // 4 * 4 if sp.kind != LINEAR or not sp.has_bias else
+                              (sp.d_in * sp.d_out + 3) // 4 * 4 + (sp.d_out + 3) // 4 * 4
+                              for k, sp in enumerate(spec_list) if k != 4)
+    th0 = synth.initial_weights(step.n_flat, 3, DEV)
+    step.theta.copy_(th0)
+    g = torch.Generator().manual_seed(33)
+    mbs = []
+    for mb in range(2):
+        data = []
+        dlogits = (torch.randn(B, T_out, V, generator=g) * 0.05).to(dt).to(DEV)
+        for sp, tk in zip(spec_list, tokens):
+            G = (torch.randn(B, tk, sp.d_out, generator=g) * 0.05).to(dt).to(DEV)
+            if sp.kind == EMBEDDING:
+                data.append(LayerData(sp, G=G, ids=torch.randint(0, V, (B, tk), generator=g, dtype=torch.int32).to(DEV)))
+            elif sp.name == "decoder":
+                data.append(LayerData(sp, G=torch.randn(B, tk, d, generator=g).to(dt).to(DEV), A=dlogits))
+            elif sp.name == "out_bias":
+                data.append(LayerData(sp, G=dlogits, A=torch.ones(B, tk, 1, dtype=dt, device=DEV)))
+            else:
+                data.append(LayerData(sp, G=G, A=torch.randn(B, tk, sp.d_in, generator=g).to(dt).to(DEV)))
+        mbs.append(to_oracle_layers(data))
+        if mb == 0:                                # a clip norm that some examples exceed and some do not
+            step.C = hp["C"] = float(np.sqrt(np.median(O.per_example_sqnorms_shared_table(mbs[0], 0, 4))))
+        lists = step.layer_lists(data)
+        assert [ll.layers[0].G.shape[1] for ll in lists] == [T, T_out, 1]
+        step.accumulate_microbatch(lists)
+    assert b.dp_poll_status() == 0 and step.examples_seen == 2 * B
+    ref = O.zero_accumulators(mbs[0])
+    ref[4][0] = ref[0][0]
+    clipped = 0
+    for ol in mbs:
+        c = O.clip_factors(O.per_example_sqnorms_shared_table(ol, 0, 4), hp["C"])
+        clipped += int((c < 1).sum())
+        O.clipped_accumulate(ol, c, ref)
+    assert 0 < clipped < 2 * B
+    flat = np.zeros(step.n_flat)
+    for li in range(len(spec_list)):
+        for k, a in enumerate(ref[li]):
+            off = step.offsets[li][k]
+            flat[off:off + a.size] = a.ravel()
+    acc = to_np(step.acc)
+    assert rel_l2(acc, flat) <= BF16_TOL
+    step.finish_macro_batch()
+    gref = O.add_noise_and_scale(acc, hp["sigma"], hp["C"], 2 * B, seed=5, step=1, elem_offset=0)
+    rt, rm, rv = O.adamw_step(to_np(th0), np.zeros(step.n_flat), np.zeros(step.n_flat), gref, hp["lr"], hp["beta1"],
+                              hp["beta2"], hp["xi"], hp["weight_decay"], 1)
+    dth, rd = to_np(step.theta) - to_np(th0), rt - to_np(th0)
+    assert np.max(np.abs(dth - rd)) <= 1e-4 * np.max(np.abs(rd)) + 1e-7 * float(th0.abs().max())
