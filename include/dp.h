@@ -242,6 +242,18 @@ DP_API int dp_poll_status(void* cuda_stream);
  * Synchronises the device. */
 DP_API int dp_last_timeout_info(int info[5]);
 
+/* Every device-side wait of the tensor-core kernels (on a TMA copy, a tensor-core commit, another warp) gives up after
+ * a limit, 4e9 SM clock cycles (2 to 3 s) by default; the kernel then records DP_ERR_TIMEOUT, skips the rest of its
+ * work and returns.  This sets the limit for the CURRENT device (cycles <= 0 restores the default); it synchronises
+ * with the device and must not be called while kernels of the library are running.  Meant for tests and for callers
+ * that prefer an earlier error over a longer stall. */
+DP_API int dp_set_wait_limit_cycles(long long cycles);
+
+/* Self-test of that mechanism: enqueues one small kernel whose waiters poll a barrier that nobody arrives on.  They
+ * give up at the limit, the kernel returns, and dp_poll_status then reports DP_ERR_TIMEOUT with
+ * dp_last_timeout_info()[0] = 98 or 99 (the two wait sites of the self-test).  Nothing else is affected. */
+DP_API int dp_selftest_wait_timeout(void* cuda_stream);
+
 /* Number of kernels this library has launched in the calling process so far (host-side counter). */
 DP_API long long dp_launch_count(void);
 

@@ -9,4 +9,4 @@ from .binding import (DP_PATH_AUTO, DP_PATH_GRAM, DP_PATH_MATERIALIZED, DpError,
                       alloc_workspace, dp_adamw_step, dp_add_noise_and_scale, dp_clip_factors, dp_clip_stats, dp_noise_scale_adamw_step_snr,
                       dp_clipped_accumulate, dp_clipped_accumulate_after_sqnorms, dp_noise_scale_adamw_step, dp_reduce_noise_adamw_step, dp_per_example_sqnorms, dp_philox_u32,
                       dp_launch_count, dp_layernorm_sqnorms_static, dp_poll_status, dp_shared_table_cross_sqnorms, dp_token_equality_mask, dp_version, dp_workspace_bytes)
-from .step import DPStep  # noqa: F401
+from .step import DeviceStatusError, DPStep  # noqa: F401

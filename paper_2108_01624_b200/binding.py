@@ -26,6 +26,7 @@ EXPORTS = ["dp_workspace_bytes", "dp_per_example_sqnorms", "dp_clip_factors", "d
            "dp_add_noise_and_scale", "dp_adamw_step", "dp_noise_scale_adamw_step", "dp_noise_scale_adamw_step_snr",
            "dp_clip_stats", "dp_philox_u32", "dp_shared_table_cross_sqnorms",
            "dp_token_equality_mask", "dp_layernorm_sqnorms_static", "dp_poll_status", "dp_last_timeout_info", "dp_launch_count",
+           "dp_set_wait_limit_cycles", "dp_selftest_wait_timeout",
            "dp_status_string", "dp_version"]
 
 
@@ -75,6 +76,8 @@ def lib() -> C.CDLL:
         L.dp_shared_table_cross_sqnorms.argtypes = [vp, vp, i32, i32, vp, vp, i32, i32, i32, i32, vp, vp]
         L.dp_layernorm_sqnorms_static.argtypes = [vp, vp, i32, vp]
         L.dp_poll_status.argtypes = [vp]
+        L.dp_set_wait_limit_cycles.argtypes = [C.c_longlong]
+        L.dp_selftest_wait_timeout.argtypes = [vp]
         L.dp_status_string.restype = C.c_char_p
         L.dp_status_string.argtypes = [i32]
         L.dp_version.restype = i32
@@ -226,6 +229,20 @@ def dp_clipped_accumulate_after_sqnorms(layers: LayerList, clip: torch.Tensor, w
            lib().dp_clipped_accumulate_after_sqnorms(layers.ptr, len(layers), _ptr(clip), ws_p, ws_n, _stream(stream)))
 
 
+def dp_accumulate_schedule(layers: LayerList, units: int, max_launches: int = 16) -> dict:
+    """Host-only view of the accumulate GEMM's work schedule on a device with `units` CTA pairs: per layer the first
+    work item and the launch it belongs to (-1: the layer takes another path), per launch the number of example
+    ranges a tile is split into and the number of item slots."""
+    n = len(layers)
+    start, launch = (C.c_int64 * n)(), (C.c_int32 * n)()
+    splits, slots = (C.c_int32 * max_launches)(), (C.c_int64 * max_launches)()
+    rc = lib().dp_accumulate_schedule(layers.ptr, n, int(units), C.cast(start, C.c_void_p), C.cast(launch, C.c_void_p),
+                                      C.cast(splits, C.c_void_p), C.cast(slots, C.c_void_p), max_launches)
+    if rc < 0:
+        raise DpError("dp_accumulate_schedule", rc)
+    return {"item_start": list(start), "launch": list(launch), "splits": list(splits)[:rc], "slots": list(slots)[:rc]}
+
+
 def dp_add_noise_and_scale(acc: torch.Tensor, sigma: float, C_: float, batch_size: int, seed: int, step: int,
                            elem_offset: int = 0, stream=None) -> torch.Tensor:
     _check("dp_add_noise_and_scale",
@@ -323,3 +340,13 @@ def dp_launch_count() -> int:
 
 def dp_poll_status(stream=None) -> int:
     return int(lib().dp_poll_status(_stream(stream)))
+
+
+def dp_set_wait_limit_cycles(cycles: int) -> None:
+    """Limit of every bounded device-side wait on the current device (<= 0: the default of 4e9 SM cycles)."""
+    _check("dp_set_wait_limit_cycles", lib().dp_set_wait_limit_cycles(int(cycles)))
+
+
+def dp_selftest_wait_timeout(stream=None) -> None:
+    """Enqueues the kernel whose waits nobody satisfies; dp_poll_status reports DP_ERR_TIMEOUT afterwards."""
+    _check("dp_selftest_wait_timeout", lib().dp_selftest_wait_timeout(_stream(stream)))

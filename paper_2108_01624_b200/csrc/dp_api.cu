@@ -454,6 +454,14 @@ int dp_last_timeout_info(int info[5]) {
   return DP_OK;
 }
 
+int dp_set_wait_limit_cycles(long long cycles) { return set_wait_limit_cycles(cycles); }
+
+int dp_selftest_wait_timeout(void* cuda_stream) {
+  int* status = status_ptr();
+  if (!status) return DP_ERR_CUDA;
+  return launch_selftest_wait(status, static_cast<cudaStream_t>(cuda_stream));
+}
+
 const char* dp_status_string(int status) {
   switch (status) {
     case DP_OK: return "ok";

@@ -366,7 +366,8 @@ cudaError_t launch_colsums_batched(const ColTaskHost* tasks, int n, cudaStream_t
           case 2: colsums_b_launch<__nv_bfloat16, 8>(P, wx, s); break;
           default: colsums_b_launch<__nv_bfloat16, 1>(P, wx, s); break;
         }
-        if (counted(1) != cudaSuccess) return cudaGetLastError();
+        const cudaError_t e = counted(1);
+        if (e != cudaSuccess) return e;
         P.n = 0;
       }
     }

@@ -92,4 +92,9 @@ long long umma_accumulate_schedule(const dp_layer* layers, const int* idx, int n
 int launch_umma_accumulate(const dp_layer* layers, const int* idx, int n, const float* clip, int* status,
                            unsigned int* wave_sync, cudaStream_t s);
 
+// Limit of every bounded device-side wait on the current device, in SM cycles (<= 0 restores the default).
+int set_wait_limit_cycles(long long cycles);
+// One CTA that waits, bounded, on a barrier nobody arrives on: records a timeout (site tag 98 or 99) and returns.
+int launch_selftest_wait(int* status, cudaStream_t s);
+
 }  // namespace dpk

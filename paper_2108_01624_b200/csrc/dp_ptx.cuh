@@ -38,8 +38,11 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 }
 
 // Wait limit in SM clock cycles (clock64 is cheap to read; %globaltimer is not and would sit on the critical
-// path of every wait that does not succeed at once): 4e9 cycles = 2 to 3 s at 1.3 to 2 GHz.
-constexpr long long kWaitLimitCycles = 4000000000ll;
+// path of every wait that does not succeed at once): 4e9 cycles = 2 to 3 s at 1.3 to 2 GHz by default.  It is a
+// device variable (read only on the slow path of a wait, once per 64 polls) so that a test can shorten it and
+// watch a wait give up; this header belongs to one translation unit, which owns the variable.
+constexpr long long kDefaultWaitLimitCycles = 4000000000ll;
+static __device__ long long g_wait_limit_cycles = kDefaultWaitLimitCycles;
 constexpr int kStatusTimeout = 1;
 
 // Waits for the phase with the given parity.  Returns false if the limit ran out or another thread
@@ -58,7 +61,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
     if (mbar_try_wait(bar, parity)) return true;
     if ((spin & 63u) == 0u) {
       if (*abort_flag) return false;
-      if (clock64() - t0 > kWaitLimitCycles) {
+      if (clock64() - t0 > g_wait_limit_cycles) {
         if (atomicCAS(status, 0, kStatusTimeout) == 0) {
           status[1] = tag;
           status[2] = (int)blockIdx.x;
@@ -79,7 +82,7 @@ __device__ __forceinline__ bool mbar_wait_drain(uint64_t* bar, uint32_t parity, 
   const long long t0 = clock64();
   for (uint32_t spin = 1;; ++spin) {
     if (mbar_try_wait(bar, parity)) return true;
-    if ((spin & 63u) == 0u && clock64() - t0 > kWaitLimitCycles) {
+    if ((spin & 63u) == 0u && clock64() - t0 > g_wait_limit_cycles) {
       atomicCAS(status, 0, kStatusTimeout);
       return false;
     }

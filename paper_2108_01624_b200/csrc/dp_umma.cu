@@ -893,7 +893,8 @@ k_accum_pair(const __grid_constant__ UmmaParams P) {
       for (int u = 0; u < 8; ++u) col[u] = 0.0f;
       for (int e = t.e0; e < t.e1; ++e) {
         const float cf = alive ? __ldg(P.clip + e) : 1.0f;
-        // c = c_hi + c_lo in bf16: x*c_hi + x*c_lo keeps the factor to ~2^-17 with two packed instructions
+        // c = c_hi + c_lo in bf16: fma(x, c_hi, x*c_lo) keeps the factor to ~2^-17 with two packed instructions; the
+        // small term is the one rounded first, so the only rounding that counts is the final one to bf16 (2^-9)
         const __nv_bfloat16 chi = __float2bfloat16_rn(cf);
         const __nv_bfloat162 chi2 = __halves2bfloat162(chi, chi);
         const __nv_bfloat16 clo = __float2bfloat16_rn(cf - __bfloat162float(chi));
@@ -917,7 +918,7 @@ k_accum_pair(const __grid_constant__ UmmaParams P) {
                   col[2 * u + 1] = fmaf(__uint_as_float(x[u] & 0xffff0000u), cf, col[2 * u + 1]);
                 }
                 const __nv_bfloat162 xv = *reinterpret_cast<const __nv_bfloat162*>(&x[u]);
-                const __nv_bfloat162 yv = __hfma2(xv, clo2, __hmul2(xv, chi2));
+                const __nv_bfloat162 yv = __hfma2(xv, chi2, __hmul2(xv, clo2));
                 x[u] = *reinterpret_cast<const uint32_t*>(&yv);
               }
               if (cf != 1.0f) *p = make_uint4(x[0], x[1], x[2], x[3]);
@@ -1058,21 +1059,33 @@ size_t umma_sqnorm_partials_per_example(const dp_layer* layers, const int* idx, 
   return c;
 }
 
+// Per-device facts, looked up once for each device a process drives (one process may drive several GPUs).
+constexpr int kMaxDevices = 64;
+static int current_device() {
+  int dev = 0;
+  return (cudaGetDevice(&dev) == cudaSuccess && dev >= 0 && dev < kMaxDevices) ? dev : -1;
+}
+
 static int sm_count() {
-  static int sms = 0;
-  if (!sms) {
-    int dev = 0;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    if (sms <= 0) sms = 148;
+  static int sms[kMaxDevices] = {};
+  const int dev = current_device();
+  if (dev < 0) return 148;
+  if (!sms[dev]) {
+    int n = 0;
+    cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+    sms[dev] = n > 0 ? n : 148;
   }
-  return sms;
+  return sms[dev];
 }
 
 template <typename K>
 static bool ensure_smem(K kernel, int bytes) {
   return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) == cudaSuccess;
 }
+
+// The opt-in to more than 48 KB of dynamic shared memory is a per-device attribute of a kernel.
+static bool sqnorm_kernels_ready();
+static bool accum_kernel_ready();
 
 // groups_g / groups_a: 64-feature groups that a box of the G / A map spans.
 // A box may be taller than T or span more groups than the layer has: what lies outside the tensor is zero-filled.
@@ -1094,13 +1107,29 @@ static bool fill_layer(UmmaLayer& U, const dp_layer& L, int box_rows, int groups
   return true;
 }
 
+static bool sqnorm_kernels_ready() {
+  static signed char state[kMaxDevices] = {};     // 0 unknown, 1 ready, -1 failed
+  const int dev = current_device();
+  if (dev < 0) return false;
+  if (!state[dev])
+    state[dev] = (ensure_smem(k_gram_sqnorm, G_SMEM) && ensure_smem(k_gram_sqnorm_wide, W_SMEM) &&
+                  ensure_smem(k_tile_sqnorm_pair, Q_SMEM)) ? 1 : -1;
+  return state[dev] > 0;
+}
+
+static bool accum_kernel_ready() {
+  static signed char state[kMaxDevices] = {};
+  const int dev = current_device();
+  if (dev < 0) return false;
+  if (!state[dev]) state[dev] = ensure_smem(k_accum_pair, P_SMEM) ? 1 : -1;
+  return state[dev] > 0;
+}
+
 int launch_umma_sqnorms(const dp_layer* layers, const int* idx, int n, const int* use_gram, float* partial,
                         int partial_stride, int partial_base, int* status, cudaStream_t s) {
   if (n <= 0) return DP_OK;
   const int B = layers[idx[0]].B, T = layers[idx[0]].T;
-  static bool attr_ok = ensure_smem(k_gram_sqnorm, G_SMEM) &&
-                        ensure_smem(k_gram_sqnorm_wide, W_SMEM) && ensure_smem(k_tile_sqnorm_pair, Q_SMEM);
-  if (!attr_ok) return DP_ERR_CUDA;
+  if (!sqnorm_kernels_ready()) return DP_ERR_CUDA;
   // Partial slots are assigned in the caller's layer order, whichever kernel fills them.
   std::vector<int> base(n);
   int pos = partial_base;
@@ -1268,8 +1297,7 @@ int launch_umma_accumulate(const dp_layer* layers, const int* idx, int n, const 
                            unsigned int* wave_sync, cudaStream_t s) {
   if (n <= 0) return DP_OK;
   const int B = layers[idx[0]].B, T = layers[idx[0]].T;
-  static bool attr_ok = ensure_smem(k_accum_pair, P_SMEM);
-  if (!attr_ok) return DP_ERR_CUDA;
+  if (!accum_kernel_ready()) return DP_ERR_CUDA;
   const int bk = P_BK;
   const int units = sm_count() / 2;      // CTA pairs that work on tiles side by side
   for (int k0 = 0; k0 < n; k0 += kMaxLayers) {
@@ -1309,6 +1337,37 @@ int launch_umma_accumulate(const dp_layer* layers, const int* idx, int n, const 
     if (counted(1) != cudaSuccess) return DP_ERR_CUDA;
   }
   return DP_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Wait limit and its self-test
+// ---------------------------------------------------------------------------------------------
+int set_wait_limit_cycles(long long cycles) {
+  if (cycles <= 0) cycles = kDefaultWaitLimitCycles;
+  return cudaMemcpyToSymbol(g_wait_limit_cycles, &cycles, sizeof(cycles)) == cudaSuccess ? DP_OK : DP_ERR_CUDA;
+}
+
+// One CTA whose two waiters poll a barrier that nobody ever arrives on, through the same bounded wait as the
+// pipelines: the first to run out records the timeout and raises the CTA's abort flag, the other leaves by its own
+// limit or by the flag, and the kernel returns.
+__global__ void __launch_bounds__(64) k_selftest_wait(int* status) {
+  __shared__ uint64_t bar;
+  __shared__ int abort_word;
+  volatile int* abort_flag = &abort_word;
+  if (threadIdx.x == 0) {
+    mbar_init(&bar, 1);
+    abort_word = 0;
+    fence_mbar_init();
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) mbar_wait(&bar, 0u, abort_flag, status, 99, 7);
+  if (threadIdx.x == 32) mbar_wait<64>(&bar, 0u, abort_flag, status, 98, 8);
+  __syncthreads();
+}
+
+int launch_selftest_wait(int* status, cudaStream_t s) {
+  k_selftest_wait<<<1, 64, 0, s>>>(status);
+  return counted(1) == cudaSuccess ? DP_OK : DP_ERR_CUDA;
 }
 
 }  // namespace dpk

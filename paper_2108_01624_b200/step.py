@@ -14,6 +14,19 @@ from . import binding as b
 from .synth import EMBEDDING, LAYERNORM, LINEAR, LayerData, LayerSpec
 
 
+class DeviceStatusError(RuntimeError):
+    """The library's device-side status word was not clean when a macro-batch was about to be applied."""
+
+    def __init__(self, code: int):
+        self.code = int(code)
+        try:
+            what = b.status_string(self.code)
+        except Exception:          # the library itself is missing
+            what = "?"
+        super().__init__(f"device status {self.code} ({what}): the macro-batch was discarded, "
+                         "parameters and optimizer state are unchanged")
+
+
 class DPStep:
     """Owns the flat fp32 state (theta, m, v, accumulator) for a list of layer specs.
 
@@ -24,8 +37,13 @@ class DPStep:
 
     def __init__(self, specs: Sequence[LayerSpec], device, C: float, sigma: float, lr: float, beta1: float,
                  beta2: float, xi: float, weight_decay: float, seed: int = 0, theta: Optional[torch.Tensor] = None,
-                 track_snr: bool = False, shared_tables: Optional[dict] = None):
-        """shared_tables maps the index of an output-projection spec (a bias-free LINEAR layer with d_in = V whose
+                 track_snr: bool = False, shared_tables: Optional[dict] = None, shard_world: int = 1):
+        """shard_world: number of data-parallel ranks the macro-batch will be finished across (parallel.ShardedUpdate).
+        The accumulator and theta are then allocated with room for `shard_world` equal shards (acc_store,
+        theta_store; acc and theta are their first n_flat elements), so that the reduce-scatter and the all-gather
+        of a macro-batch's end run in place.
+
+        shared_tables maps the index of an output-projection spec (a bias-free LINEAR layer with d_in = V whose
         A is dlogits and whose G is the projection's input) to the index of the EMBEDDING spec whose [V, d] table it
         also trains (BERT's masked-LM decoder): the projection gets no storage of its own, both layers accumulate into
         the table, and the per-example norm includes the inner product of their two contributions."""
@@ -64,10 +82,14 @@ class DPStep:
             self.offsets.append(offs)
             self.shapes.append(shp)
         self.n_flat = pos
-        self.acc = torch.zeros(pos, dtype=torch.float32, device=self.device)
-        self.m = torch.zeros_like(self.acc)
-        self.v = torch.zeros_like(self.acc)
-        self.theta = torch.zeros_like(self.acc) if theta is None else theta
+        from .parallel import padded_length
+        cap = padded_length(pos, shard_world)
+        self.acc_store = torch.zeros(cap, dtype=torch.float32, device=self.device)
+        self.acc = self.acc_store[:pos]
+        self.m = torch.zeros(pos, dtype=torch.float32, device=self.device)
+        self.v = torch.zeros_like(self.m)
+        self.theta_store = torch.zeros_like(self.acc_store) if theta is None else None
+        self.theta = self.theta_store[:pos] if theta is None else theta
         self.t = 0
         self.examples_seen = 0
         # gradient-SNR of Section 5.2.1: (sum acc^2, sum noise^2) of the last macro-batch, filled by the fused pass
@@ -137,8 +159,29 @@ class DPStep:
         self.examples_seen += B
         return self._sqnorm, self._clip
 
-    def finish_macro_batch(self, batch_size: Optional[int] = None, fused: bool = True, stream=None):
-        """Noise, division by the macro-batch size and the AdamW update; clears the accumulator."""
+    def discard_macro_batch(self) -> None:
+        """Drops the partly accumulated macro-batch: the accumulator is cleared, theta, m, v and t stay as they are."""
+        self.acc.zero_()
+        self.examples_seen = 0
+
+    def check_device_status(self, stream=None) -> None:
+        """Waits for the stream and reads the library's sticky status word.  A bounded wait that ran out or a token
+        id out of range makes the kernels skip the offending work, so a squared norm may be wrong and the factor
+        min(1, C/||g_i||) would no longer bound that example's contribution by C -- the sensitivity that the noise of
+        Algorithm 1 is calibrated to.  In that case the macro-batch is discarded and DeviceStatusError raised."""
+        code = b.dp_poll_status(stream)
+        if code != b.DP_OK:
+            self.discard_macro_batch()
+            raise DeviceStatusError(code)
+
+    def finish_macro_batch(self, batch_size: Optional[int] = None, fused: bool = True, stream=None,
+                           check_status: bool = True):
+        """Noise, division by the macro-batch size and the AdamW update; clears the accumulator.
+        With check_status (one host synchronisation per macro-batch) a device-side error reported since the last
+        poll raises DeviceStatusError BEFORE anything is applied: theta, m, v and t are untouched and the
+        accumulator is cleared."""
+        if check_status:
+            self.check_device_status(stream)
         N = self.examples_seen if batch_size is None else batch_size
         self.t += 1
         if fused and self.sq_sums is not None:

@@ -45,7 +45,7 @@ def _worker(rank, world, port, n, out_dir):
     g = torch.Generator().manual_seed(100 + rank)
     local_acc = torch.randn(n, generator=g, dtype=torch.float64)
     st = _State(n, local_acc)
-    sh = ShardedUpdate(st, dist, world, rank, update_fn=_oracle_update(st))
+    sh = ShardedUpdate(st, dist, world, rank, update_fn=_oracle_update(st), poll_fn=lambda: 0)
     for step in range(2):
         st.acc.copy_(local_acc * (step + 1))
         st.examples_seen = 64 * world
@@ -130,7 +130,8 @@ def _fused_worker(rank, world, port, n, accs, thetas, out_dir):
     st = _State(n, local_acc)
     st.acc, st.theta = accs[rank], thetas[rank]          # this rank's buffers are the shared ones
     st.theta.copy_(torch.linspace(-1, 1, n, dtype=torch.float64))
-    sh = ShardedUpdate(st, dist, world, rank, peer_acc=accs, peer_theta=thetas, fused_fn=_oracle_fused(st))
+    sh = ShardedUpdate(st, dist, world, rank, peer_acc=accs, peer_theta=thetas, fused_fn=_oracle_fused(st),
+                       poll_fn=lambda: 0)
     for step in range(2):
         st.acc.copy_(local_acc * (step + 1))
         st.examples_seen = 64 * world
@@ -164,3 +165,101 @@ def test_peer_buffers_given_as_addresses():
     assert ShardedUpdate._shard_of(4096, 8, 16) == 4096 + 32
     t = torch.arange(20.0)
     assert torch.equal(ShardedUpdate._shard_of(t, 8, 16), t[8:16])
+
+
+def _rendezvous_worker(rank, world, port, n, out_dir):
+    """Every rank allocates its own accumulator and replica, the ranks exchange handles over the process group
+    (exchange_peer_buffers) and finish two macro-batches with the one-kernel way over the mapped buffers."""
+    sys.path.insert(0, ROOT)
+    import torch.distributed as dist
+    from paper_2108_01624_b200.parallel import ShardedUpdate, exchange_peer_buffers
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    g = torch.Generator().manual_seed(100 + rank)
+    local_acc = torch.randn(n, generator=g, dtype=torch.float64)
+    st = _State(n, local_acc)
+    accs = exchange_peer_buffers(st.acc, dist, world, rank)
+    thetas = exchange_peer_buffers(st.theta, dist, world, rank)
+    assert accs[rank] is st.acc and thetas[rank] is st.theta
+    # a write through the mapping is seen by the owner
+    dist.barrier()
+    if rank == 0:
+        accs[world - 1][n - 1] = 12345.0
+    dist.barrier()
+    if rank == world - 1:
+        assert float(st.acc[n - 1]) == 12345.0
+    dist.barrier()
+    sh = ShardedUpdate(st, dist, world, rank, peer_acc=accs, peer_theta=thetas, fused_fn=_oracle_fused(st),
+                       poll_fn=lambda: 0)
+    for step in range(2):
+        st.acc.copy_(local_acc * (step + 1))
+        st.examples_seen = 64 * world
+        sh.finish_macro_batch()
+    torch.save({"theta": st.theta.clone(), "acc": st.acc.clone(), "lo": sh.lo, "hi": sh.hi, "m": st.m},
+               f"{out_dir}/x{rank}.pt")
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+@pytest.mark.parametrize("world,n", [(2, 1003), (3, 257)])
+def test_handle_exchange_then_fused_update(world, n, tmp_path):
+    mp.spawn(_rendezvous_worker, args=(world, _free_port(), n, str(tmp_path)), nprocs=world, join=True)
+    outs = [torch.load(f"{tmp_path}/x{r}.pt") for r in range(world)]
+    src = [torch.randn(n, generator=torch.Generator().manual_seed(100 + r), dtype=torch.float64) for r in range(world)]
+    st = _State(n, sum(src))
+    fn = _oracle_update(st)
+    for step in range(2):
+        st.t += 1
+        fn(st.theta, st.m, st.v, (sum(src) * (step + 1)).clone(), 0, 64 * world, st.t)
+    for o in outs:
+        np.testing.assert_allclose(o["theta"].numpy(), st.theta.numpy(), rtol=1e-12, atol=1e-14)
+        assert float(o["acc"].abs().max()) == 0.0
+
+
+def _status_worker(rank, world, port, n, bad_rank, out_dir):
+    sys.path.insert(0, ROOT)
+    import torch.distributed as dist
+    from paper_2108_01624_b200.parallel import ShardedUpdate
+    from paper_2108_01624_b200.step import DeviceStatusError
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    st = _State(n, torch.ones(n, dtype=torch.float64))
+    calls = []
+    codes = iter([-5 if rank == bad_rank else 0, 0])      # first macro-batch: one rank reports a timeout
+
+    def update(theta, m, v, acc, elem_offset, batch_size, t):
+        calls.append(t)
+        acc.zero_()
+    sh = ShardedUpdate(st, dist, world, rank, update_fn=update, poll_fn=lambda: next(codes))
+    theta0 = st.theta.clone()
+    st.examples_seen = 8
+    raised = None
+    try:
+        sh.finish_macro_batch()
+    except DeviceStatusError as e:
+        raised = e.code
+    ok_first = (raised == -5 and not calls and st.t == 0 and st.examples_seen == 0
+                and float(st.acc.abs().max()) == 0.0 and torch.equal(st.theta, theta0))
+    st.acc.fill_(1.0)
+    st.examples_seen = 8
+    sh.finish_macro_batch()                               # the next macro-batch goes through on every rank
+    ok_second = calls == [1] and st.t == 1
+    torch.save({"ok_first": ok_first, "ok_second": ok_second}, f"{out_dir}/s{rank}.pt")
+    dist.destroy_process_group()
+
+
+def test_device_error_on_one_rank_discards_the_macro_batch_on_all(tmp_path):
+    world = 2
+    mp.spawn(_status_worker, args=(world, _free_port(), 40, 1, str(tmp_path)), nprocs=world, join=True)
+    for r in range(world):
+        o = torch.load(f"{tmp_path}/s{r}.pt")
+        assert o["ok_first"] and o["ok_second"], (r, o)
+
+
+def test_padded_storage_is_reused_or_made():
+    from paper_2108_01624_b200.parallel import padded_length, shard_length
+    assert padded_length(1003, 1) == 1003
+    assert padded_length(1003, 2) == 2 * shard_length(1003, 2) == 1008
+    assert padded_length(333_563_904, 8) == 333_563_904

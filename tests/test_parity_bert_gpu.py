@@ -24,29 +24,62 @@ def _subset(data, rows):
                             ids=None if ld.ids is None else ld.ids[rows].contiguous()) for ld in data]
 
 
-def _sampled_entries_check(data, accs, clip, n_samples, seed):
-    """acc_w[p,q] = sum_r clip[r/T] A[r,p] G[r,q] recomputed in fp64 on the host for random (p,q)."""
+ENTRY_TOL = 0.01      # of the root-sum-square of an entry's terms; see _tile_sampled_check
+
+
+def _tile_sampled_check(data, accs, clips, seed, counts=None, bias_layers=3):
+    """The clipped sum at the full launch size, one sampled entry for EVERY 128 x 128 block of every linear layer's
+    accumulator (eight per 256 x 512 tile of the accumulate GEMM: each CTA of a pair, each half of its accumulator,
+    each 128-column group), recomputed in fp64 on the host from columns gathered on the device:
+        acc_w[p, q] = sum over the microbatches of  sum_r clip[r / T] A[r, p] G[r, q].
+    `data`, `clips`: one entry per distinct microbatch, `counts[k]` = how often microbatch k was accumulated.
+    Bound per entry: 1 % of the root-sum-square of its terms.  The bf16 rounding of clip * G (relative 2^-9 per term,
+    independent) puts the error near 0.1 % of that scale; a dropped or unscaled 64-token stage is 1 / 512 of the
+    terms, about 4 % of it, and a dropped tile or a misplaced block is of order 100 %.
+    Every bias element of `bias_layers` layers is checked the same way."""
     rng = np.random.default_rng(seed)
-    c = to_np(clip)
-    for ld, acc in zip(data, accs):
-        if ld.spec.kind != LINEAR:
-            continue
-        B, T, _ = ld.G.shape
-        w = np.repeat(c, T)
-        errs, mags = [], []
-        for _ in range(n_samples):
-            p, q = int(rng.integers(ld.spec.d_in)), int(rng.integers(ld.spec.d_out))
-            a = to_np(ld.A[:, :, p]).reshape(-1)
-            g = to_np(ld.G[:, :, q]).reshape(-1)
-            ref = float(np.sum(w * a * g))
-            errs.append(abs(float(acc[0][p, q]) - ref))
-            mags.append(abs(ref))
-        scale = float(np.sqrt(np.mean(np.square(mags)))) + 1e-30
-        assert max(errs) <= BF16_TOL * scale, f"{ld.spec.name}: {max(errs):.3e} vs rms {scale:.3e}"
-        if ld.spec.has_bias:
-            q = int(rng.integers(ld.spec.d_out))
-            ref = float(np.sum(w * to_np(ld.G[:, :, q]).reshape(-1)))
-            assert abs(float(acc[1][q]) - ref) <= BF16_TOL * (abs(ref) + scale)
+    counts = [1] * len(data) if counts is None else counts
+    lin = [k for k, ld in enumerate(data[0]) if ld.spec.kind == LINEAR]
+    n_entries = 0
+    for k in lin:
+        sp = data[0][k].spec
+        nb_in, nb_out = (sp.d_in + 127) // 128, (sp.d_out + 127) // 128
+        ps = np.array([min(sp.d_in - 1, bi * 128 + int(rng.integers(128))) for bi in range(nb_in) for _ in range(nb_out)])
+        qs = np.array([min(sp.d_out - 1, bo * 128 + int(rng.integers(128))) for _ in range(nb_in) for bo in range(nb_out)])
+        ref = np.zeros(len(ps))
+        sq = np.zeros(len(ps))
+        for mb, clip, cnt in zip(data, clips, counts):
+            ld = mb[k]
+            B, T, _ = ld.G.shape
+            w = np.repeat(to_np(clip), T)
+            a = to_np(ld.A.reshape(B * T, -1)[:, torch.from_numpy(ps).to(ld.A.device)])       # [B T, n]
+            g = to_np(ld.G.reshape(B * T, -1)[:, torch.from_numpy(qs).to(ld.G.device)])
+            terms = a * g * w[:, None]
+            ref += cnt * terms.sum(0)
+            sq += cnt * cnt * (terms ** 2).sum(0)
+        got = to_np(accs[k][0][torch.from_numpy(ps).to(DEV), torch.from_numpy(qs).to(DEV)])
+        err = np.abs(got - ref)
+        bound = ENTRY_TOL * np.sqrt(sq) + 1e-30
+        worst = int(np.argmax(err / bound))
+        assert np.all(err <= bound), (f"{sp.name}: entry ({ps[worst]}, {qs[worst]}) off by {err[worst]:.3e}, "
+                                      f"bound {bound[worst]:.3e}")
+        n_entries += len(ps)
+    with_bias = [k for k in lin if data[0][k].spec.has_bias]
+    for k in rng.choice(with_bias, size=min(bias_layers, len(with_bias)), replace=False):
+        k = int(k)
+        ref = np.zeros(data[0][k].spec.d_out)
+        sq = np.zeros_like(ref)
+        for mb, clip, cnt in zip(data, clips, counts):
+            G = to_np(mb[k].G) * to_np(clip)[:, None, None]
+            ref += cnt * G.sum((0, 1))
+            sq += cnt * cnt * (G ** 2).sum((0, 1))
+        err = np.abs(to_np(accs[k][1]) - ref)
+        assert np.all(err <= 1e-3 * np.sqrt(sq) + 1e-30), data[0][k].spec.name      # fp32 sums of exact products
+    return n_entries
+
+
+def _sampled_entries_check(data, accs, clip, seed):
+    return _tile_sampled_check([data], accs, [clip], seed)
 
 
 def _full_size_ln_and_embedding_check(data, accs, clip, n_ln, seed):
@@ -126,7 +159,8 @@ def test_bert_large_stack_subset_and_samples(n_layers):
     np.testing.assert_allclose(to_np(n[rows]), n_ref, rtol=2 * CLIP_TOL)
     np.testing.assert_allclose(to_np(c[rows]), c_ref, rtol=CLIP_TOL)
     # (b) full launch size: sampled accumulator entries in fp64
-    _sampled_entries_check(data, accs, c, n_samples=6, seed=1)
+    n_entries = _sampled_entries_check(data, accs, c, seed=1)
+    assert n_entries == 24 * (8 * 24 + 8 * 8 + 8 * 32 + 32 * 8)       # every 128 x 128 block of all 96 linear layers
     _full_size_ln_and_embedding_check(data, accs, c, n_ln=3, seed=2)
     # (b') all 256 norms of the linear layers: the Gram kernel against the materialised-tile kernel, two different
     # algorithms for the same quantity (the identity of Section 4.3 holds at any size)
@@ -180,7 +214,7 @@ def test_long_sequence_crossover_all_paths():
     ll, accs = make_layer_list(data, DEV)
     n, c, ws = gpu_norms_clip(ll, wl.C)
     b.dp_clipped_accumulate(ll, c, ws)
-    _sampled_entries_check(data, accs, c, n_samples=6, seed=2)
+    _sampled_entries_check(data, accs, c, seed=2)
 
 
 def test_mega_batch_accumulation_invariants():
@@ -223,3 +257,58 @@ def test_mega_batch_accumulation_invariants():
     assert rel_l2(to_np(many.m), rm) <= 1e-5 and rel_l2(to_np(many.v), rv) <= 1e-5
     d, rd = to_np(many.theta) - to_np(th0), rt - to_np(th0)
     assert np.max(np.abs(d - rd)) <= 1e-4 * np.max(np.abs(rd)) + 1e-7 * float(th0.abs().max())
+
+
+def test_mega_batch_at_bert_large_shapes():
+    """The mega-batch accumulation of Section 5.3 at the full 24-block shapes: two DISTINCT microbatches of 256
+    examples clipped and summed in place (norms and clip factors of a spread subset against the checker, one sampled
+    entry per 128 x 128 accumulator block against fp64), then one microbatch accumulated M = 16 times against 16 times
+    the single pass, the bound ||acc|| <= N C, and the macro-batch's noise + AdamW update on sampled windows."""
+    wl = synth.workload("bert_large")
+    step = DPStep(wl.specs, DEV, wl.C, wl.sigma, wl.lr, wl.beta1, wl.beta2, wl.xi, wl.weight_decay, seed=5)
+    pool = [synth.generate(wl, seed=11, device=DEV, microbatch=k) for k in range(2)]
+    lists = [step.layer_list(d) for d in pool]
+    clips = []
+    rows = [0, 77, 128, 255]
+    for d, ll in zip(pool, lists):
+        sq, clip = step.accumulate_microbatch(ll)
+        clips.append(clip.clone())
+        ol = to_oracle_layers(_subset(d, rows))
+        n_ref = O.per_example_sqnorms(ol)
+        np.testing.assert_allclose(to_np(sq[rows]), n_ref, rtol=2 * CLIP_TOL)
+        np.testing.assert_allclose(to_np(clip[rows]), O.clip_factors(n_ref, wl.C), rtol=CLIP_TOL)
+    torch.cuda.synchronize()
+    assert b.dp_poll_status() == 0 and step.examples_seen == 2 * wl.B
+    assert not torch.equal(clips[0], clips[1])                       # the microbatches are distinct
+    accs = [[step.view(step.acc, li, k) for k in range(len(step.shapes[li]))] for li in range(len(wl.specs))]
+    _tile_sampled_check(pool, accs, clips, seed=3)
+    two = step.acc.clone()
+    assert float(two.double().norm()) <= 2 * wl.B * wl.C * (1 + 1e-3)
+    # the same microbatch M times: M x the single pass (equal addends round the same way every time)
+    step.discard_macro_batch()
+    step.accumulate_microbatch(lists[0])
+    single = step.acc.clone()
+    M = 16
+    for _ in range(M - 1):
+        step.accumulate_microbatch(lists[0])
+    torch.cuda.synchronize()
+    assert b.dp_poll_status() == 0 and step.examples_seen == M * wl.B
+    diff = float((step.acc.double() - M * single.double()).norm() / (M * single.double().norm()))
+    assert diff <= 1e-5, diff
+    assert float(step.acc.double().norm()) <= M * wl.B * wl.C * (1 + 1e-3)
+    # once per macro-batch: noise + AdamW over all 333.6M parameters, the checker on windows of the flat vector
+    del two, single
+    th0 = synth.initial_weights(step.n_flat, 0, DEV)
+    step.theta.copy_(th0)
+    acc_before = step.acc.clone()
+    step.finish_macro_batch()
+    assert step.t == 1 and float(step.acc.abs().max()) == 0.0
+    n = step.n_flat
+    for lo in (0, 4 * 1_000_003, n // 2 - 12, n - 50_000):
+        hi = min(n, lo + 50_000)
+        g = O.add_noise_and_scale(to_np(acc_before[lo:hi]), wl.sigma, wl.C, M * wl.B, seed=5, step=1, elem_offset=lo)
+        z = np.zeros(hi - lo)
+        rt, rm, rv = O.adamw_step(to_np(th0[lo:hi]), z, z, g, wl.lr, wl.beta1, wl.beta2, wl.xi, wl.weight_decay, 1)
+        assert rel_l2(to_np(step.m[lo:hi]), rm) <= 1e-5 and rel_l2(to_np(step.v[lo:hi]), rv) <= 1e-5
+        d, rd = to_np(step.theta[lo:hi]) - to_np(th0[lo:hi]), rt - to_np(th0[lo:hi])
+        assert np.max(np.abs(d - rd)) <= 1e-4 * np.max(np.abs(rd)) + 1e-7 * float(th0[lo:hi].abs().max())

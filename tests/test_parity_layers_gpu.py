@@ -37,6 +37,9 @@ def check_against_checker(data, C, paths=None, sum_tol=BF16_TOL, rows=None):
             assert x.shape == y.shape
             err = rel_l2(to_np(x), y)
             assert err <= sum_tol, f"{ld.spec.name or ld.spec.kind}[{k}] rel L2 {err:.3e}"
+            if ld.G.dtype == torch.float32:      # fp32 paths: every element within 1e-4 of the tensor's largest
+                emax = rel_max(to_np(x), y)
+                assert emax <= F32_TOL, f"{ld.spec.name or ld.spec.kind}[{k}] max error {emax:.3e} of the largest entry"
     return n_ref, c_ref, accs
 
 
@@ -301,6 +304,72 @@ def test_embedding_mask_gram_equals_grouped_rows():
         np.testing.assert_allclose(got[b.DP_PATH_GRAM], got[b.DP_PATH_MATERIALIZED], rtol=1e-4)
     assert b.dp_poll_status() == 0
     assert len(b.dp_last_timeout_info()) == 5
+
+
+def test_embedding_mask_counts_equal_pairs_exactly():
+    """G of all ones makes every entry of G G^T equal d, so the embedding norm is d times the NUMBER of token pairs
+    with equal ids: an integer that fp32 holds exactly.  The id compares inside the norm kernels (the mask applied
+    to the Gram in the tensor-core kernel's epilogue, and the grouping of equal ids in the CUDA-core kernel) must
+    reproduce it bit for bit."""
+    for B, T, d, V, dup in ((6, 128, 128, 40, 9), (3, 200, 64, 500, 30), (4, 33, 192, 11, 11), (2, 300, 128, 7, 3)):
+        spec = [LayerSpec(EMBEDDING, V, d, False, "emb")]
+        data = random_layers(spec, B, T, torch.bfloat16, DEV, seed=T + d, g_scale=1.0, vocab_dup=dup)
+        data[0].G.fill_(1.0)
+        ids = data[0].ids.cpu().numpy()
+        pairs = np.array([int((row[:, None] == row[None, :]).sum()) for row in ids], dtype=np.int64)
+        assert pairs.max() * d < 2 ** 24
+        for path in (b.DP_PATH_GRAM, b.DP_PATH_MATERIALIZED):
+            ll, _ = make_layer_list(data, DEV, [path])
+            n, _, _ = gpu_norms_clip(ll, 1.0)
+            got = n.cpu().numpy().astype(np.float64)
+            assert np.array_equal(got, (pairs * d).astype(np.float64)), (path, T, got, pairs * d)
+        # the checker agrees with the count as well
+        np.testing.assert_array_equal(O.per_example_sqnorms(to_oracle_layers(data)), (pairs * d).astype(np.float64))
+    assert b.dp_poll_status() == 0
+
+
+def test_unsplit_accumulate_is_bitwise_repeatable():
+    """With no example split every accumulator element has one owner and a fixed summation order, so repeated runs
+    with clip factors other than 1 (every stage of G rescaled in shared memory before the tensor cores read it)
+    must agree bit for bit; a stage consumed before its scaling was visible would show up as a difference."""
+    specs = []
+    for blk in range(2):
+        specs += [LayerSpec(LINEAR, 1024, 3072, True, f"qkv{blk}"), LayerSpec(LINEAR, 1024, 1024, True, f"o{blk}"),
+                  LayerSpec(LINEAR, 1024, 4096, True, f"f1{blk}"), LayerSpec(LINEAR, 4096, 1024, True, f"f2{blk}")]
+    B, T = 24, 128
+    data = random_layers(specs, B, T, torch.bfloat16, DEV, seed=91, g_scale=0.02)
+    ll, accs = make_layer_list(data, DEV)
+    units = torch.cuda.get_device_properties(0).multi_processor_count // 2
+    sched = b.dp_accumulate_schedule(ll, units)
+    assert sched["splits"] == [1], sched                 # the case this test is about
+    g = torch.Generator().manual_seed(4)
+    clip = (0.05 + 0.9 * torch.rand(B, generator=g)).to(DEV)
+    ws = b.alloc_workspace(ll)
+    first = None
+    for rep in range(6):
+        for acc in accs:
+            for x in acc:
+                x.zero_()
+        b.dp_clipped_accumulate(ll, clip, ws)
+        torch.cuda.synchronize()
+        snap = [[x.clone() for x in acc] for acc in accs]
+        if first is None:
+            first = snap
+        else:
+            for sp, a0, a1 in zip(specs, first, snap):
+                for x, y in zip(a0, a1):
+                    assert torch.equal(x, y), f"{sp.name}: run {rep} differs from run 0"
+    assert b.dp_poll_status() == 0
+    # and the result is the checker's on a few sampled entries per layer (fp64 on the host)
+    c = to_np(clip)
+    w = np.repeat(c, T)
+    rng = np.random.default_rng(0)
+    for ld, acc in zip(data, first):
+        for _ in range(4):
+            p, q = int(rng.integers(ld.spec.d_in)), int(rng.integers(ld.spec.d_out))
+            ref = float(np.sum(w * to_np(ld.A[:, :, p]).reshape(-1) * to_np(ld.G[:, :, q]).reshape(-1)))
+            scale = float(np.sqrt(np.sum((w * to_np(ld.A[:, :, p]).reshape(-1) * to_np(ld.G[:, :, q]).reshape(-1)) ** 2)))
+            assert abs(float(acc[0][p, q]) - ref) <= 0.01 * scale + 1e-12
 
 
 def test_workspace_too_small_is_refused():

@@ -2,12 +2,12 @@
 (their framework or server owns the device's memory, or cudaMalloc's synchronisation is not acceptable where
 they run).  Its scratch is a fixed array inside the library, so the test calls it through the C ABI twice in a
 row -- the second call meets the first call's leftovers in that array -- and compares each result with the
-workspace-based dp_per_example_sqnorms on the same layer.  Collected last on purpose."""
+workspace-based dp_per_example_sqnorms on the same layer and with the CPU checker.  Collected last on purpose."""
 import numpy as np
 import pytest
 import torch
 
-from .helpers import LAYERNORM, LayerSpec, b, make_layer_list, random_layers, to_np
+from .helpers import LAYERNORM, LayerSpec, O, b, make_layer_list, random_layers, to_np, to_oracle_layers
 
 pytestmark = pytest.mark.gpu
 
@@ -33,6 +33,8 @@ def test_static_scratch_matches_workspace_path_twice_in_a_row(dtype):
         got = torch.full((B,), float("nan"), dtype=torch.float32, device=DEV)
         b.dp_layernorm_sqnorms_static(ll, got, False)
         np.testing.assert_allclose(to_np(got), ref, rtol=2e-3)
+        # and against the CPU checker directly, not only against the library's other path
+        np.testing.assert_allclose(to_np(got), O.per_example_sqnorms(to_oracle_layers(data)), rtol=2e-3)
         # accumulate_into adds to what is there
         b.dp_layernorm_sqnorms_static(ll, got, True)
         np.testing.assert_allclose(to_np(got), 2 * ref, rtol=2e-3)
