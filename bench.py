@@ -31,10 +31,13 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
-# DRAM bytes (read + write) of one k_accum_pair launch over the 24-block stack: the two dram__bytes counters are a
-# single-pass ncu capture, taken on the full workload (profiles/k_accum_pair_2blocks_full.md gives the command).
-# Set to None whenever that kernel changes.
-ACCUM_TRAFFIC_BYTES = 31.35e9
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of one k_accum_pair launch over TWO encoder blocks
+# (`--blocks 2`, 2.7 GB on the device), from the ncu capture summarised in profiles/k_accum_pair_2blocks_full.md.
+# The kernel's traffic grows with the number of blocks (every block's operands are read once, its accumulators read
+# and written once), so a launch over n blocks is reported as this figure x n / 2.  Not to be re-taken on the full
+# 32 GB workload.  Set to None whenever that kernel changes until the capture has been repeated.
+ACCUM_TRAFFIC_2BLOCKS_BYTES = None
+HBM_NOMINAL_GBS = 8000.0          # the figure the target quotes; fractions are reported against it and the measured copy
 
 METRIC = "dp_sgd_examples_per_s_bert_large"
 UNIT = "examples/s"
@@ -93,7 +96,7 @@ class ClockSampler:
             self.proc.wait(timeout=5)
         except Exception:
             self.proc.kill()
-        sm, mx, reasons = [], [], set()
+        sm, mx, pw, reasons = [], [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for r in self.rows:
             f = [x.strip() for x in r.split(",")]
@@ -102,13 +105,21 @@ class ClockSampler:
             try:
                 sm.append(float(f[0]))
                 mx.append(float(f[1]))
+                pw.append(float(f[2]))
             except ValueError:
                 continue
             for name, val in zip(names, f[4:8]):
                 if val.lower().startswith("active"):
                     reasons.add(name)
         return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "reasons": sorted(reasons), "samples": len(sm)}
+                "reasons": sorted(reasons), "samples": len(sm), "power_w": float(np.mean(pw)) if pw else None}
+
+
+def config_dict(wl, n_params, n_gpus, blocks=24):
+    """The workload description, identical in both arms."""
+    return {"workload": WORKLOAD if blocks == 24 else f"{WORKLOAD}[first {blocks} blocks only]",
+            "B": wl.B, "T": wl.T, "layers": len(wl.specs), "params": n_params, "microbatches_per_step": 1,
+            "parallelism": f"dp{n_gpus}", "l2": "inputs (32 GB per microbatch) far exceed L2; no flush"}
 
 
 def oracle_layers(data, rows):
@@ -135,9 +146,16 @@ def oracle_threads() -> int:
         return cores
 
 
-def time_oracle(wl, data, n_params, budget_s=15.0, max_examples=8):
+def time_oracle(wl, data, n_params, budget_s=15.0, max_examples=8, threads=None):
     """The CPU checker as it stands on a bounded sample: k examples through every layer (norms, clip,
-    accumulate) plus noise + AdamW on 1/64 of the parameters; scaled linearly to one 256-example step."""
+    accumulate) plus noise + AdamW on 1/64 of the parameters; scaled linearly to one 256-example step.
+    threads: cap on numpy's BLAS pool for this measurement (None: as the process found it)."""
+    if threads is not None:
+        from threadpoolctl import threadpool_limits
+        with threadpool_limits(limits=threads, user_api="blas"):
+            out = time_oracle(wl, data, n_params, budget_s, max_examples)
+        out["cores"] = threads
+        return out
     from oracle import dp_oracle as O
     t0 = time.perf_counter()
     k = 0
@@ -191,7 +209,7 @@ def run_reference(args):
     line = {"impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * wl.B / v, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": WORKLOAD, "B": wl.B, "T": wl.T, "layers": len(wl.specs), "params": n_params},
+            "config": config_dict(wl, n_params, args.gpus),
             "cpu_baseline": cb,
             "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(line))
@@ -205,6 +223,11 @@ def main():
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-extras", action="store_true",
+                    help="skip the per-phase power loops and the other workloads' timings (profiler captures)")
+    ap.add_argument("--fused-reduce", action="store_true",
+                    help="N > 1: end each step with ONE kernel per rank over the ranks' peer-mapped accumulators and "
+                         "replicas (dp_reduce_noise_adamw_step) instead of reduce-scatter + update + all-gather")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--blocks", type=int, default=24,
                     help="encoder blocks of the stack (24 = the benchmark workload; fewer only for profiler captures)")
@@ -251,7 +274,8 @@ def main():
     if args.blocks != 24:
         wl.specs = wl.specs[:6 * args.blocks] + [wl.specs[-1]]
     data = synth.generate(wl, seed=1000 + rank, device=dev)
-    step = pkg.DPStep(wl.specs, dev, wl.C, wl.sigma, wl.lr, wl.beta1, wl.beta2, wl.xi, wl.weight_decay, seed=0)
+    step = pkg.DPStep(wl.specs, dev, wl.C, wl.sigma, wl.lr, wl.beta1, wl.beta2, wl.xi, wl.weight_decay, seed=0,
+                      shard_world=world)
     step.theta.copy_(synth.initial_weights(step.n_flat, 0, dev))
     n_params = wl.n_params()
     lin_idx = [k for k, sp in enumerate(wl.specs) if sp.kind == "linear"]
@@ -266,7 +290,16 @@ def main():
     ws_rest = torch.empty(max(pkg.dp_workspace_bytes(ll_rest), 256), dtype=torch.uint8, device=dev)
     sq = torch.empty(wl.B, dtype=torch.float32, device=dev)
     clip = torch.empty(wl.B, dtype=torch.float32, device=dev)
-    sharded = ShardedUpdate(step, dist, world, rank) if world > 1 else None
+    sharded = None
+    if world > 1 and args.fused_reduce:
+        # every rank's accumulator and replica of theta mapped into this process (CUDA IPC; plain loads and stores)
+        from paper_2108_01624_b200.parallel import exchange_peer_buffers
+        peers = (exchange_peer_buffers(step.acc, dist, world, rank), exchange_peer_buffers(step.theta, dist, world, rank))
+        sharded = ShardedUpdate(step, dist, world, rank, peer_acc=peers[0], peer_theta=peers[1])
+    elif world > 1:
+        sharded = ShardedUpdate(step, dist, world, rank)
+    if sharded is not None:
+        sharded.time_phases()
     stream = torch.cuda.current_stream()
 
     if args.macro_microbatches > 0:
@@ -296,10 +329,11 @@ def main():
         if ev:
             ev[3].record(stream)
         step.examples_seen = wl.B * world
+        # the status word is read once after the loop, not with a host synchronisation in every step
         if sharded is None:
-            step.finish_macro_batch()
+            step.finish_macro_batch(check_status=False)
         else:
-            sharded.finish_macro_batch()
+            sharded.finish_macro_batch(check_status=False)
         if ev:
             ev[4].record(stream)
 
@@ -315,6 +349,8 @@ def main():
         raise RuntimeError("device status not clean after warm-up")
 
     evs = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(args.steps)]
+    if sharded is not None:
+        sharded.timings()          # drop the warm-up steps' records
     sampler = ClockSampler(local)
     sampler.start()
     l0 = pkg.dp_launch_count()
@@ -328,6 +364,8 @@ def main():
     barrier()
     launches = pkg.dp_launch_count() - l0
     clocks = sampler.stop()
+    if pkg.dp_poll_status() != 0:
+        raise RuntimeError("device status not clean after the timed steps")
     total_ms = t_start.elapsed_time(t_end)
     if dist is not None:
         t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
@@ -336,6 +374,11 @@ def main():
     ms_per_step = total_ms / args.steps
     value = wl.B * world / (ms_per_step * 1e-3)
     phases = np.array([[e[i].elapsed_time(e[i + 1]) for i in range(4)] for e in evs]).mean(axis=0)
+    # N > 1: the exchange inside the last phase (reduce-scatter | update | all-gather, or barrier | fused kernel |
+    # barrier), device milliseconds on this rank, mean over the timed steps
+    collective = sharded.timings() if sharded is not None else None
+    if collective is not None:
+        collective["way"] = "one kernel over peer memory" if args.fused_reduce else "reduce-scatter + all-gather, in place"
 
     peaks = measured_peaks()
     T, B = wl.T, wl.B
@@ -343,66 +386,214 @@ def main():
     ach_tf = flops_acc / (phases[1] * 1e-3) / 1e12
     bytes_acc = sum(2.0 * B * T * (wl.specs[k].d_in + wl.specs[k].d_out)
                     + 8.0 * wl.specs[k].d_in * wl.specs[k].d_out for k in lin_idx)
+    traffic = None if ACCUM_TRAFFIC_2BLOCKS_BYTES is None else ACCUM_TRAFFIC_2BLOCKS_BYTES * args.blocks / 2.0
     roofline = {"kernel": "clipped-accumulate GEMM (all linear layers, one call)", "bound": "tensor",
                 "achieved": ach_tf, "peak": peaks["tf_sustained"], "unit": "TFLOP/s",
                 "frac": ach_tf / peaks["tf_sustained"], "frac_of_burst": ach_tf / peaks["tf_burst"],
                 "peak_source": peaks["source"] + " (sustained bf16; kernel timed inside a long step)",
-                "traffic": ACCUM_TRAFFIC_BYTES if args.blocks == 24 else None,
+                "traffic": traffic, "traffic_source": "ncu capture of a 2-block launch, scaled by blocks / 2",
                 "algorithmic_bytes": bytes_acc}
     bytes_norm = sum(2.0 * B * T * (wl.specs[k].d_in + wl.specs[k].d_out) for k in lin_idx) \
         + sum(2.0 * 2 * B * T * wl.specs[k].d_out for k in rest_idx if wl.specs[k].kind == "layernorm") \
         + sum(2.0 * B * T * wl.specs[k].d_out + 4.0 * B * T for k in rest_idx if wl.specs[k].kind == "embedding")
     bytes_upd = 32.0 * step.n_flat
+    # algorithmic flops of the Gram norms: the upper triangle (with the diagonal) of each T x T Gram, i.e. half of
+    # 2 T^2 (d_in + d_out) up to the diagonal -- whatever the kernel executes
+    flops_gram = sum(2.0 * B * (T * (T + 1) / 2.0) * (wl.specs[k].d_in + wl.specs[k].d_out) for k in lin_idx)
+    tf_both = (flops_acc + flops_gram) / ((phases[0] + phases[1]) * 1e-3) / 1e12
+
+    def hbm(nbytes, ms):
+        gbs = nbytes / (ms * 1e-3) / 1e9
+        return {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                "frac": gbs / peaks["hbm_gbs"], "frac_of_nominal_8TBs": gbs / HBM_NOMINAL_GBS}
     extra = {
-        "norm_pass": {"bound": "hbm", "achieved": bytes_norm / (phases[0] * 1e-3) / 1e9, "peak": peaks["hbm_gbs"],
-                      "unit": "GB/s", "frac": bytes_norm / (phases[0] * 1e-3) / 1e9 / peaks["hbm_gbs"]},
-        "noise_adamw": {"bound": "hbm", "achieved": bytes_upd / (phases[3] * 1e-3) / 1e9, "peak": peaks["hbm_gbs"],
-                        "unit": "GB/s", "frac": bytes_upd / (phases[3] * 1e-3) / 1e9 / peaks["hbm_gbs"]},
+        "norm_pass": hbm(bytes_norm, phases[0]),
+        "noise_adamw": hbm(bytes_upd, phases[3]),
+        "gram_plus_accumulate": {"bound": "tensor", "achieved": tf_both, "unit": "TFLOP/s",
+                                 "algorithmic_flops": flops_acc + flops_gram,
+                                 "frac_of_sustained": tf_both / peaks["tf_sustained"],
+                                 "frac_of_burst": tf_both / peaks["tf_burst"],
+                                 "note": "flop-weighted over the norm pass and the accumulate GEMM; the norm pass is "
+                                         "bound by HBM (intensity T = 128 flop/B), so its time counts in full"},
     }
 
+    others = None
+    energy = None
+    if world == 1 and not args.no_extras:
+        energy = phase_energy(pkg, wl, local, stream, step,
+                              {"norms+clip": lambda: (pkg.dp_per_example_sqnorms(ll_lin, sq, False, ws),
+                                                      pkg.dp_per_example_sqnorms(ll_rest, sq, True, ws_rest),
+                                                      pkg.dp_clip_factors(sq, wl.C, clip)),
+                               "accumulate_linear": lambda: pkg.dp_clipped_accumulate(ll_lin, clip, ws),
+                               "noise_adamw": lambda: step.finish_macro_batch(batch_size=wl.B, check_status=False)},
+                              {"norms+clip": phases[0], "accumulate_linear": phases[1], "noise_adamw": phases[3]})
+        others = {"megabatch_proxy": megabatch_proxy(pkg, synth, wl, step, data, lin_idx, rest_idx,
+                                                     (ws, ws_rest, sq, clip), stream, rank, dev, n_micro=64)}
     e2e = None
     if not args.no_e2e and world == 1:
         e2e = run_e2e(pkg, synth, wl, data, one_step, make_lists, clip, stream, args.e2e_steps)
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         cpu_baseline = time_oracle(wl, data, n_params)
+        one = time_oracle(wl, data, n_params, budget_s=1.0, max_examples=1, threads=1)
+        cpu_baseline["single_thread"] = {"value": one["value"], "unit": UNIT, "cores": 1, "sample": one["sample"]}
+    if others is not None:
+        # the other workloads, after the 32 GB stack has been released
+        del data, ll_all, ll_lin, ll_rest, ws, ws_rest, step, sharded
+        torch.cuda.empty_cache()
+        others["bert_base_layer"] = small_workload(pkg, synth, "bert_base_layer", dev, stream, reps=50)
+        others["bert_large_layer_t512"] = long_sequence_paths(pkg, synth, dev, stream, args.warmup, max(args.steps, 10))
 
     if rank == 0:
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
                 "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
                 "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-                "config": {"workload": WORKLOAD if args.blocks == 24 else f"{WORKLOAD}[first {args.blocks} blocks only]",
-                           "B": B, "T": T, "layers": len(wl.specs), "params": n_params,
-                           "microbatches_per_step": 1, "parallelism": f"dp{world}",
-                           "l2": "inputs (32 GB per microbatch) far exceed L2; no flush"},
+                "config": config_dict(wl, n_params, world, args.blocks),
                 "phases_ms": {"norms+clip": phases[0], "accumulate_linear": phases[1],
                               "accumulate_ln_embedding": phases[2], "noise_adamw": phases[3]},
-                "roofline": roofline, "rooflines_other": extra, "cpu_baseline": cpu_baseline, "e2e": e2e,
+                "collective_ms": collective, "roofline": roofline, "rooflines_other": extra,
+                "phase_energy": energy, "other_workloads": others, "cpu_baseline": cpu_baseline, "e2e": e2e,
                 "gpu_launches": int(launches), "clocks": clocks}
         print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()
 
 
-def run_long_sequence_paths(args):
+def phase_energy(pkg, wl, device_index, stream, step, fns, in_step_ms, seconds=1.5):
+    """Each phase of the step repeated ALONE, back to back, for about `seconds`, with the clock and power sampler
+    running: its time per repetition, the mean board power and the median SM clock while it ran, and the energy of
+    one repetition (power x time).  Beside it the phase's time inside the step, where the phases alternate every
+    few milliseconds under one power cap."""
+    out = {}
+    for name, fn in fns.items():
+        reps = max(3, int(seconds * 1e3 / max(in_step_ms[name], 1e-3)))
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        sampler = ClockSampler(device_index)
+        sampler.start()
+        time.sleep(0.25)                       # idle samples first; they are cut off below
+        n_idle = len(sampler.rows)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(reps):
+            fn()
+        e1.record(stream)
+        torch.cuda.synchronize()
+        sampler.rows = sampler.rows[n_idle + 1:]          # the first sample under load straddles the start
+        c = sampler.stop()
+        ms = e0.elapsed_time(e1) / reps
+        out[name] = {"ms_alone": ms, "ms_in_step": in_step_ms[name], "repetitions": reps, "power_w": c["power_w"],
+                     "sm_mhz": c["sm_mhz"], "reasons": c["reasons"], "samples": c["samples"],
+                     "joules": None if c["power_w"] is None else c["power_w"] * ms * 1e-3}
+    if pkg.dp_poll_status() != 0:
+        raise RuntimeError("device status not clean after the per-phase loops")
+    return out
+
+
+def megabatch_proxy(pkg, synth, wl, step, data0, lin_idx, rest_idx, bufs, stream, rank, dev, n_micro):
+    """A short stand-in for the 8192-microbatch macro-step (`--macro-microbatches 8192` runs the real one): n_micro
+    microbatches rotating over two distinct resident inputs, accumulated in place, then one noise + AdamW pass."""
+    ws, ws_rest, sq, clip = bufs
+    second = synth.generate(wl, seed=1000 + rank, device=dev, microbatch=1)
+    lists = []
+    for d in (data0, second):
+        ll = step.layer_list(d)
+        lists.append((pkg.LayerList([ll.layers[k] for k in lin_idx]), pkg.LayerList([ll.layers[k] for k in rest_idx])))
+
+    def microbatch(k):
+        lin, rest = lists[k % 2]
+        pkg.dp_per_example_sqnorms(lin, sq, False, ws)
+        pkg.dp_per_example_sqnorms(rest, sq, True, ws_rest)
+        pkg.dp_clip_factors(sq, wl.C, clip)
+        pkg.dp_clipped_accumulate(lin, clip, ws)
+        pkg.dp_clipped_accumulate_after_sqnorms(rest, clip, ws_rest)
+
+    step.discard_macro_batch()
+    for k in range(3):
+        microbatch(k)
+    step.discard_macro_batch()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for k in range(n_micro):
+        microbatch(k)
+    step.examples_seen = wl.B * n_micro
+    step.finish_macro_batch(check_status=False)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    if pkg.dp_poll_status() != 0:
+        raise RuntimeError("device status not clean after the mega-batch proxy")
+    ms = e0.elapsed_time(e1)
+    del lists, second
+    torch.cuda.empty_cache()
+    return {"workload": f"bert_large x {n_micro} microbatches, then one noise + AdamW pass (stand-in for the "
+                        "8192-microbatch mega-batch)", "microbatches": n_micro, "examples": wl.B * n_micro,
+            "ms": ms, "ms_per_microbatch": ms / n_micro, "examples_per_s": wl.B * n_micro / (ms * 1e-3)}
+
+
+def small_workload(pkg, synth, name, dev, stream, reps):
+    """One of the smaller workloads through the same calls: per-phase device times over `reps` repetitions."""
+    wl = synth.workload(name)
+    data = synth.generate(wl, seed=0, device=dev)
+    step = pkg.DPStep(wl.specs, dev, wl.C, wl.sigma, wl.lr, wl.beta1, wl.beta2, wl.xi, wl.weight_decay, seed=0)
+    ll = step.layer_list(data)
+    ws = pkg.alloc_workspace(ll)
+    sq = torch.empty(wl.B, dtype=torch.float32, device=dev)
+    clip = torch.empty_like(sq)
+    flush = torch.empty(96 * 1024 * 1024, dtype=torch.float32, device=dev)     # 384 MB > L2, written between repetitions
+
+    def one(ev=None):
+        flush.fill_(0.0)
+        if ev:
+            ev[0].record(stream)
+        pkg.dp_per_example_sqnorms(ll, sq, False, ws)
+        pkg.dp_clip_factors(sq, wl.C, clip)
+        if ev:
+            ev[1].record(stream)
+        pkg.dp_clipped_accumulate_after_sqnorms(ll, clip, ws)
+        if ev:
+            ev[2].record(stream)
+        step.examples_seen = wl.B
+        step.finish_macro_batch(check_status=False)
+        if ev:
+            ev[3].record(stream)
+
+    for _ in range(3):
+        one()
+    torch.cuda.synchronize()
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(reps)]
+    for k in range(reps):
+        one(evs[k])
+    torch.cuda.synchronize()
+    if pkg.dp_poll_status() != 0:
+        raise RuntimeError("device status not clean")
+    ph = np.array([[e[i].elapsed_time(e[i + 1]) for i in range(3)] for e in evs]).mean(axis=0)
+    lin = [sp for sp in wl.specs if sp.kind == "linear"]
+    flops = sum(2.0 * wl.B * wl.T * sp.d_in * sp.d_out for sp in lin)
+    nbytes = sum(2.0 * wl.B * wl.T * (sp.d_in + sp.d_out) for sp in lin) \
+        + sum(4.0 * wl.B * wl.T * sp.d_out for sp in wl.specs if sp.kind == "layernorm")
+    total = float(ph.sum())
+    return {"workload": name, "B": wl.B, "T": wl.T, "params": wl.n_params(), "repetitions": reps,
+            "l2": "384 MB written between repetitions",
+            "ms": total, "examples_per_s": wl.B / (total * 1e-3),
+            "phases_ms": {"norms+clip": ph[0], "accumulate": ph[1], "noise_adamw": ph[2]},
+            "norms_GBs": nbytes / (ph[0] * 1e-3) / 1e9, "accumulate_TFLOPs": flops / (ph[1] * 1e-3) / 1e12}
+
+
+def long_sequence_paths(pkg, synth, dev, stream, warmup, reps):
     """The long-sequence crossover: one BERT-Large block at T=512, B=64.  Norms of the four linear layers with the
     path forced per layer (token Gram / materialised tiles) and auto-selected, then the clipped accumulate; each
-    call device-timed alone over `--steps` repetitions (inputs 1.07 GB, larger than L2)."""
-    import paper_2108_01624_b200 as pkg
+    call device-timed alone over `reps` repetitions (inputs 1.07 GB, larger than L2)."""
     from paper_2108_01624_b200 import binding as b
-    from paper_2108_01624_b200 import synth
-    dev = torch.device("cuda", 0)
-    torch.cuda.set_device(dev)
     wl = synth.workload("bert_large_layer_t512")
     data = [ld for ld in synth.generate(wl, seed=0, device=dev) if ld.spec.kind == "linear"]
     accs = [(torch.zeros(ld.spec.d_in, ld.spec.d_out, device=dev), torch.zeros(ld.spec.d_out, device=dev)) for ld in data]
     sq = torch.empty(wl.B, dtype=torch.float32, device=dev)
     clip = torch.empty_like(sq)
-    stream = torch.cuda.current_stream()
-    reps = max(args.steps, 10)
 
     def timed(fn):
-        for _ in range(args.warmup):
+        for _ in range(warmup):
             fn()
         torch.cuda.synchronize()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -434,9 +625,19 @@ def run_long_sequence_paths(args):
     torch.cuda.synchronize()
     if pkg.dp_poll_status() != 0:
         raise RuntimeError("device status not clean")
-    print(json.dumps({"workload": "bert_large_layer_t512", "B": B, "T": T, "linear_layers": len(data),
-                      "input_bytes": nbytes, "repetitions": reps, "timings": out,
-                      "gpu_launches": int(pkg.dp_launch_count() - l0), "peaks": measured_peaks()}))
+    return {"workload": "bert_large_layer_t512", "B": B, "T": T, "linear_layers": len(data),
+            "input_bytes": nbytes, "repetitions": reps, "timings": out,
+            "gpu_launches": int(pkg.dp_launch_count() - l0)}
+
+
+def run_long_sequence_paths(args):
+    import paper_2108_01624_b200 as pkg
+    from paper_2108_01624_b200 import synth
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    out = long_sequence_paths(pkg, synth, dev, torch.cuda.current_stream(), args.warmup, max(args.steps, 10))
+    out["peaks"] = measured_peaks()
+    print(json.dumps(out))
 
 
 def run_macro_step(args, pkg, synth, wl, step, sharded, dist, world, rank, dev, data0, lin_idx, rest_idx, bufs, stream):

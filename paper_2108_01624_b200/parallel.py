@@ -172,20 +172,27 @@ class ShardedUpdate:
 
     def _mark(self, k: int):
         if self._events is not None:
-            self._events[k].record()
-
-    def timings(self):
-        """Device milliseconds of the last finished macro-batch's phases, when `time_phases()` was called before it:
-        {"reduce": reduce-scatter (or the first barrier of the fused way), "update": the shard update,
-         "gather": all-gather + zeroing (or the closing barrier)}.  Synchronises the device."""
-        if self._events is None:
-            return None
-        torch.cuda.synchronize()
-        e = self._events
-        return {"reduce": e[0].elapsed_time(e[1]), "update": e[1].elapsed_time(e[2]), "gather": e[2].elapsed_time(e[3])}
+            if k == 0:
+                self._events.append([torch.cuda.Event(enable_timing=True) for _ in range(4)])
+            self._events[-1][k].record()
 
     def time_phases(self, on: bool = True):
-        self._events = [torch.cuda.Event(enable_timing=True) for _ in range(4)] if on and self.state.acc.is_cuda else None
+        """From now on every finished macro-batch records four device events around its three phases."""
+        self._events = [] if on and self.state.acc.is_cuda else None
+
+    def timings(self):
+        """Mean device milliseconds of the phases of the macro-batches finished since time_phases() (or since the
+        last call): {"reduce": reduce-scatter (or the opening barrier of the one-kernel way), "update": the shard
+        update, "gather": all-gather + zeroing (or the closing barrier), "macro_batches": how many}.
+        Synchronises the device; None when nothing was recorded."""
+        if not self._events:
+            return None
+        torch.cuda.synchronize()
+        ev, self._events = self._events, []
+        names = ("reduce", "update", "gather")
+        out = {n: sum(e[i].elapsed_time(e[i + 1]) for e in ev) / len(ev) for i, n in enumerate(names)}
+        out["macro_batches"] = len(ev)
+        return out
 
     # ---- the two ways to end a macro-batch ----------------------------------------------------------------------
     def _finish_fused(self):
