@@ -459,9 +459,9 @@ def main():
         dist.destroy_process_group()
 
 
-def phase_energy(pkg, wl, device_index, stream, step, fns, in_step_ms, seconds=1.5):
+def phase_energy(pkg, wl, device_index, stream, step, fns, in_step_ms, seconds=3.0):
     """Each phase of the step repeated ALONE, back to back, for about `seconds`, with the clock and power sampler
-    running: its time per repetition, the mean board power and the median SM clock while it ran, and the energy of
+    running (samples of the first 1.2 s dropped): its time per repetition, the mean board power and the median SM clock while it ran, and the energy of
     one repetition (power x time).  Beside it the phase's time inside the step, where the phases alternate every
     few milliseconds under one power cap."""
     out = {}
@@ -472,15 +472,19 @@ def phase_energy(pkg, wl, device_index, stream, step, fns, in_step_ms, seconds=1
         torch.cuda.synchronize()
         sampler = ClockSampler(device_index)
         sampler.start()
-        time.sleep(0.25)                       # idle samples first; they are cut off below
-        n_idle = len(sampler.rows)
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record(stream)
+        t_host = time.perf_counter()
+        n_settled = None
         for _ in range(reps):
             fn()
+            if n_settled is None and time.perf_counter() - t_host > 1.2:
+                stream.synchronize()           # the launches run ahead of the device: meet it once, then count samples
+                n_settled = len(sampler.rows)
         e1.record(stream)
         torch.cuda.synchronize()
-        sampler.rows = sampler.rows[n_idle + 1:]          # the first sample under load straddles the start
+        # the power reading is a moving average: only samples taken after more than a second under load count
+        sampler.rows = sampler.rows[(n_settled if n_settled is not None else 0) + 1:]
         c = sampler.stop()
         ms = e0.elapsed_time(e1) / reps
         out[name] = {"ms_alone": ms, "ms_in_step": in_step_ms[name], "repetitions": reps, "power_w": c["power_w"],

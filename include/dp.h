@@ -63,13 +63,15 @@ typedef enum { DP_F32 = 0, DP_BF16 = 1 } dp_dtype;
  *                 T <= 128; beyond, GRAM iff the multiply-accumulates it executes, 128 * 128 * (d_in + d_out) per
  *                 block pair of the upper triangle of the ceil(T/128)^2 token blocks, are at most 1.75 times
  *                 T * d_in * d_out;
- *                 embedding: GRAM whenever the tensor-core kernel accepts the layer (bf16, d_out % 64 == 0). */
+ *                 embedding: GRAM whenever the tensor-core kernel accepts the layer (bf16, d_out % 8 == 0). */
 typedef enum { DP_PATH_AUTO = 0, DP_PATH_GRAM = 1, DP_PATH_MATERIALIZED = 2 } dp_path;
-/* Which kernels a layer gets.  A bf16 LINEAR layer whose d_in and d_out are multiples of 64 and whose A and G are
- * 16-byte aligned runs on the tensor cores (norms and clipped sum); every other linear layer (fp32, other widths,
- * e.g. a vocabulary-sized output that was not padded to a multiple of 64) runs on plain CUDA-core kernels, which
- * give the same results and are far slower.  LAYERNORM and the EMBEDDING accumulate are bandwidth-bound kernels
- * for any width; they use 16-byte loads when d is a multiple of 8 (bf16) or 4 (fp32) and the tensors are aligned. */
+/* Which kernels a layer gets.  A bf16 LINEAR layer whose d_in and d_out are multiples of 8 (a token row is then a
+ * multiple of 16 bytes) and whose A and G are 16-byte aligned runs on the tensor cores (norms and clipped sum); widths
+ * that are also multiples of 64 take one tensor copy per operand tile, the others one copy per 64-feature group
+ * (the group that overhangs the width is filled with zeros).  Every other linear layer (fp32, other widths) runs on
+ * plain CUDA-core kernels, which give the same results and are far slower.  LAYERNORM and the EMBEDDING accumulate are
+ * bandwidth-bound kernels for any width; they use 16-byte loads when d is a multiple of 8 (bf16) or 4 (fp32) and
+ * the tensors are aligned. */
 
 /* One trainable layer of one microbatch.  B and T must be equal across the layers of a call. */
 typedef struct dp_layer {

@@ -350,3 +350,4 @@ def dp_set_wait_limit_cycles(cycles: int) -> None:
 def dp_selftest_wait_timeout(stream=None) -> None:
     """Enqueues the kernel whose waits nobody satisfies; dp_poll_status reports DP_ERR_TIMEOUT afterwards."""
     _check("dp_selftest_wait_timeout", lib().dp_selftest_wait_timeout(_stream(stream)))
+

@@ -4,7 +4,18 @@
 // kernels exclude.  Every reduction runs in a fixed order, so results are reproducible.
 #include "dp_internal.h"
 
+// Tunables of the column-sum kernel (overridable with -D for experiments).
+#ifndef DP_COLSUMS_MINBLOCKS
+#define DP_COLSUMS_MINBLOCKS 2          // resident CTAs per SM asked of the compiler (caps the registers per thread)
+#endif
+#ifndef DP_COLSUMS_UNROLL
+#define DP_COLSUMS_UNROLL 8             // token rows whose loads are issued together (8 with 2 CTAs per SM measured
+                                        // best: 6.15 against 6.31 ms for the norm pass; 3 or 4 CTAs with 2 or 4 rows: no gain)
+#endif
+
 namespace dpk {
+
+constexpr int kColsumsUnroll = DP_COLSUMS_UNROLL;
 
 template <typename T> __device__ __forceinline__ float ldf(const T* p);
 template <> __device__ __forceinline__ float ldf<float>(const float* p) { return __ldg(p); }
@@ -237,7 +248,7 @@ k_colsums_body(const T* __restrict__ X, const T* __restrict__ G, int Tn, int d, 
 #pragma unroll
     for (int k = 0; k < VEC; ++k) { sx[k] = 0.0f; sg[k] = 0.0f; }
     if (col < d) {
-#pragma unroll 4
+#pragma unroll kColsumsUnroll
       for (int t = tg; t < Tn; t += 4) {
         float g[VEC], x[VEC];
         VecLoad<T, VEC>::ld(Gi + (size_t)t * d + col, g);
@@ -283,7 +294,7 @@ struct ColBatch {
 };
 
 template <typename T, int VEC, bool WITH_X>
-__global__ void __launch_bounds__(512) k_colsums_b(const __grid_constant__ ColBatch P) {
+__global__ void __launch_bounds__(512, DP_COLSUMS_MINBLOCKS) k_colsums_b(const __grid_constant__ ColBatch P) {
   const ColTask& t = P.t[blockIdx.y];
   k_colsums_body<T, VEC, WITH_X>(static_cast<const T*>(t.X), static_cast<const T*>(t.G), P.T, t.d, t.out);
 }

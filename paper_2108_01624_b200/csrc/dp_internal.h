@@ -74,7 +74,7 @@ cudaError_t launch_fill_zero(float* p, long long n, cudaStream_t s);
 cudaError_t launch_reduce_partials(const float* partial, int B, int count, float* sqnorm, cudaStream_t s);
 
 // ---- tcgen05 / TMA kernels for bf16 layers (dp_umma.cu) ----------------------------------------
-// A layer qualifies when dtype is bf16, d_in and d_out are multiples of 64 and pointers are 16-byte aligned.
+// A layer qualifies when dtype is bf16, d_in and d_out are multiples of 8 and pointers are 16-byte aligned.
 bool umma_supported(const dp_layer& L);
 // Number of fp32 partial sums the squared-norm kernels write for these layers (per example).
 // The partial buffer is [B][count] and is summed by launch_reduce_partials.

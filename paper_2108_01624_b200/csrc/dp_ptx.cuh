@@ -51,14 +51,15 @@ constexpr int kStatusTimeout = 1;
 // issue slots and power that the tensor pipe could use).
 // `tag` and `aux` identify the wait in the diagnostic record that the first waiter to give up leaves behind
 // (status[1..5] = tag, block, aux, parity, thread), read on the host by dp_last_timeout_info.
-template <int SLEEP_NS = 0>
+__device__ __forceinline__ bool mbar_try_wait_cluster(uint64_t* bar, uint32_t parity);
+template <int SLEEP_NS = 0, bool CLUSTER_ACQUIRE = false>
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status,
                                           int tag = 0, int aux = 0) {
-  if (mbar_try_wait(bar, parity)) return true;
+  if (CLUSTER_ACQUIRE ? mbar_try_wait_cluster(bar, parity) : mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   for (uint32_t spin = 1;; ++spin) {
     if (SLEEP_NS > 0) __nanosleep(SLEEP_NS);
-    if (mbar_try_wait(bar, parity)) return true;
+    if (CLUSTER_ACQUIRE ? mbar_try_wait_cluster(bar, parity) : mbar_try_wait(bar, parity)) return true;
     if ((spin & 63u) == 0u) {
       if (*abort_flag) return false;
       if (clock64() - t0 > g_wait_limit_cycles) {
@@ -184,6 +185,29 @@ __device__ __forceinline__ void mbar_arrive_cluster(uint64_t* bar, uint32_t cta)
   uint32_t remote;
   asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(smem_u32(bar)), "r"(cta));
   asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(remote) : "memory");
+}
+// The same arrival with release semantics at cluster scope: everything the arriving thread wrote before it, and
+// what it observed other threads write (through a CTA barrier), is visible to whoever acquires the phase at cluster
+// scope.  It stalls the arriving thread until its earlier memory operations are done.
+__device__ __forceinline__ void mbar_arrive_cluster_release(uint64_t* bar, uint32_t cta) {
+  uint32_t remote;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(smem_u32(bar)), "r"(cta));
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(remote) : "memory");
+}
+__device__ __forceinline__ void fence_acq_rel_cluster() { asm volatile("fence.acq_rel.cluster;" ::: "memory"); }
+// try_wait with acquire semantics at cluster scope (the waiter consumes data that a thread of the PEER CTA released).
+__device__ __forceinline__ bool mbar_try_wait_cluster(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n"
+      ".reg .pred p;\n"
+      "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n"
+      "selp.u32 %0, 1, 0, p;\n"
+      "}\n"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
 }
 // TMEM of both CTAs of the pair; executed by one warp in each of the two CTAs.
 __device__ __forceinline__ void tmem_alloc_pair(uint32_t* dst_smem, uint32_t ncols) {

@@ -34,6 +34,14 @@ constexpr int kMaxLayers = kUmmaMaxLayers;
 #ifndef DP_ACCUM_ALIGN
 #define DP_ACCUM_ALIGN 1                // accumulate kernel: soft per-wave alignment of the CTA pairs
 #endif
+#ifndef DP_ACCUM_READY
+// accumulate kernel: how the worker warps of the odd CTA hand a rescaled G stage to the UMMA issuer in the even CTA
+//   0  every warp: fence.proxy.async, then a plain remote mbarrier.arrive (16 arrivals per stage)
+//   1  every warp: fence.proxy.async, fence.acq_rel.cluster, plain remote arrive (16 arrivals per stage)
+//   2  the eight warps of a CTA meet at a named barrier and ONE thread (rotating over the warps) arrives with
+//      release semantics at cluster scope (2 arrivals per stage); the issuer acquires at cluster scope
+#define DP_ACCUM_READY 0
+#endif
 #ifndef DP_TMA_L2_PROMOTION
 #define DP_TMA_L2_PROMOTION 2          // 0 none, 1 128 B, 2 256 B
 #endif
@@ -49,7 +57,8 @@ struct alignas(64) UmmaLayer {
   int partial_base;       // first per-example partial slot of this layer
   uint16_t tiles_m, tiles_n;   // tile kernels: tiles over d_out and over d_in
   uint8_t has_bias, is_emb;
-  uint8_t pad[18];        // to 320 bytes (a multiple of the tensor maps' 64-byte alignment)
+  uint8_t rag_g, rag_a;   // the width of G / A is not a multiple of 64: its map is the 3-D one (one 64-feature group per copy)
+  uint8_t pad[16];        // to 320 bytes (a multiple of the tensor maps' 64-byte alignment)
 };
 static_assert(sizeof(UmmaLayer) == 320, "UmmaLayer grew: 96 of them must fit the kernel parameter block");
 
@@ -76,11 +85,25 @@ __device__ __forceinline__ uint8_t* align1024(uint8_t* p) {
   return reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(p) + 1023) & ~uintptr_t(1023));
 }
 
+// One operand tile of `groups` 64-feature groups (each `group_bytes` apart in shared memory), token rows from
+// `row`, features from `f0` (a multiple of 64), example `ex`.  Widths that are multiples of 64 use the 4-D view of
+// the tensor (one copy for all groups).  Other widths (multiples of 8) cannot: a 64-feature group that overhangs
+// the row would run into the next token, so their map is the plain (feature, token, example) view, whose copies
+// are bounded by the width and read zeros beyond it, one copy per group.
+__device__ __forceinline__ void load_groups(uint8_t* dst, const CUtensorMap* map, uint64_t* bar, bool ragged, int groups,
+                                            int group_bytes, int f0, int row, int ex) {
+  if (!ragged) {
+    tma_load_4d(dst, map, bar, 0, row, f0 / 64, ex);
+  } else {
+    for (int g = 0; g < groups; ++g) tma_load_3d(dst + g * group_bytes, map, bar, f0 + 64 * g, row, ex);
+  }
+}
+
 // =================================================================================================
 // Gram kernel
 // =================================================================================================
 constexpr int G_GROUPS = 2;                      // 64-feature tiles per TMA copy and ring slot
-constexpr int G_SLOTS = 6;
+constexpr int G_SLOTS = 6;                       // (7 slots, or L2 prefetch of the tiles ahead of the ring: measured, no gain)
 constexpr int G_TILE_BYTES = 128 * 128;          // 128 tokens x 64 bf16 features, 128-byte swizzle
 constexpr int G_SLOT_BYTES = G_GROUPS * G_TILE_BYTES;
 constexpr int G_THREADS = 192;                   // warp 0: TMA, warp 1: MMA, warps 2..5: epilogue
@@ -92,6 +115,7 @@ struct GramCtl {
   int abort;
 };
 constexpr int G_SMEM = 1024 + G_SLOTS * G_SLOT_BYTES + (int)sizeof(GramCtl);
+static_assert(G_SMEM <= 232448, "over the shared memory of one CTA");
 
 // item -> (layer, example, token-block pair r <= c)
 __device__ __forceinline__ void gram_decode(const UmmaParams& P, int item, int npairs, int nblk, int& l, int& i, int& pair,
@@ -146,7 +170,8 @@ __global__ void __launch_bounds__(G_THREADS, 1) k_gram_sqnorm(const __grid_const
               const uint32_t slot = it % G_SLOTS, ph = (it / G_SLOTS) & 1u;
               if (!mbar_wait(&S->empty[slot], ph ^ 1u, abort_flag, P.status)) { alive = false; break; }
               mbar_arrive_expect_tx(&S->full[slot], (uint32_t)G_SLOT_BYTES);
-              tma_load_4d(tiles + slot * G_SLOT_BYTES, map, &S->full[slot], 0, (half ? c : r) * 128, k0 / 64, i);
+              load_groups(tiles + slot * G_SLOT_BYTES, map, &S->full[slot], which ? L.rag_g : L.rag_a, G_GROUPS,
+                          G_TILE_BYTES, k0, (half ? c : r) * 128, i);
               ++it;
             }
           }
@@ -593,8 +618,9 @@ k_tile_sqnorm_pair(const __grid_constant__ UmmaParams P) {
           // two boxes of 64 features x Q_BK tokens x 2 feature groups; tokens beyond T and groups beyond the
           // layer's width arrive as zeros
           mbar_arrive_expect_tx(&S->full[slot], (uint32_t)Q_STAGE_BYTES);
-          tma_load_4d(st, &L.mapG, &S->full[slot], 0, tb * Q_BK, (t.m0 + 128 * (int)rank) / 64, t.e);
-          tma_load_4d(st + Q_HALF_BYTES, &L.mapA, &S->full[slot], 0, tb * Q_BK, (t.n0 + 128 * (int)rank) / 64, t.e);
+          load_groups(st, &L.mapG, &S->full[slot], L.rag_g, 2, Q_ATOM_BYTES, t.m0 + 128 * (int)rank, tb * Q_BK, t.e);
+          load_groups(st + Q_HALF_BYTES, &L.mapA, &S->full[slot], L.rag_a, 2, Q_ATOM_BYTES, t.n0 + 128 * (int)rank,
+                      tb * Q_BK, t.e);
           ++it;
         }
       }
@@ -767,7 +793,7 @@ k_accum_pair(const __grid_constant__ UmmaParams P) {
     for (int s = 0; s < P_STAGES; ++s) {
       mbar_init(&S->full[s], 1);
       mbar_init(&S->empty[s], 1);
-      mbar_init(&S->ready[s], 16);
+      mbar_init(&S->ready[s], DP_ACCUM_READY == 2 ? 2 : 16);
     }
     mbar_init(&S->tmem_full, 1);
     mbar_init(&S->tmem_empty, 16);
@@ -814,8 +840,8 @@ k_accum_pair(const __grid_constant__ UmmaParams P) {
             // two boxes of 64 features x 64 tokens x (2 | 4) feature groups; tokens beyond T and feature groups
             // beyond the layer's width are outside the tensor and arrive as zeros
             mbar_arrive_expect_tx(&S->full[slot], (uint32_t)P_STAGE_BYTES);
-            tma_load_4d(st, &L.mapG, &S->full[slot], 0, tb * P_BK, mh / 64, e);
-            tma_load_4d(st + P_M_BYTES, &L.mapA, &S->full[slot], 0, tb * P_BK, nh / 64, e);
+            load_groups(st, &L.mapG, &S->full[slot], L.rag_g, 2, P_ATOM_BYTES, mh, tb * P_BK, e);
+            load_groups(st + P_M_BYTES, &L.mapA, &S->full[slot], L.rag_a, 4, P_ATOM_BYTES, nh, tb * P_BK, e);
             ++it;
           }
         }
@@ -840,7 +866,10 @@ k_accum_pair(const __grid_constant__ UmmaParams P) {
           for (int tb = 0; tb < n_tb; ++tb) {
             const uint32_t slot = it % P_STAGES, ph = (it / P_STAGES) & 1u;
             ++it;
-            if (!mbar_wait(&S->ready[slot], ph, abort_flag, P.status, 13, (int)it)) { alive = false; break; }
+            if (!mbar_wait<0, DP_ACCUM_READY != 0>(&S->ready[slot], ph, abort_flag, P.status, 13, (int)it)) {
+              alive = false;
+              break;
+            }
             tc_fence_after();
             const uint32_t am = smem_u32(tiles + slot * P_STAGE_BYTES), an = am + P_M_BYTES;
             const int left = P.T - tb * P_BK;
@@ -903,8 +932,10 @@ k_accum_pair(const __grid_constant__ UmmaParams P) {
           const uint32_t slot = it % P_STAGES, ph = (it / P_STAGES) & 1u;
           ++it;
           if (alive && !mbar_wait(&S->full[slot], ph, abort_flag, P.status, 14, (int)it)) alive = false;
+#if DP_ACCUM_READY != 2
           if (!alive) continue;
-          if (cf != 1.0f || need_bias) {
+#endif
+          if (alive && (cf != 1.0f || need_bias)) {
             uint8_t* base = tiles + slot * P_STAGE_BYTES + ta * P_ATOM_BYTES + kk * 128 + jp * 16;
 #pragma unroll
             for (int i4 = 0; i4 < P_BK / 16; ++i4) {   // rows kk, kk+16, ... of atom ta
@@ -925,8 +956,33 @@ k_accum_pair(const __grid_constant__ UmmaParams P) {
             }
             fence_proxy_async_smem();
           }
+#if DP_ACCUM_READY == 2
+          // one barrier per stage: all 256 workers have rescaled their share (and agree on whether anyone gave up)
+          {
+            uint32_t all_alive;
+            asm volatile(
+                "{\n"
+                ".reg .pred p, q;\n"
+                "setp.ne.b32 q, %1, 0;\n"
+                "bar.red.and.pred p, 3, 256, q;\n"
+                "selp.u32 %0, 1, 0, p;\n"
+                "}\n"
+                : "=r"(all_alive)
+                : "r"((uint32_t)alive)
+                : "memory");
+            alive = all_alive != 0;
+          }
+          if (alive && tt == (int)((it & 7u) << 5)) mbar_arrive_cluster_release(&S->ready[slot], 0u);
+#elif DP_ACCUM_READY == 1
+          __syncwarp();
+          if (lane == 0) {
+            fence_acq_rel_cluster();
+            mbar_arrive_cluster(&S->ready[slot], 0u);
+          }
+#else
           __syncwarp();
           if (lane == 0) mbar_arrive_cluster(&S->ready[slot], 0u);
+#endif
         }
       }
       if (need_bias) {      // uniform over the 256 worker threads; executed even after an abort
@@ -1030,12 +1086,13 @@ static bool encode_map3(CUtensorMap* map, const void* base, int B, int T, int d,
 }
 
 bool umma_supported(const dp_layer& L) {
+  // widths must be multiples of 8: a token row is then a multiple of 16 bytes, which the tensor maps require
   if (L.kind == DP_EMBEDDING) {   // mask-Gram norm only (the accumulate is a scatter, not a contraction)
-    return L.dtype == DP_BF16 && L.d_out % 64 == 0 && (reinterpret_cast<uintptr_t>(L.G) & 15u) == 0 &&
+    return L.dtype == DP_BF16 && L.d_out % 8 == 0 && (reinterpret_cast<uintptr_t>(L.G) & 15u) == 0 &&
            (long long)L.T * L.d_out * 2 < (1ll << 40);
   }
   if (L.kind != DP_LINEAR || L.dtype != DP_BF16) return false;
-  if (L.d_in % 64 != 0 || L.d_out % 64 != 0) return false;
+  if (L.d_in % 8 != 0 || L.d_out % 8 != 0) return false;
   if ((reinterpret_cast<uintptr_t>(L.A) | reinterpret_cast<uintptr_t>(L.G)) & 15u) return false;
   if ((long long)L.T * (L.d_in > L.d_out ? L.d_in : L.d_out) * 2 >= (1ll << 40)) return false;
   return true;
@@ -1091,9 +1148,13 @@ static bool accum_kernel_ready();
 // A box may be taller than T or span more groups than the layer has: what lies outside the tensor is zero-filled.
 static bool fill_layer(UmmaLayer& U, const dp_layer& L, int box_rows, int groups_g, int groups_a) {
   const bool emb = L.kind == DP_EMBEDDING;
-  if (!encode_map4(&U.mapG, L.G, L.B, L.T, L.d_out, box_rows, groups_g)) return false;
+  U.rag_g = L.d_out % 64 != 0;
+  U.rag_a = !emb && L.d_in % 64 != 0;
+  if (!(U.rag_g ? encode_map3(&U.mapG, L.G, L.B, L.T, L.d_out, box_rows)
+                : encode_map4(&U.mapG, L.G, L.B, L.T, L.d_out, box_rows, groups_g))) return false;
   if (emb) U.mapA = U.mapG;      // never used: an embedding streams no A operand (d_in = 0 below)
-  else if (!encode_map4(&U.mapA, L.A, L.B, L.T, L.d_in, box_rows, groups_a)) return false;
+  else if (!(U.rag_a ? encode_map3(&U.mapA, L.A, L.B, L.T, L.d_in, box_rows)
+                     : encode_map4(&U.mapA, L.A, L.B, L.T, L.d_in, box_rows, groups_a))) return false;
   U.acc_w = L.acc_w;
   U.acc_b = L.acc_b;
   U.ids = emb ? L.ids : nullptr;

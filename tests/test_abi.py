@@ -148,10 +148,10 @@ def test_accumulate_schedule_splits_large_groups_and_launches(lib):
     assert rc == 2 and launch[:96] == [0] * 96 and launch[96:] == [1] * 34
     assert splits[:2] == [2, 2] and slots[:2] == [3 * 74, 74]      # 192 items in 3 waves, 68 items in 1
     assert sorted(start[:96]) == [2 * k for k in range(96)] and sorted(start[96:]) == [2 * k for k in range(34)]
-    # layers the tensor-core GEMM does not take (fp32, widths not a multiple of 64) are left out
-    L = _fake_bf16_linears([(64, 64), (72, 40)], 3, 32)
+    # widths that are multiples of 8 go to the tensor-core GEMM (a 72 x 40 layer is one tile); others are left out
+    L = _fake_bf16_linears([(64, 64), (72, 40), (68, 40)], 3, 32)
     rc, start, launch, _, _ = _schedule(lib, L, 74)
-    assert rc == 1 and start[1] == -1 and launch[1] == -1
+    assert rc == 1 and launch[:2] == [0, 0] and start[0] != start[1] and start[2] == -1 and launch[2] == -1
     # argument checks
     assert lib.dp_accumulate_schedule(C.cast(L, C.c_void_p), 2, 0, 256, 256, 256, 256, 1) == -1
 

@@ -157,6 +157,29 @@ def test_tensor_core_tile_edges(B, T):
     check_against_checker(data, C, [b.DP_PATH_MATERIALIZED] * len(WIDE))
 
 
+RAGGED = [LayerSpec(LINEAR, 200, 72, True, "r200x72"),        # widths that are multiples of 8 but not of 64:
+          LayerSpec(LINEAR, 136, 264, False, "r136x264"),     # the last 64-feature group overhangs the row and must
+          LayerSpec(LINEAR, 584, 328, True, "r584x328"),      # arrive as zeros; tiles overhang as well
+          LayerSpec(LINEAR, 1096, 200, True, "r1096x200"),
+          LayerSpec(LINEAR, 64, 40, True, "r64x40"),          # one operand ragged, the other not
+          LayerSpec(LINEAR, 8, 8, True, "r8x8"),
+          LayerSpec(EMBEDDING, 30, 200, False, "emb200")]
+
+
+@pytest.mark.parametrize("B,T", [(1, 1), (5, 16), (4, 64), (3, 130), (2, 300)])
+def test_tensor_core_ragged_widths(B, T):
+    """bf16 widths with d % 8 == 0 and d % 64 != 0 on the tensor-core kernels: every norm path and the accumulate."""
+    data = random_layers(RAGGED, B, T, torch.bfloat16, DEV, seed=300 * B + T, g_scale=0.02, vocab_dup=9)
+    ol = to_oracle_layers(data)
+    C = float(np.sqrt(np.median(O.per_example_sqnorms(ol))))
+    ll, _ = make_layer_list(data, DEV)
+    units = torch.cuda.get_device_properties(0).multi_processor_count // 2
+    assert all(x >= 0 for x in b.dp_accumulate_schedule(ll, units)["launch"][:6])     # they are on the tensor-core GEMM
+    check_against_checker(data, C)
+    check_against_checker(data, C, [b.DP_PATH_GRAM] * len(RAGGED))
+    check_against_checker(data, C, [b.DP_PATH_MATERIALIZED] * len(RAGGED))
+
+
 @pytest.mark.parametrize("B,T", [(3, 129), (2, 256), (3, 300), (2, 384), (2, 640), (1, 700), (2, 2050)])
 def test_long_examples_gram_and_tiles(B, T):
     """More than one 128-token block per example: the Gram kernel pairs the column blocks of every row block
