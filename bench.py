@@ -254,12 +254,20 @@ def main():
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
+    # One rank per GPU.  With fewer GPUs than ranks (a functional check of the N > 1 path on one GPU; no kernel of
+    # this library waits for another rank) the ranks share devices, and DP_BENCH_BACKEND=gloo replaces NCCL, which
+    # refuses two ranks on one device.
+    local = local % max(1, torch.cuda.device_count())
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
     dist = None
     if world > 1:
         import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=dev)
+        backend = os.environ.get("DP_BENCH_BACKEND", "nccl")
+        if backend == "nccl":
+            dist.init_process_group("nccl", device_id=dev)
+        else:
+            dist.init_process_group(backend)
 
     import paper_2108_01624_b200 as pkg
     from paper_2108_01624_b200 import build as builder
@@ -338,9 +346,10 @@ def main():
             ev[4].record(stream)
 
     def barrier():
+        torch.cuda.synchronize()
         if dist is not None:
             dist.barrier()
-        torch.cuda.synchronize()
+            torch.cuda.synchronize()
 
     for _ in range(args.warmup):
         one_step()
@@ -456,6 +465,11 @@ def main():
                 "gpu_launches": int(launches), "clocks": clocks}
         print(json.dumps(line))
     if dist is not None:
+        if args.fused_reduce:          # unmap the peers' buffers before any owner exits
+            barrier()
+            sharded = peers = None
+            torch.cuda.ipc_collect()
+            barrier()
         dist.destroy_process_group()
 
 
@@ -673,9 +687,10 @@ def run_macro_step(args, pkg, synth, wl, step, sharded, dist, world, rank, dev, 
             sharded.finish_macro_batch()
 
     def barrier():
+        torch.cuda.synchronize()
         if dist is not None:
             dist.barrier()
-        torch.cuda.synchronize()
+            torch.cuda.synchronize()
 
     for k in range(max(args.warmup, 3)):
         microbatch(k)
