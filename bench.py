@@ -32,7 +32,7 @@ if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of one k_accum_pair launch over TWO encoder blocks
-# (`--blocks 2`, 2.7 GB on the device), from the ncu capture summarised in profiles/k_accum_pair_2blocks_full.md.
+# (`--blocks 2`, 2.7 GB on the device), from an `ncu --set full` capture of that small case.
 # The kernel's traffic grows with the number of blocks (every block's operands are read once, its accumulators read
 # and written once), so a launch over n blocks is reported as this figure x n / 2.  Not to be re-taken on the full
 # 32 GB workload.  Set to None whenever that kernel changes until the capture has been repeated.
