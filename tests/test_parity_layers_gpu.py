@@ -395,6 +395,29 @@ def test_unsplit_accumulate_is_bitwise_repeatable():
             assert abs(float(acc[0][p, q]) - ref) <= 0.01 * scale + 1e-12
 
 
+@pytest.mark.parametrize("dtype,slack", [(torch.bfloat16, 2.0 ** -8), (torch.float32, 1e-5)])
+def test_each_clipped_contribution_is_bounded_by_C(dtype, slack):
+    """The sensitivity that the noise is calibrated to: one example's clipped contribution to the whole accumulator
+    (every layer kind) has norm at most C -- up to the rounding of c * G to bf16 on the tensor-core path (2^-9 per
+    element, hence per norm) plus the 1e-3 tolerance of the clip factor's own norm.  One example per call, so the
+    accumulator IS that contribution."""
+    specs = SMALL + WIDE[:2]
+    C = 0.37
+    for seed in range(4):
+        data = random_layers(specs, 1, 96, dtype, DEV, seed=400 + seed, g_scale=3.0, vocab_dup=5)
+        ll, accs = make_layer_list(data, DEV)
+        n, c, ws = gpu_norms_clip(ll, C)
+        assert float(c[0]) < 1.0                              # the example clips
+        b.dp_clipped_accumulate(ll, c, ws)
+        total = np.sqrt(sum(float((x.double() ** 2).sum()) for acc in accs for x in acc))
+        n_ref = float(O.per_example_sqnorms(to_oracle_layers(data))[0])
+        true_c = min(1.0, C / np.sqrt(n_ref))
+        assert total <= C * (1 + slack) * (float(c[0]) / true_c), (total, C)
+        assert total <= C * (1 + slack + CLIP_TOL)
+        assert total >= C * (1 - slack - CLIP_TOL)            # and it is not over-clipped either
+    assert b.dp_poll_status() == 0
+
+
 def test_workspace_too_small_is_refused():
     data = random_layers(SMALL, 2, 16, torch.bfloat16, DEV, seed=2)
     ll, _ = make_layer_list(data, DEV)
