@@ -6,6 +6,8 @@
 //                       K-major 128x64 tiles, two per TMA copy.  For a token embedding the input is one-hot, so
 //                       A_i A_i^T is the token-id equality mask: only G_i G_i^T is formed on the tensor cores and
 //                       the epilogue multiplies it by [id_t == id_s] (integer compares; any T).
+//   k_gram_sqnorm_short the same for T <= 112 with copies as high as the example is long (T rounded up to 16) and as many
+//                       64-feature groups per copy as fit a ring slot, and 128 x T' x 16 UMMAs.
 //   k_gram_sqnorm_wide  the same identity for T > 128: a row block against two column blocks per item
 //                       (128x256 UMMAs), upper triangle of the block grid only.
 //   k_tile_sqnorm_pair  the materialised-tile norm on CTA pairs: 256 (d_out) x 256 (d_in) tiles of ONE example's
@@ -66,6 +68,7 @@ struct UmmaParams {
   UmmaLayer L[kMaxLayers];
   int n_layers, total_items, B, T;
   int splits;             // accumulate: number of example ranges a tile is split into
+  int box_rows, box_groups;   // short-example Gram kernel: token rows and 64-feature groups of one copy
   int partial_stride;
   unsigned int* wave_sync;  // accumulate: arrival counter of the soft per-wave alignment (zeroed before the launch)
   long long align_limit;    // accumulate: longest wait at a wave boundary, in SM cycles (a few tile durations)
@@ -281,6 +284,160 @@ __global__ void __launch_bounds__(G_THREADS, 1) k_gram_sqnorm(const __grid_const
       for (int o = 16; o > 0; o >>= 1) sum += __shfl_down_sync(0xffffffffu, sum, o);
       if (lane == 0)
         P.partial[(size_t)i * P.partial_stride + L.partial_base + pair * 4 + (int)q] = (r == c) ? sum : 2.0f * sum;
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    __syncwarp();
+    tc_fence_after();
+    tmem_dealloc(tmem_base, 512);
+  }
+}
+
+// =================================================================================================
+// Gram kernel for short examples (T <= 112: the masked positions of a masked-LM head, a pooler's single token)
+//
+// The same identity and roles as k_gram_sqnorm with one token block per example, but a copy is `rows` tokens high
+// (T rounded up to 16) and carries as many 64-feature groups as fit the 32 KB ring slot, so that a short example
+// does not pay for 128-token boxes of mostly zero fill (the copies, whose cost is per instruction and per byte
+// written to shared memory, set the pace there), and the UMMAs are 128 x rows x 16.  Only the first `rows` rows
+// of a tile are written; the UMMA's M operand reads 128, so accumulator rows from `rows` on hold whatever the
+// ring held before and the epilogue leaves the lanes of tokens beyond T out.  Columns below `rows` are clean
+// (tokens between T and `rows` arrive as zeros).
+// =================================================================================================
+// The M operand of a UMMA spans 128 rows (16 KB) from the start of a group, which for the last groups of a slot
+// reaches into the next slot and, for the last slot, beyond the ring: a pad of one tile keeps those reads inside the
+// CTA's shared memory (what they return feeds accumulator rows that nobody reads).
+constexpr int G_SMEM_SHORT = 1024 + G_SLOTS * G_SLOT_BYTES + G_TILE_BYTES + (int)sizeof(GramCtl);
+static_assert(G_SMEM_SHORT <= 232448, "over the shared memory of one CTA");
+
+__global__ void __launch_bounds__(G_THREADS, 1) k_gram_sqnorm_short(const __grid_constant__ UmmaParams P) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* tiles = align1024(smem_raw);
+  GramCtl* S = reinterpret_cast<GramCtl*>(tiles + G_SLOTS * G_SLOT_BYTES + G_TILE_BYTES);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  volatile int* abort_flag = &S->abort;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < G_SLOTS; ++s) { mbar_init(&S->full[s], 1); mbar_init(&S->empty[s], 1); }
+    for (int b = 0; b < 2; ++b) { mbar_init(&S->tmem_full[b], 1); mbar_init(&S->tmem_empty[b], 4); }
+    mbar_init(&S->drain, 1);
+    S->abort = 0;
+    fence_mbar_init();
+  }
+  if (warp == 1) { tmem_alloc(&S->tmem_base, 512); tmem_relinquish(); }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = S->tmem_base;
+  const int rows = P.box_rows, groups = P.box_groups;      // rows: a multiple of 16 below 128; groups * rows <= 256
+  const int group_bytes = rows * 128;
+  const uint32_t slot_tx = (uint32_t)(groups * group_bytes);
+
+  if (warp == 0) {
+    if (lane == 0) {   // ---------------- TMA producer ----------------
+      uint32_t it = 0;
+      bool alive = true;
+      for (int item = blockIdx.x; item < P.total_items && alive; item += gridDim.x) {
+        const int l = find_layer(P, item), i = item - P.L[l].item_start;
+        const UmmaLayer& L = P.L[l];
+        for (int which = 0; which < 2 && alive; ++which) {
+          const CUtensorMap* map = which ? &L.mapG : &L.mapA;
+          const int d = which ? L.d_out : L.d_in;
+          for (int k0 = 0; k0 < d; k0 += 64 * groups) {
+            const uint32_t slot = it % G_SLOTS, ph = (it / G_SLOTS) & 1u;
+            if (!mbar_wait(&S->empty[slot], ph ^ 1u, abort_flag, P.status, 31, (int)it)) { alive = false; break; }
+            mbar_arrive_expect_tx(&S->full[slot], slot_tx);
+            load_groups(tiles + slot * G_SLOT_BYTES, map, &S->full[slot], which ? L.rag_g : L.rag_a, groups, group_bytes,
+                        k0, 0, i);
+            ++it;
+          }
+        }
+      }
+      const uint32_t pending = it < (uint32_t)G_SLOTS ? it : (uint32_t)G_SLOTS;
+      for (uint32_t k = 0; k < pending; ++k) {
+        const uint32_t j = it - 1 - k;
+        mbar_wait_drain(&S->full[j % G_SLOTS], (j / G_SLOTS) & 1u, P.status);
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {   // ---------------- MMA issuer ----------------
+      const uint32_t idesc = idesc_bf16_f32(128, rows, false, false);
+      uint32_t it = 0, tile_it = 0;
+      bool alive = true;
+      for (int item = blockIdx.x; item < P.total_items && alive; item += gridDim.x, ++tile_it) {
+        const int l = find_layer(P, item);
+        const UmmaLayer& L = P.L[l];
+        const uint32_t buf = tile_it & 1u, tph = (tile_it >> 1) & 1u;
+        if (!mbar_wait(&S->tmem_empty[buf], tph ^ 1u, abort_flag, P.status, 32, (int)tile_it)) { alive = false; break; }
+        tc_fence_after();
+        for (int which = 0; which < 2 && alive; ++which) {
+          const int d = which ? L.d_out : L.d_in;
+          const uint32_t d_tmem = tmem_base + buf * 256u + (uint32_t)which * 128u;
+          for (int k0 = 0; k0 < d; k0 += 64 * groups) {
+            const uint32_t sr = it % G_SLOTS, pr = (it / G_SLOTS) & 1u;
+            ++it;
+            if (!mbar_wait(&S->full[sr], pr, abort_flag, P.status, 33, (int)it)) { alive = false; break; }
+            tc_fence_after();
+            const uint32_t a0 = smem_u32(tiles + sr * G_SLOT_BYTES);
+            for (int g = 0; g < groups && k0 + 64 * g < d; ++g) {
+#pragma unroll
+              for (int k4 = 0; k4 < 4; ++k4) {
+                const uint64_t desc = smem_desc_sw128(a0 + g * group_bytes + k4 * 32, 16, 1024);
+                umma_bf16(d_tmem, desc, desc, idesc, (k0 | g | k4) ? 1u : 0u);
+              }
+            }
+            umma_commit(&S->empty[sr]);
+          }
+        }
+        if (alive) umma_commit(&S->tmem_full[buf]);
+      }
+      umma_commit(&S->drain);
+      mbar_wait_drain(&S->drain, 0u, P.status);
+    }
+  } else {   // ---------------- epilogue warps 2..5 ----------------
+    const uint32_t q = (uint32_t)warp & 3u;
+    const int trow = (int)q * 32 + lane;
+    uint32_t tile_it = 0;
+    bool alive = true;
+    for (int item = blockIdx.x; item < P.total_items; item += gridDim.x, ++tile_it) {
+      const int l = find_layer(P, item), i = item - P.L[l].item_start;
+      const UmmaLayer& L = P.L[l];
+      const uint32_t buf = tile_it & 1u, tph = (tile_it >> 1) & 1u;
+      if (alive) alive = __all_sync(0xffffffffu, mbar_wait(&S->tmem_full[buf], tph, abort_flag, P.status, 34, (int)tile_it));
+      if (!alive) continue;
+      tc_fence_after();
+      const float bias1 = L.has_bias ? 1.0f : 0.0f;
+      const int32_t* idrow = L.is_emb ? L.ids + (size_t)i * P.T : nullptr;
+      const int32_t my_id = (L.is_emb && trow < P.T) ? __ldg(idrow + trow) : -1;
+      float sum = 0.0f;
+      if ((int)q * 32 < rows) {                       // warps whose lanes all lie beyond the box have nothing to add
+#pragma unroll 1
+        for (int ch = 0; ch * 32 < rows; ++ch) {
+          uint32_t pv[32], qv[32];
+          const uint32_t ta = tmem_base + ((q * 32u) << 16) + buf * 256u + (uint32_t)ch * 32u;
+          if (!L.is_emb) tmem_ld_32x32(ta, pv);
+          tmem_ld_32x32(ta + 128u, qv);
+          tmem_ld_wait();
+          if (trow < P.T) {                            // lanes of tokens beyond T hold stale accumulator rows
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+              const int s = ch * 32 + j;
+              if (s < P.T) {
+                if (L.is_emb) sum += (__ldg(idrow + s) == my_id) ? __uint_as_float(qv[j]) : 0.0f;
+                else sum = fmaf(__uint_as_float(pv[j]) + bias1, __uint_as_float(qv[j]), sum);
+              }
+            }
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&S->tmem_empty[buf]);
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) sum += __shfl_down_sync(0xffffffffu, sum, o);
+      if (lane == 0) P.partial[(size_t)i * P.partial_stride + L.partial_base + (int)q] = sum;
     }
   }
   tc_fence_before();
@@ -1173,7 +1330,8 @@ static bool sqnorm_kernels_ready() {
   const int dev = current_device();
   if (dev < 0) return false;
   if (!state[dev])
-    state[dev] = (ensure_smem(k_gram_sqnorm, G_SMEM) && ensure_smem(k_gram_sqnorm_wide, W_SMEM) &&
+    state[dev] = (ensure_smem(k_gram_sqnorm, G_SMEM) && ensure_smem(k_gram_sqnorm_short, G_SMEM_SHORT) &&
+                  ensure_smem(k_gram_sqnorm_wide, W_SMEM) &&
                   ensure_smem(k_tile_sqnorm_pair, Q_SMEM)) ? 1 : -1;
   return state[dev] > 0;
 }
@@ -1243,6 +1401,10 @@ int launch_umma_sqnorms(const dp_layer* layers, const int* idx, int n, const int
       if (counted(1) != cudaSuccess) return DP_ERR_CUDA;
     }
   }
+  // Short examples (one token block that is mostly empty): copies of T rounded up to 16 token rows, as many feature
+  // groups per copy as fit a ring slot
+  const int short_rows = T <= 112 ? ((T + 15) / 16) * 16 : 0;
+  const int short_groups = short_rows ? 256 / short_rows : 0;
   for (int pass = 0; pass < 2; ++pass) {             // pass 0: one-block-pair Gram layers, pass 1: materialised tiles
     const bool gram = pass == 0;
     int k = 0;
@@ -1257,7 +1419,10 @@ int launch_umma_sqnorms(const dp_layer* layers, const int* idx, int n, const int
         const long long add = (long long)B * (gram ? gram_pairs(T) : tile_count(L));
         if (items + add > 0x7fffffffll) break;
         UmmaLayer& U = P.L[P.n_layers];
-        if (!(gram ? fill_layer(U, L, 128, G_GROUPS, G_GROUPS) : fill_layer(U, L, Q_BK, 2, 2))) return DP_ERR_CUDA;
+        if (!(gram ? fill_layer(U, L, short_rows ? short_rows : 128, short_rows ? short_groups : G_GROUPS,
+                                short_rows ? short_groups : G_GROUPS)
+                   : fill_layer(U, L, Q_BK, 2, 2)))
+          return DP_ERR_CUDA;
         if (!gram) {
           U.tiles_m = (uint16_t)ceil_div(L.d_out, 256);
           U.tiles_n = (uint16_t)ceil_div(L.d_in, 256);
@@ -1279,7 +1444,11 @@ int launch_umma_sqnorms(const dp_layer* layers, const int* idx, int n, const int
       P.partial = partial;
       P.status = status;
       const int grid = P.total_items < sm_count() ? P.total_items : sm_count();
-      if (gram) {
+      P.box_rows = short_rows;
+      P.box_groups = short_groups;
+      if (gram && short_rows) {
+        k_gram_sqnorm_short<<<grid, G_THREADS, G_SMEM_SHORT, s>>>(P);
+      } else if (gram) {
         k_gram_sqnorm<<<grid, G_THREADS, G_SMEM, s>>>(P);
       } else {
         const int units = sm_count() / 2;
