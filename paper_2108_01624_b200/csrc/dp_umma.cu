@@ -44,6 +44,10 @@ constexpr int kMaxLayers = kUmmaMaxLayers;
 //      release semantics at cluster scope (2 arrivals per stage); the issuer acquires at cluster scope
 #define DP_ACCUM_READY 0
 #endif
+#ifndef DP_ACCUM_A_REUSE
+#define DP_ACCUM_A_REUSE 1             // accumulate kernel: the two UMMAs of a k-step share the G tile through the operand
+                                       // collector (16.03-16.13 against 16.11-16.19 ms per launch sustained, six alternating runs)
+#endif
 #ifndef DP_TMA_L2_PROMOTION
 #define DP_TMA_L2_PROMOTION 2          // 0 none, 1 128 B, 2 256 B
 #endif
@@ -1034,11 +1038,19 @@ k_accum_pair(const __grid_constant__ UmmaParams P) {
 #pragma unroll
               for (int k4 = 0; k4 < P_BK / 16; ++k4) {
                 const uint64_t adesc = smem_desc_sw128(am + k4 * 2048, P_ATOM_BYTES, 1024);
+#if DP_ACCUM_A_REUSE
+                umma_bf16_pair_a_reuse<true>(tmem_base, adesc, smem_desc_sw128(an + k4 * 2048, P_ATOM_BYTES, 1024), IDESC,
+                                             acc | (uint32_t)k4);
+                umma_bf16_pair_a_reuse<false>(tmem_base + 256u, adesc,
+                                              smem_desc_sw128(an + 2 * P_ATOM_BYTES + k4 * 2048, P_ATOM_BYTES, 1024), IDESC,
+                                              acc | (uint32_t)k4);
+#else
 #pragma unroll
                 for (int j = 0; j < 2; ++j)
                   umma_bf16_pair(tmem_base + (uint32_t)j * 256u, adesc,
                                  smem_desc_sw128(an + j * 2 * P_ATOM_BYTES + k4 * 2048, P_ATOM_BYTES, 1024), IDESC,
                                  acc | (uint32_t)k4);
+#endif
               }
             } else {                                   // ragged last stage or narrow tile: only the UMMAs that carry data
               const int nk = left >= P_BK ? P_BK / 16 : (left + 15) >> 4, nj = t.narrow ? 1 : 2;
