@@ -107,6 +107,7 @@ class ShardedUpdate:
         self.poll_fn = poll_fn or self._poll_library
         self.nccl = dist.get_backend() == "nccl"
         self._events = None
+        self._in_place = True          # collectives on aliased buffers; cleared if the process group refuses them
         if peer_acc is None:
             self.acc_full = self._padded(state, "acc")
             self.theta_full = self._padded(state, "theta")
@@ -215,17 +216,29 @@ class ShardedUpdate:
         mine_theta = theta[r * per:(r + 1) * per]
         lo, hi = self.lo, self.hi
         self._mark(0)
-        if self.nccl:
-            dist.reduce_scatter_tensor(mine_acc, acc)           # in place: the output is this rank's slice of the input
-        else:
+        if self.nccl and self._in_place:
+            try:
+                dist.reduce_scatter_tensor(mine_acc, acc)       # in place: the output is this rank's slice of the input
+            except (RuntimeError, ValueError):                  # a front end that refuses aliased buffers: stage once
+                self._in_place = False
+        if self.nccl and not self._in_place:
+            out = torch.empty_like(mine_acc)
+            dist.reduce_scatter_tensor(out, acc)
+            mine_acc.copy_(out)
+        elif not self.nccl:
             dist.all_reduce(acc)
         self._mark(1)
         if hi > lo:
             self.update_fn(s.theta[lo:hi], s.m[lo:hi], s.v[lo:hi], acc[lo:hi], lo, s.examples_seen, s.t)
         self._mark(2)
-        if self.nccl:
-            dist.all_gather_into_tensor(theta, mine_theta)      # in place: the input is this rank's slice of the output
-        else:
+        if self.nccl and self._in_place:
+            try:
+                dist.all_gather_into_tensor(theta, mine_theta)  # in place: the input is this rank's slice of the output
+            except (RuntimeError, ValueError):
+                self._in_place = False
+        if self.nccl and not self._in_place:
+            dist.all_gather_into_tensor(theta, mine_theta.clone())
+        elif not self.nccl:
             dist.all_gather([theta[k * per:(k + 1) * per] for k in range(self.world)], mine_theta.clone())
         # the other ranks' shards of the accumulator still hold this rank's sums
         acc[:r * per].zero_()
